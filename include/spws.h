@@ -1,0 +1,175 @@
+/* spws -- sparse-workspace kernels for NVIDIA B200 (sm_100a): C ABI.
+ *
+ * The library evaluates sparse tensor expressions whose result is scattered into a compressed
+ * sparse output through a per-row workspace (arXiv 2404.04541, "Compilation of Modular and
+ * General Sparse Workspaces"):
+ *
+ *   row-wise SpGEMM          C(i,j)   = sum_k A(i,k)   * B(k,j)    A, B, C in CSR
+ *   tensor-times-matrix      C(i,j,l) = sum_k A(i,j,k) * B(k,l)    A, C in CSF, B in CSR
+ *
+ * following the paper's statement of the problem: an expression over named index variables
+ * (Sec. 3), a level format per operand (Sec. 2.1, Fig. 4) and a workspace policy (Sec. 6.1:
+ * the workspace tensor's format and policy; Sec. 6.2: dense-workspace optimisation).  Both
+ * expressions are first-order scatters (Sec. 2.2): the loop order i -> k -> j differs from the
+ * output order i -> j only by the reduction variable, so every output row (every (i,j) fibre,
+ * after hoisting the shared outer loops, Sec. 6.2) owns a first-order workspace along the last
+ * index.
+ *
+ * Work is split in two device passes (Sec. 5.4: a symbolic phase that precomputes the output
+ * structure removes the all array):
+ *   spws_symbolic : per-row product count, work binning, exact output size per row through the
+ *                   chosen workspace, exclusive scan into C's pos array; returns the sizes.
+ *   spws_numeric  : fills C's coordinates and values through the chosen workspace.
+ *
+ * Memory: every pointer inside a spws_tensor_t and the scratch pointer are DEVICE pointers owned
+ * by the caller.  The library never allocates or frees device memory and keeps no pointer after
+ * a call returns, except that spws_numeric reads what spws_symbolic left in the same scratch
+ * buffer.  All kernels are enqueued on the stream set with spws_set_stream.  Inputs are not
+ * modified.  spws_execute_host is the one entry that takes HOST tensors.
+ *
+ * Errors: every function returns a spws_status_t; nothing aborts, throws or prints.
+ */
+#ifndef SPWS_H
+#define SPWS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int spws_status_t;
+enum {
+    SPWS_OK = 0,
+    SPWS_INVALID_ARGUMENT = 1,       /* null pointer, bad enum, bad option value                    */
+    SPWS_UNSUPPORTED_EXPRESSION = 2, /* not one of the two first-order scatters above (any names)   */
+    SPWS_DIM_MISMATCH = 3,           /* contracted dimension or output dimensions disagree          */
+    SPWS_NONCANONICAL_INPUT = 4,     /* unsorted / duplicate / out-of-range coordinate, bad pos     */
+    SPWS_SCRATCH_TOO_SMALL = 5,      /* scratch (or arena) smaller than this call needs             */
+    SPWS_WORKSPACE_TOO_LARGE = 6,    /* policy DENSE forced on a row needing > max_dense_tiles tiles*/
+    SPWS_CUDA_ERROR = 7,             /* a CUDA runtime call failed                                  */
+    SPWS_INTERNAL_OVERFLOW = 8,      /* a bounded device loop hit its limit                         */
+    SPWS_OUTPUT_TOO_SMALL = 9,       /* C's capacity (n[]) is smaller than the result               */
+    SPWS_BAD_SEQUENCE = 10           /* numeric without a successful symbolic on this plan          */
+};
+
+typedef struct spws_handle_s* spws_handle_t;
+typedef struct spws_plan_s* spws_plan_t;
+
+/* Level formats (Sec. 2.1, Fig. 4).  CSR = {Dense, Compressed}; CSF3 = three Compressed levels. */
+typedef enum { SPWS_CSR = 0, SPWS_CSF3 = 1 } spws_format_t;
+typedef enum { SPWS_F32 = 0, SPWS_F64 = 1 } spws_dtype_t;
+/* Workspace policy.  DENSE: value array + occupancy bitmap along the last index (Gustavson's
+ * workspace, Table 2), column-tiled in shared memory.  SPARSE_ISM: insert-sort-merge with the
+ * coordinate-sort policy (Algorithm 1, Sec. 5.2).  AUTO: chosen per row bin from the product
+ * count and the column span.  The policy changes the route, never the result. */
+typedef enum { SPWS_DENSE = 0, SPWS_SPARSE_ISM = 1, SPWS_AUTO = 2 } spws_policy_t;
+
+/* A tensor stored level by level.  Level l of a CSR matrix: l = 0 is Dense (pos[0], crd[0] unused,
+ * n[0] = dims[0]); l = 1 is Compressed: pos[1] has dims[0]+1 entries, crd[1] has n[1] = nnz.
+ * CSF3: pos[0] has 2 entries, crd[0] has n[0]; pos[1] has n[0]+1, crd[1] has n[1]; pos[2] has
+ * n[1]+1, crd[2] has n[2] = nnz; no level stores an empty fibre.  Coordinates are zero-based and
+ * strictly increasing inside a row / fibre.  pos is int64, crd is int32, val is float or double
+ * (the plan's value type) with n[order-1] entries.
+ * For an OUTPUT tensor n[] holds the CAPACITY of crd[l] (and val) on entry to spws_symbolic /
+ * spws_numeric; spws_symbolic overwrites n[] with the sizes of the result. */
+typedef struct {
+    int32_t order;          /* 2 or 3 */
+    int32_t reserved;
+    int64_t dims[3];
+    int64_t n[3];
+    int64_t* pos[3];
+    int32_t* crd[3];
+    void* val;
+} spws_tensor_t;
+
+/* Plan options; zero in a field selects its default.  The thresholds exist so tests can force
+ * every route on small inputs. */
+typedef struct {
+    int32_t validate;         /* 1: check inputs are canonical before any other kernel runs      */
+    int32_t ism_warp_cap;     /* rows with <= this many products use the register ISM (<= 32)    */
+    int32_t ism_cta_cap;      /* accumulation-array capacity of the shared-memory ISM, power of
+                                 two in [64, 4096]; default 4096                                  */
+    int32_t dense_tile_cols;  /* columns per dense tile, power of two in [256, 16384];
+                                 default 8192 (f64) / 16384 (f32)                                 */
+    int32_t max_dense_tiles;  /* a row may use at most this many tiles; default 64               */
+    int32_t fallback_cap;     /* accumulation-array capacity (the paper's `cap`) of the global-
+                                 memory ISM, power of two in [2, 2048]; default 2048              */
+    float dense_span_words_per_product; /* AUTO picks DENSE for a single-tile row when
+                                 span/32 <= this * products; default 4                            */
+    int32_t reserved[5];
+} spws_options_t;
+
+typedef struct {
+    int64_t rows;             /* output rows (SpGEMM) / input fibres (TTM)                        */
+    int64_t products;         /* intermediate products = sum of the per-row upper bounds          */
+    int64_t nnz;              /* stored entries of C                                              */
+    int64_t max_row_products;
+    int64_t rows_per_class[8];/* empty, ISM-register, ISM-shared(small), ISM-shared, dense,
+                                 ISM-global, reserved, reserved                                   */
+    int64_t dense_units;      /* (row, column tile) work units of the dense route                 */
+    int32_t device_status;    /* last status word read back from the device                      */
+    int32_t reserved;
+} spws_stats_t;
+
+spws_status_t spws_create(spws_handle_t* handle);
+spws_status_t spws_destroy(spws_handle_t handle);
+/* `cuda_stream` is a cudaStream_t (NULL = the default stream). */
+spws_status_t spws_set_stream(spws_handle_t handle, void* cuda_stream);
+
+/* Parses `expr` -- "C(i,j)=A(i,k)*B(k,j)" or "C(i,j,l)=A(i,j,k)*B(k,l)" with any tensor and index
+ * names and optional blanks -- and checks it against the formats: fmts[0] is the result's,
+ * fmts[1], fmts[2] the operands' in the order written.  The expression is accepted when it has
+ * exactly one reduction variable, the second operand is a CSR matrix indexed (reduction, last
+ * output index), and the first operand's and result's level orders match the loop order
+ * (Sec. 2.2 classification: first-order scatter).  Anything else: SPWS_UNSUPPORTED_EXPRESSION. */
+spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spws_format_t fmts[3],
+                               spws_dtype_t value_type, spws_policy_t policy,
+                               const spws_options_t* options /* may be NULL */, spws_plan_t* plan);
+spws_status_t spws_plan_destroy(spws_plan_t plan);
+
+/* The expression check of spws_plan_create on its own (host only, needs no device): the
+ * classification of Sec. 2.2 applied to `expr` and `fmts`.  `kind` (may be NULL) receives 0 for
+ * the matrix form, 1 for the 3-tensor form. */
+spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3], int* kind);
+
+/* Upper bound of the scratch bytes spws_symbolic + spws_numeric need for these operands (reads
+ * only dims and n[] of A and B; host-side, launches nothing).  256-byte alignment is required of
+ * the scratch pointer. */
+spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                                  size_t* bytes);
+
+/* Symbolic pass.  C->pos[] must be allocated by the caller: CSR: pos[1] with dims[0]+1 entries;
+ * CSF3: pos[0] (2), crd[0] (A->n[0]), pos[1] (A->n[0]+1), crd[1] (A->n[1]), pos[2] (A->n[1]+1),
+ * i.e. the sizes of A's upper levels, which bound C's.  On return C->n[] holds the result sizes
+ * and `sizes_out` (host, 3 entries, may be NULL) a copy.  Synchronises the stream once, to read
+ * the sizes back. */
+spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                            spws_tensor_t* C, void* scratch, size_t scratch_bytes,
+                            int64_t* sizes_out);
+
+/* Numeric pass.  C->crd[last] and C->val must now hold C->n[last] entries.  Asynchronous: returns
+ * after enqueueing; a device-side failure is reported by the next spws_get_stats. */
+spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                           spws_tensor_t* C, void* scratch, size_t scratch_bytes);
+
+/* Synchronises the plan's stream and reports the last symbolic pass's statistics. */
+spws_status_t spws_get_stats(spws_plan_t plan, spws_stats_t* stats);
+
+/* Whole path with HOST tensors: copies A and B to the device, runs both passes, copies C back.
+ * A, B, C hold host pointers; C's arrays must be allocated with capacities n[] (crd/val of the
+ * last level sized for the expected nnz; SPWS_OUTPUT_TOO_SMALL if the result is larger, with
+ * C->n[] set to the needed sizes).  `arena` is DEVICE memory of `arena_bytes` supplied by the
+ * caller, from which the call carves the device copies, C and the scratch.  `arena_needed`
+ * (may be NULL) receives the bytes this call needed.  Synchronous. */
+spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                                spws_tensor_t* C, void* arena, size_t arena_bytes,
+                                size_t* arena_needed);
+
+const char* spws_status_string(spws_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPWS_H */

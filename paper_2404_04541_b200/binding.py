@@ -1,0 +1,242 @@
+"""ctypes binding of libspws.so: the same entry points as include/spws.h, argument marshalling
+only.  PyTorch supplies device memory and the stream; every step of the path runs in the
+library's kernels.  Importing this module fails loudly when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspws.so")
+
+# status codes
+SPWS_OK = 0
+SPWS_INVALID_ARGUMENT = 1
+SPWS_UNSUPPORTED_EXPRESSION = 2
+SPWS_DIM_MISMATCH = 3
+SPWS_NONCANONICAL_INPUT = 4
+SPWS_SCRATCH_TOO_SMALL = 5
+SPWS_WORKSPACE_TOO_LARGE = 6
+SPWS_CUDA_ERROR = 7
+SPWS_INTERNAL_OVERFLOW = 8
+SPWS_OUTPUT_TOO_SMALL = 9
+SPWS_BAD_SEQUENCE = 10
+# enums
+SPWS_CSR, SPWS_CSF3 = 0, 1
+SPWS_F32, SPWS_F64 = 0, 1
+SPWS_DENSE, SPWS_SPARSE_ISM, SPWS_AUTO = 0, 1, 2
+POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPARSE_ISM, "auto": SPWS_AUTO}
+
+EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create", "spws_plan_destroy",
+           "spws_check_expression", "spws_workspace_size", "spws_symbolic", "spws_numeric",
+           "spws_get_stats", "spws_execute_host", "spws_status_string")
+
+
+class spws_tensor_t(ctypes.Structure):
+    _fields_ = [("order", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("dims", ctypes.c_int64 * 3), ("n", ctypes.c_int64 * 3),
+                ("pos", ctypes.c_void_p * 3), ("crd", ctypes.c_void_p * 3), ("val", ctypes.c_void_p)]
+
+
+class spws_options_t(ctypes.Structure):
+    _fields_ = [("validate", ctypes.c_int32), ("ism_warp_cap", ctypes.c_int32), ("ism_cta_cap", ctypes.c_int32),
+                ("dense_tile_cols", ctypes.c_int32), ("max_dense_tiles", ctypes.c_int32),
+                ("fallback_cap", ctypes.c_int32), ("dense_span_words_per_product", ctypes.c_float),
+                ("reserved", ctypes.c_int32 * 5)]
+
+
+class spws_stats_t(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int64), ("products", ctypes.c_int64), ("nnz", ctypes.c_int64),
+                ("max_row_products", ctypes.c_int64), ("rows_per_class", ctypes.c_int64 * 8),
+                ("dense_units", ctypes.c_int64), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class SpwsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if libspws.so is missing (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2404_04541_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        T = ctypes.POINTER(spws_tensor_t)
+        L.spws_create.argtypes = [ctypes.POINTER(vp)]
+        L.spws_destroy.argtypes = [vp]
+        L.spws_set_stream.argtypes = [vp, vp]
+        L.spws_plan_create.argtypes = [vp, ctypes.c_char_p, ctypes.POINTER(i32), i32, i32,
+                                       ctypes.POINTER(spws_options_t), ctypes.POINTER(vp)]
+        L.spws_plan_destroy.argtypes = [vp]
+        L.spws_check_expression.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.spws_workspace_size.argtypes = [vp, T, T, ctypes.POINTER(sz)]
+        L.spws_symbolic.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(ctypes.c_int64)]
+        L.spws_numeric.argtypes = [vp, T, T, T, vp, sz]
+        L.spws_get_stats.argtypes = [vp, ctypes.POINTER(spws_stats_t)]
+        L.spws_execute_host.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(sz)]
+        L.spws_status_string.argtypes = [i32]
+        L.spws_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name != "spws_status_string":
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().spws_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != SPWS_OK:
+        raise SpwsError(status, where)
+
+
+def check_expression(expr: str, fmts) -> int:
+    """Host-only classification; returns the status and does not raise."""
+    arr = (ctypes.c_int * 3)(*fmts)
+    kind = ctypes.c_int(-1)
+    return lib().spws_check_expression(expr.encode(), arr, ctypes.byref(kind))
+
+
+# ---------------------------------------------------------------------------- tensors
+def _ptr(t):
+    """Address of a torch tensor's (or numpy array's) storage, or None."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data if t.size else None
+    return t.data_ptr() if t.numel() else None
+
+
+@dataclass
+class TensorArrays:
+    """Level arrays of a CSR matrix (order 2) or CSF 3-tensor (order 3); torch tensors on the
+    device, or numpy arrays for the host entry point."""
+    order: int
+    dims: tuple
+    pos: list
+    crd: list
+    val: object
+    n: list = field(default_factory=lambda: [0, 0, 0])
+
+    def c_struct(self) -> spws_tensor_t:
+        t = spws_tensor_t()
+        t.order = self.order
+        for a in range(3):
+            t.dims[a] = int(self.dims[a]) if a < len(self.dims) else 0
+            t.n[a] = int(self.n[a])
+            t.pos[a] = _ptr(self.pos[a]) if a < len(self.pos) else None
+            t.crd[a] = _ptr(self.crd[a]) if a < len(self.crd) else None
+        t.val = _ptr(self.val)
+        return t
+
+
+def csr_arrays(nrows, ncols, pos, crd, val) -> TensorArrays:
+    nnz = int(crd.shape[0]) if crd is not None else 0
+    return TensorArrays(2, (nrows, ncols, 0), [None, pos, None], [None, crd, None], val, [nrows, nnz, 0])
+
+
+def csf3_arrays(dims, pos0, crd0, pos1, crd1, pos2, crd2, val) -> TensorArrays:
+    n = [int(crd0.shape[0]), int(crd1.shape[0]), int(crd2.shape[0]) if crd2 is not None else 0]
+    return TensorArrays(3, tuple(dims), [pos0, pos1, pos2], [crd0, crd1, crd2], val, n)
+
+
+# ---------------------------------------------------------------------------- handle / plan
+class Handle:
+    def __init__(self, stream_ptr: int | None = None):
+        self._h = ctypes.c_void_p()
+        _check(lib().spws_create(ctypes.byref(self._h)), "spws_create")
+        if stream_ptr is not None:
+            self.set_stream(stream_ptr)
+
+    def set_stream(self, stream_ptr: int):
+        _check(lib().spws_set_stream(self._h, ctypes.c_void_p(stream_ptr)), "spws_set_stream")
+
+    def close(self):
+        if self._h:
+            lib().spws_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Plan:
+    def __init__(self, handle: Handle, expr: str, fmts, dtype, policy="auto", **options):
+        self.handle = handle
+        self._p = ctypes.c_void_p()
+        self.np_dtype = np.dtype(dtype)
+        vt = SPWS_F64 if self.np_dtype == np.float64 else SPWS_F32
+        if self.np_dtype not in (np.dtype(np.float32), np.dtype(np.float64)):
+            raise SpwsError(SPWS_INVALID_ARGUMENT, "Plan: value type")
+        opt = spws_options_t()
+        for k, v in options.items():
+            if not hasattr(opt, k):
+                raise SpwsError(SPWS_INVALID_ARGUMENT, f"Plan: unknown option {k}")
+            setattr(opt, k, v)
+        arr = (ctypes.c_int * 3)(*fmts)
+        pol = POLICIES[policy] if isinstance(policy, str) else int(policy)
+        _check(lib().spws_plan_create(handle._h, expr.encode(), arr, vt, pol, ctypes.byref(opt),
+                                      ctypes.byref(self._p)), "spws_plan_create")
+
+    def workspace_size(self, A: TensorArrays, B: TensorArrays) -> int:
+        out = ctypes.c_size_t(0)
+        a, b = A.c_struct(), B.c_struct()
+        _check(lib().spws_workspace_size(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(out)),
+               "spws_workspace_size")
+        return int(out.value)
+
+    def symbolic(self, A, B, C, scratch_ptr: int, scratch_bytes: int):
+        a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
+        sizes = (ctypes.c_int64 * 3)()
+        _check(lib().spws_symbolic(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                   ctypes.c_void_p(scratch_ptr), scratch_bytes, sizes), "spws_symbolic")
+        C.n = [int(sizes[0]), int(sizes[1]), int(sizes[2])]
+        return C.n
+
+    def numeric(self, A, B, C, scratch_ptr: int, scratch_bytes: int):
+        a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
+        _check(lib().spws_numeric(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                  ctypes.c_void_p(scratch_ptr), scratch_bytes), "spws_numeric")
+
+    def get_stats(self) -> dict:
+        s = spws_stats_t()
+        st = lib().spws_get_stats(self._p, ctypes.byref(s))
+        d = dict(rows=s.rows, products=s.products, nnz=s.nnz, max_row_products=s.max_row_products,
+                 rows_per_class=list(s.rows_per_class), dense_units=s.dense_units, device_status=s.device_status)
+        _check(st, "spws_get_stats")
+        return d
+
+    def execute_host(self, A: TensorArrays, B: TensorArrays, C: TensorArrays, arena_ptr: int, arena_bytes: int):
+        """A, B, C hold numpy (ideally pinned) host arrays; returns (status, sizes, arena_needed)."""
+        a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
+        need = ctypes.c_size_t(0)
+        st = lib().spws_execute_host(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                     ctypes.c_void_p(arena_ptr), arena_bytes, ctypes.byref(need))
+        return st, [int(c.n[0]), int(c.n[1]), int(c.n[2])], int(need.value)
+
+    def close(self):
+        if self._p:
+            lib().spws_plan_destroy(self._p)
+            self._p = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

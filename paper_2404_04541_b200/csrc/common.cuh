@@ -1,0 +1,164 @@
+// Shared device-side definitions of the spws kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spws {
+
+typedef long long i64;
+typedef unsigned long long u64;
+
+constexpr int NCLASS = 8;
+// Row classes = the workspace a row (or (i,j) fibre) is routed to.
+enum RowClass : int {
+    CLS_EMPTY = 0,     // no intermediate product
+    CLS_ISM_REG = 1,   // insert-sort-merge in registers, one lane group per row
+    CLS_ISM_SMEM_S = 2,// insert-sort-merge in shared memory, small CTA
+    CLS_ISM_SMEM = 3,  // insert-sort-merge in shared memory, full CTA
+    CLS_DENSE = 4,     // dense accumulator + occupancy bitmap, (row, column tile) units
+    CLS_ISM_GLOBAL = 5 // accumulation array in shared memory, all array in global memory
+};
+
+enum DevStatus : int {
+    DEV_OK = 0,
+    DEV_NONCANONICAL = 4,
+    DEV_SCRATCH_TOO_SMALL = 5,
+    DEV_WORKSPACE_TOO_LARGE = 6,
+    DEV_INTERNAL_OVERFLOW = 8
+};
+
+// Control block at the start of the scratch buffer (zeroed when a symbolic pass starts).
+struct DevCtl {
+    i64 nnz;
+    i64 products;
+    i64 max_ub;
+    i64 max_ub_global;      // largest product count among CLS_ISM_GLOBAL rows
+    i64 kept[2];            // TTM: surviving slices (level 0) and fibres (level 1)
+    int status;
+    int n_units;
+    int class_count[NCLASS];
+    int class_cursor[NCLASS];
+    int work_counter[16];   // dynamic work distribution; cleared before each pass
+    int global_slots;       // slots the global-memory ISM actually used
+    int pad[7];
+};
+
+struct ClassParams {
+    int policy;             // spws_policy_t
+    int reg_cap;            // CLS_ISM_REG: products <= reg_cap
+    int smem_small_cap;     // CLS_ISM_SMEM_S
+    int smem_cap;           // CLS_ISM_SMEM
+    int tile_cols;          // W
+    int max_tiles;
+    float span_words_per_product;
+    int unit_cap;           // entries available in the unit tables
+};
+
+struct Csr {
+    const i64* pos;
+    const int* crd;
+    const void* val;
+    int nrows;
+    int ncols;
+};
+
+// Per-row tables in scratch.
+struct RowTables {
+    i64* ub;
+    int* cnt;
+    int* jmin;
+    int* jmax;
+    unsigned char* cls;
+    int* perm;
+    int* row_unit0;
+    int* unit_row;
+    int* unit_cnt;
+};
+
+__device__ __forceinline__ void raise_status(DevCtl* ctl, int s) { atomicCAS(&ctl->status, 0, s); }
+
+// Rows of class `cls` are perm[off, off + n).
+__device__ __forceinline__ void class_range(const DevCtl* ctl, int cls, int& off, int& n) {
+    off = 0;
+    for (int c = 0; c < cls; ++c) off += ctl->class_count[c];
+    n = ctl->class_count[cls];
+}
+
+__device__ __forceinline__ int warp_incl_scan(int v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, v, d);
+        if (lane >= d) v += t;
+    }
+    return v;
+}
+
+// Exclusive scan over a block of THREADS threads; `ws` needs 33 ints; every thread gets `total`.
+template <int THREADS>
+__device__ __forceinline__ int block_excl_scan(int v, int* ws, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int incl = warp_incl_scan(v);
+    __syncthreads();                       // ws may still be read from a previous call
+    if (lane == 31) ws[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int s = (lane < THREADS / 32) ? ws[lane] : 0;
+        const int si = warp_incl_scan(s);
+        if (lane < THREADS / 32) ws[lane] = si - s;
+        if (lane == 31) ws[32] = si;
+    }
+    __syncthreads();
+    total = ws[32];
+    return ws[warp] + incl - v;
+}
+
+// First position in crd[lo, hi) whose coordinate is >= c (rows are sorted).
+__device__ __forceinline__ i64 lower_bound_crd(const int* __restrict__ crd, i64 lo, i64 hi, int c) {
+    while (lo < hi) {
+        const i64 mid = (lo + hi) >> 1;
+        if (__ldg(crd + mid) < c) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// Products are formed as a rounded multiply followed by rounded adds (no contraction), so the
+// ISM routes, which sum in product order, reproduce a plain sequential sum bit for bit.
+__device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
+__device__ __forceinline__ float mul_rn(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
+__device__ __forceinline__ float add_rn(float a, float b) { return __fadd_rn(a, b); }
+
+// ---- launchers (defined in the .cu files) ------------------------------------------------
+struct LaunchCtx {
+    cudaStream_t stream;
+    int sm_count;
+    DevCtl* ctl;
+    ClassParams prm;
+    RowTables tab;
+    int is_f64;
+    char* global_arena;      // scratch for CLS_ISM_GLOBAL all arrays
+    size_t global_arena_bytes;
+    int global_cap;          // accumulation-array capacity of CLS_ISM_GLOBAL
+};
+
+// setup.cu
+cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA, i64 nnzB);
+cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA);
+cudaError_t launch_bin_rows(const LaunchCtx& c, int m);
+cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out);
+cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
+                               const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
+                               i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2);
+// ism_reg.cu / ism_smem.cu / dense.cu / ism_global.cu: n_host < 0 means "read the count from ctl".
+cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+                           const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_ism_smem(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
+                            const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_dense(const LaunchCtx& c, bool numeric, int n_units_host, const Csr& A, const Csr& B,
+                         const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+                              const i64* rowptr, int* Ccrd, void* Cval);
+size_t dense_smem_bytes(int tile_cols, int is_f64);
+
+}  // namespace spws

@@ -1,0 +1,147 @@
+// Insert-sort-merge workspace held in registers: one group of G lanes per output row whose
+// product count is at most G (Algorithm 1 with the accumulation array = the lanes of the group;
+// coordinate-sort policy, Sec. 5.2: append without reduction, sort, reduce equal coordinates).
+//   Insert : lane t takes the t-th product of the row in loop order (k, then j).
+//   Sort   : bitonic network over the group on the packed word (j - jmin) << 5 | lane -- only
+//            this integer moves (accumulation indexing, Sec. 5.1); values stay in their lane.
+//   Merge  : equal coordinates are adjacent; the first lane of a run sums the run in product
+//            order and writes it at row_ptr[i] + rank.
+#include "common.cuh"
+
+namespace spws {
+
+template <typename T, int G, bool NUMERIC>
+__global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ perm, const DevCtl* __restrict__ ctl,
+                                                      Csr A, Csr B, const int* __restrict__ jmin, int* __restrict__ cnt,
+                                                      const i64* __restrict__ rowptr, int* __restrict__ Ccrd, T* __restrict__ Cval) {
+    if (ctl->status != 0) return;
+    int off, n;
+    class_range(ctl, CLS_ISM_REG, off, n);
+    const int* __restrict__ rows = perm + off;
+    const unsigned lane = threadIdx.x & 31;
+    const int gl = threadIdx.x % G;
+    const unsigned gshift = lane - gl;
+    const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << gshift);
+    const i64 group = ((i64)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const i64 ngroups = ((i64)gridDim.x * blockDim.x) / G;
+    const T* __restrict__ Aval = (const T*)A.val;
+    const T* __restrict__ Bval = (const T*)B.val;
+
+    for (i64 r = group; r < n; r += ngroups) {
+        const int row = rows[r];
+        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        const int base = jmin[row];
+
+        // ---- Insert: lane gl receives product number gl
+        unsigned packed = 0xffffffffu;
+        T val = 0;
+        int done = 0;
+        for (i64 p0 = ps; p0 < pe; p0 += G) {
+            const i64 p = p0 + gl;
+            int len = 0;
+            i64 qs = 0;
+            if (p < pe) {
+                const int k = __ldg(A.crd + p);
+                if ((unsigned)k < (unsigned)B.nrows) {
+                    qs = __ldg(B.pos + k);
+                    len = (int)(__ldg(B.pos + k + 1) - qs);
+                }
+            }
+            int incl = len;
+#pragma unroll
+            for (int d = 1; d < G; d <<= 1) {
+                const int t = __shfl_up_sync(gmask, incl, d, G);
+                if (gl >= d) incl += t;
+            }
+            const int excl = incl - len + done;
+            const int total = __shfl_sync(gmask, incl, G - 1, G);
+            // entry that owns product gl: the last entry whose first product is <= gl
+            int e = 0;
+#pragma unroll
+            for (int s = G / 2; s >= 1; s >>= 1) {
+                const int v = __shfl_sync(gmask, excl, e + s, G);
+                if (v <= gl) e += s;
+            }
+            const int e_excl = __shfl_sync(gmask, excl, e, G);
+            const i64 e_qs = __shfl_sync(gmask, qs, e, G);
+            if (gl >= done && gl < done + total) {
+                const i64 q = e_qs + (gl - e_excl);
+                const int j = __ldg(B.crd + q);
+                packed = ((unsigned)(j - base) << 5) | (unsigned)gl;
+                if (NUMERIC) val = mul_rn(__ldg(Aval + p0 + e), __ldg(Bval + q));
+            }
+            done += total;
+        }
+
+        // ---- Sort
+#pragma unroll
+        for (int k = 2; k <= G; k <<= 1) {
+#pragma unroll
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                const unsigned other = __shfl_xor_sync(gmask, packed, j, G);
+                const bool up = (gl & k) == 0;
+                const bool low = (gl & j) == 0;
+                packed = (up == low) ? min(packed, other) : max(packed, other);
+            }
+        }
+
+        // ---- Merge
+        const bool valid = packed != 0xffffffffu;
+        const unsigned key = packed >> 5;
+        const unsigned prev = __shfl_up_sync(gmask, key, 1, G);
+        const bool head = valid && (gl == 0 || key != prev);
+        const unsigned heads = (__ballot_sync(gmask, head) >> gshift) & ((G == 32) ? 0xffffffffu : ((1u << G) - 1u));
+        if (!NUMERIC) {
+            if (gl == 0) cnt[row] = __popc(heads);
+        } else {
+            T v = __shfl_sync(gmask, val, packed & 31u, G);
+            T sum = v;
+            for (int d = 1; d < G; ++d) {
+                const unsigned k2 = __shfl_down_sync(gmask, key, d, G);
+                const T v2 = __shfl_down_sync(gmask, v, d, G);
+                const bool more = valid && (gl + d < G) && (k2 == key);
+                if (!__any_sync(gmask, more)) break;
+                if (more) sum = add_rn(sum, v2);
+            }
+            if (head) {
+                const int rank = __popc(heads & ((1u << gl) - 1u));
+                const i64 out = rowptr[row] + rank;
+                Ccrd[out] = (int)key + base;
+                Cval[out] = sum;
+            }
+        }
+    }
+}
+
+template <typename T, int G>
+static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+                            const i64* rowptr, int* Ccrd, void* Cval) {
+    const int threads = 256;
+    i64 groups = (n_host >= 0) ? n_host : A.nrows;
+    i64 want = (groups * G + threads - 1) / threads;
+    i64 cap = (i64)c.sm_count * 16;
+    int grid = (int)(want < cap ? want : cap);
+    if (grid < 1) grid = 1;
+    if (numeric)
+        ism_reg_kernel<T, G, true><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, A, B,
+                                                                 c.tab.jmin, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
+    else
+        ism_reg_kernel<T, G, false><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, A, B,
+                                                                  c.tab.jmin, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+                           const i64* rowptr, int* Ccrd, void* Cval) {
+    const int cap = c.prm.reg_cap;
+    if (c.is_f64) {
+        if (cap <= 8) return launch_g<double, 8>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+        if (cap <= 16) return launch_g<double, 16>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+        return launch_g<double, 32>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+    }
+    if (cap <= 8) return launch_g<float, 8>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+    if (cap <= 16) return launch_g<float, 16>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+    return launch_g<float, 32>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+}
+
+}  // namespace spws

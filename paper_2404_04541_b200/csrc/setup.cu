@@ -1,0 +1,356 @@
+// Symbolic-pass set-up kernels: input validation, per-row product upper bound and column
+// span, routing of rows to workspaces (binning), exclusive scans, CSF level rebuild.
+#include "common.cuh"
+
+namespace spws {
+
+// ---------------------------------------------------------------------------------------
+// Validation: pos non-decreasing with pos[0] = 0 and pos[rows] = nnz; coordinates in range
+// and strictly increasing inside a row.
+// ---------------------------------------------------------------------------------------
+__global__ void validate_csr_kernel(Csr M, i64 nnz, int coord_limit, DevCtl* ctl) {
+    const i64 stride = (i64)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < M.nrows; r += stride) {
+        const i64 s = M.pos[r], e = M.pos[r + 1];
+        if (r == 0 && s != 0) bad = true;
+        if (r == M.nrows - 1 && e != nnz) bad = true;
+        if (s > e || s < 0 || e > nnz) { bad = true; continue; }
+        int prev = -1;
+        for (i64 p = s; p < e; ++p) {
+            const int c = M.crd[p];
+            if (c <= prev || c >= coord_limit) bad = true;
+            prev = c;
+        }
+    }
+    if (M.nrows == 0 && threadIdx.x == 0 && blockIdx.x == 0 && nnz != 0) bad = true;
+    if (bad) raise_status(ctl, DEV_NONCANONICAL);
+}
+
+cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA, i64 nnzB) {
+    const int grid = c.sm_count * 8;
+    validate_csr_kernel<<<grid, 256, 0, c.stream>>>(A, nnzA, B.nrows, c.ctl);
+    validate_csr_kernel<<<grid, 256, 0, c.stream>>>(B, nnzB, B.ncols, c.ctl);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Per-row upper bound ub[i] = sum over A(i,:) of the picked B row's length, the exact span
+// [jmin, jmax] of the candidate columns (first / last coordinate of the picked B rows, which
+// are sorted), and the workspace class of the row.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const ClassParams& prm, DevCtl* ctl) {
+    if (ub == 0) return CLS_EMPTY;
+    const i64 span = (i64)jmax - jmin + 1;
+    const i64 ntiles = (span + prm.tile_cols - 1) / prm.tile_cols;
+    const bool reg_ok = ub <= prm.reg_cap && span <= (1ll << 26);
+    if (prm.policy == 0) {                       // dense forced
+        if (ntiles > prm.max_tiles) { raise_status(ctl, DEV_WORKSPACE_TOO_LARGE); return CLS_EMPTY; }
+        return CLS_DENSE;
+    }
+    if (prm.policy == 1) {                       // sparse ISM forced
+        if (reg_ok) return CLS_ISM_REG;
+        if (ub <= prm.smem_small_cap) return CLS_ISM_SMEM_S;
+        if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
+        return CLS_ISM_GLOBAL;
+    }
+    // auto: few products -> sort them; a narrow span relative to the work -> dense tile;
+    // mid-size rows -> shared-memory ISM; long rows -> column-tiled dense; otherwise global ISM.
+    if (reg_ok) return CLS_ISM_REG;
+    const i64 span_words = (span + 31) >> 5;
+    if (ntiles == 1 && (float)span_words <= prm.span_words_per_product * (float)ub) return CLS_DENSE;
+    if (ub <= prm.smem_small_cap) return CLS_ISM_SMEM_S;
+    if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
+    if (ntiles <= prm.max_tiles) return CLS_DENSE;
+    return CLS_ISM_GLOBAL;
+}
+
+template <int G>
+__global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl) {
+    __shared__ int s_hist[NCLASS];
+    __shared__ i64 s_products, s_max_ub, s_max_ub_global;
+    if (threadIdx.x < NCLASS) s_hist[threadIdx.x] = 0;
+    if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; }
+    __syncthreads();
+    const int gl = threadIdx.x % G;
+    const unsigned lane = threadIdx.x & 31;
+    const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane - gl));
+    const i64 group = ((i64)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const i64 ngroups = ((i64)gridDim.x * blockDim.x) / G;
+    i64 my_products = 0, my_max = 0, my_max_global = 0;
+    for (i64 row = group; row < A.nrows; row += ngroups) {
+        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        i64 u = 0;
+        int lo = 0x7fffffff, hi = -1;
+        bool bad = false;
+        for (i64 p = ps + gl; p < pe; p += G) {
+            const int k = __ldg(A.crd + p);
+            if ((unsigned)k < (unsigned)B.nrows) {
+                const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                if (qe > qs) {
+                    u += qe - qs;
+                    lo = min(lo, __ldg(B.crd + qs));
+                    hi = max(hi, __ldg(B.crd + qe - 1));
+                }
+            } else {
+                bad = true;
+            }
+        }
+#pragma unroll
+        for (int d = G / 2; d > 0; d >>= 1) {
+            u += __shfl_xor_sync(gmask, u, d, G);
+            lo = min(lo, __shfl_xor_sync(gmask, lo, d, G));
+            hi = max(hi, __shfl_xor_sync(gmask, hi, d, G));
+        }
+        if (bad) raise_status(ctl, DEV_NONCANONICAL);
+        if (gl == 0) {
+            if (lo < 0 || hi >= B.ncols) { raise_status(ctl, DEV_NONCANONICAL); u = 0; }
+            const int cls = classify_row(u, lo, hi, prm, ctl);
+            tab.ub[row] = u;
+            tab.jmin[row] = lo;
+            tab.jmax[row] = hi;
+            tab.cnt[row] = 0;
+            tab.cls[row] = (unsigned char)cls;
+            atomicAdd(&s_hist[cls], 1);
+            my_products += u;
+            my_max = max(my_max, u);
+            if (cls == CLS_ISM_GLOBAL) my_max_global = max(my_max_global, u);
+        }
+    }
+    if (gl == 0 && my_products) atomicAdd((u64*)&s_products, (u64)my_products);
+    if (gl == 0 && my_max) atomicMax(&s_max_ub, my_max);
+    if (gl == 0 && my_max_global) atomicMax(&s_max_ub_global, my_max_global);
+    __syncthreads();
+    if (threadIdx.x < NCLASS && s_hist[threadIdx.x]) atomicAdd(&ctl->class_count[threadIdx.x], s_hist[threadIdx.x]);
+    if (threadIdx.x == 0) {
+        if (s_products) atomicAdd((u64*)&ctl->products, (u64)s_products);
+        if (s_max_ub) atomicMax(&ctl->max_ub, s_max_ub);
+        if (s_max_ub_global) atomicMax(&ctl->max_ub_global, s_max_ub_global);
+    }
+}
+
+cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA) {
+    if (A.nrows == 0) return cudaSuccess;
+    const double avg = (double)nnzA / (double)A.nrows;
+    const int threads = 256;
+    auto grid_for = [&](int G) {
+        i64 want = ((i64)A.nrows * G + threads - 1) / threads;
+        i64 cap = (i64)c.sm_count * 16;
+        return (int)(want < cap ? want : cap);
+    };
+    if (avg <= 6.0) row_bounds_kernel<4><<<grid_for(4), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
+    else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
+    else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Binning: rows grouped by class into perm (class c occupies [off[c], off[c+1])); dense rows
+// also reserve their (row, tile) units.  Order inside a class follows block arrival.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
+    __shared__ int s_hist[NCLASS], s_base[NCLASS], s_off[NCLASS];
+    const int rows_per_block = blockDim.x * 4;
+    if (threadIdx.x == 0) {
+        int o = 0;
+        for (int c = 0; c < NCLASS; ++c) { s_off[c] = o; o += ctl->class_count[c]; }
+    }
+    for (i64 r0 = (i64)blockIdx.x * rows_per_block; r0 < m; r0 += (i64)gridDim.x * rows_per_block) {
+        if (threadIdx.x < NCLASS) s_hist[threadIdx.x] = 0;
+        __syncthreads();
+        int cls[4], rank[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const i64 row = r0 + x * blockDim.x + threadIdx.x;
+            cls[x] = -1;
+            if (row < m) {
+                cls[x] = tab.cls[row];
+                rank[x] = atomicAdd(&s_hist[cls[x]], 1);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < NCLASS && s_hist[threadIdx.x])
+            s_base[threadIdx.x] = atomicAdd(&ctl->class_cursor[threadIdx.x], s_hist[threadIdx.x]);
+        __syncthreads();
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const i64 row = r0 + x * blockDim.x + threadIdx.x;
+            if (cls[x] < 0) continue;
+            tab.perm[s_off[cls[x]] + s_base[cls[x]] + rank[x]] = (int)row;
+            if (cls[x] == CLS_DENSE) {
+                const int ntiles = (tab.jmax[row] - tab.jmin[row]) / prm.tile_cols + 1;
+                const int u0 = atomicAdd(&ctl->n_units, ntiles);
+                if (u0 + ntiles > prm.unit_cap) {
+                    raise_status(ctl, DEV_SCRATCH_TOO_SMALL);
+                    tab.row_unit0[row] = -1;
+                } else {
+                    tab.row_unit0[row] = u0;
+                    for (int t = 0; t < ntiles; ++t) tab.unit_row[u0 + t] = (int)row;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_bin_rows(const LaunchCtx& c, int m) {
+    if (m == 0) return cudaSuccess;
+    i64 want = ((i64)m + 1023) / 1024;
+    i64 cap = (i64)c.sm_count * 8;
+    bin_rows_kernel<<<(int)(want < cap ? want : cap), 256, 0, c.stream>>>(m, c.tab, c.prm, c.ctl);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Exclusive scan int32[n] -> int64[n+1] (reduce, scan of block sums, scan): no waits between
+// blocks.  out[n] (and *total_out when given) receive the total.
+// ---------------------------------------------------------------------------------------
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 8;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+__global__ void __launch_bounds__(SCAN_THREADS) scan_reduce_kernel(const int* __restrict__ in, int n, i64* block_sums) {
+    __shared__ i64 s_part[SCAN_THREADS / 32];
+    const i64 base = (i64)blockIdx.x * SCAN_TILE;
+    i64 s = 0;
+    for (int x = 0; x < SCAN_ITEMS; ++x) {
+        const i64 i = base + x * SCAN_THREADS + threadIdx.x;
+        if (i < n) s += in[i];
+    }
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        i64 t = 0;
+        for (int w = 0; w < SCAN_THREADS / 32; ++w) t += s_part[w];
+        block_sums[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(1024) scan_block_sums_kernel(i64* block_sums, int nblocks, i64* out_total, i64* total_out2) {
+    __shared__ i64 s_warp[32];
+    __shared__ i64 s_carry;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = 0; base < nblocks; base += 1024) {
+        const int i = base + threadIdx.x;
+        const i64 v = (i < nblocks) ? block_sums[i] : 0;
+        i64 incl = v;
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        for (int d = 1; d < 32; d <<= 1) {
+            const i64 t = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += t;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            i64 w = s_warp[lane];
+            i64 wi = w;
+            for (int d = 1; d < 32; d <<= 1) {
+                const i64 t = __shfl_up_sync(0xffffffffu, wi, d);
+                if (lane >= d) wi += t;
+            }
+            s_warp[lane] = wi - w;
+        }
+        __syncthreads();
+        const i64 carry = s_carry;
+        if (i < nblocks) block_sums[i] = carry + s_warp[warp] + incl - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) s_carry = carry + s_warp[warp] + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        *out_total = s_carry;
+        if (total_out2) *total_out2 = s_carry;
+    }
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int* __restrict__ in, int n, const i64* __restrict__ block_sums, i64* __restrict__ out) {
+    __shared__ int ws[33];
+    const i64 base = (i64)blockIdx.x * SCAN_TILE + (i64)threadIdx.x * SCAN_ITEMS;
+    int v[SCAN_ITEMS];
+    int s = 0;
+#pragma unroll
+    for (int x = 0; x < SCAN_ITEMS; ++x) {
+        v[x] = (base + x < n) ? in[base + x] : 0;
+        s += v[x];
+    }
+    int total;
+    const int excl = block_excl_scan<SCAN_THREADS>(s, ws, total);
+    i64 run = block_sums[blockIdx.x] + excl;
+#pragma unroll
+    for (int x = 0; x < SCAN_ITEMS; ++x) {
+        if (base + x < n) out[base + x] = run;
+        run += v[x];
+    }
+}
+
+cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out) {
+    const int nblocks = (n + SCAN_TILE - 1) / SCAN_TILE;
+    if (nblocks > 0) scan_reduce_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums);
+    scan_block_sums_kernel<<<1, 1024, 0, c.stream>>>(block_sums, nblocks, out + n, total_out);
+    if (nblocks > 0) scan_apply_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums, out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// TTM: rebuild C's two upper CSF levels.  A fibre (i,j) survives when it produced at least
+// one output; a slice i survives when one of its fibres does.
+// ---------------------------------------------------------------------------------------
+__global__ void ttm_fibre_flags_kernel(int n_ij, const int* __restrict__ cnt, int* flags) {
+    for (i64 f = (i64)blockIdx.x * blockDim.x + threadIdx.x; f < n_ij; f += (i64)gridDim.x * blockDim.x)
+        flags[f] = cnt[f] > 0;
+}
+
+__global__ void ttm_fibre_compact_kernel(int n_ij, const int* __restrict__ flags, const i64* __restrict__ fpos,
+                                         const int* __restrict__ Acrd1, const i64* __restrict__ rowptr_raw,
+                                         int* Ccrd1, i64* Cpos2) {
+    for (i64 f = (i64)blockIdx.x * blockDim.x + threadIdx.x; f <= n_ij; f += (i64)gridDim.x * blockDim.x) {
+        if (f == n_ij) { Cpos2[fpos[n_ij]] = rowptr_raw[n_ij]; continue; }
+        if (flags[f]) {
+            Ccrd1[fpos[f]] = Acrd1[f];
+            Cpos2[fpos[f]] = rowptr_raw[f];
+        }
+    }
+}
+
+__global__ void ttm_slice_flags_kernel(int n_i, const i64* __restrict__ Apos1, const i64* __restrict__ fpos, int* sflags) {
+    for (i64 s = (i64)blockIdx.x * blockDim.x + threadIdx.x; s < n_i; s += (i64)gridDim.x * blockDim.x)
+        sflags[s] = fpos[Apos1[s + 1]] > fpos[Apos1[s]];
+}
+
+__global__ void ttm_slice_compact_kernel(int n_i, int n_ij, const int* __restrict__ sflags, const i64* __restrict__ spos,
+                                         const i64* __restrict__ Apos1, const i64* __restrict__ fpos,
+                                         const int* __restrict__ Acrd0, int* Ccrd0, i64* Cpos1, i64* Cpos0, DevCtl* ctl) {
+    for (i64 s = (i64)blockIdx.x * blockDim.x + threadIdx.x; s <= n_i; s += (i64)gridDim.x * blockDim.x) {
+        if (s == n_i) {
+            Cpos1[spos[n_i]] = fpos[n_ij];
+            Cpos0[0] = 0;
+            Cpos0[1] = spos[n_i];
+            ctl->kept[0] = spos[n_i];
+            ctl->kept[1] = fpos[n_ij];
+            continue;
+        }
+        if (sflags[s]) {
+            Ccrd0[spos[s]] = Acrd0[s];
+            Cpos1[spos[s]] = fpos[Apos1[s]];
+        }
+    }
+}
+
+cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
+                               const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
+                               i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2) {
+    const int grid = c.sm_count * 8;
+    if (n_ij > 0) ttm_fibre_flags_kernel<<<grid, 256, 0, c.stream>>>(n_ij, c.tab.cnt, flags);
+    cudaError_t e = launch_scan_counts(c, flags, n_ij, fpos, block_sums, nullptr);
+    if (e != cudaSuccess) return e;
+    ttm_fibre_compact_kernel<<<grid, 256, 0, c.stream>>>(n_ij, flags, fpos, Acrd1, rowptr_raw, Ccrd1, Cpos2);
+    if (n_i > 0) ttm_slice_flags_kernel<<<grid, 256, 0, c.stream>>>(n_i, Apos1, fpos, sflags);
+    e = launch_scan_counts(c, sflags, n_i, spos, block_sums, nullptr);
+    if (e != cudaSuccess) return e;
+    ttm_slice_compact_kernel<<<grid, 256, 0, c.stream>>>(n_i, n_ij, sflags, spos, Apos1, fpos, Acrd0, Ccrd0, Cpos1, Cpos0, c.ctl);
+    return cudaGetLastError();
+}
+
+}  // namespace spws

@@ -1,0 +1,575 @@
+// C ABI of the spws library: handles, plans, expression check, scratch layout and the launch
+// sequences of the symbolic and numeric passes.  Host code only.
+#include <cctype>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/spws.h"
+#include "common.cuh"
+
+using namespace spws;
+
+struct spws_handle_s {
+    cudaStream_t stream = nullptr;
+    int device = 0;
+    int sm_count = 0;
+};
+
+struct spws_plan_s {
+    spws_handle_t h = nullptr;
+    int kind = 0;               // 0 SpGEMM (CSR x CSR -> CSR), 1 TTM (CSF3 x CSR -> CSF3)
+    int is_f64 = 1;
+    int policy = SPWS_AUTO;
+    spws_options_t opt{};
+    DevCtl* host_ctl = nullptr; // pinned
+    bool symbolic_ok = false;
+    spws_stats_t stats{};
+    // what the last symbolic pass saw (numeric must be called with the same shapes and scratch)
+    int64_t m = 0;
+    void* scratch = nullptr;
+};
+
+namespace {
+
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+// int64_t is `long` on this ABI, the kernels use `long long`: same width, distinct types
+inline i64* LL(int64_t* p) { return reinterpret_cast<i64*>(p); }
+inline const i64* LL(const int64_t* p) { return reinterpret_cast<const i64*>(p); }
+
+// ---- expression -------------------------------------------------------------------------
+struct Access { std::string name; std::vector<std::string> idx; };
+
+bool parse_access(const char*& s, Access& a) {
+    while (*s && isspace((unsigned char)*s)) ++s;
+    if (!(isalpha((unsigned char)*s) || *s == '_')) return false;
+    while (isalnum((unsigned char)*s) || *s == '_') a.name.push_back(*s++);
+    while (*s && isspace((unsigned char)*s)) ++s;
+    if (*s != '(') return false;
+    ++s;
+    for (;;) {
+        while (*s && isspace((unsigned char)*s)) ++s;
+        std::string v;
+        if (!(isalpha((unsigned char)*s) || *s == '_')) return false;
+        while (isalnum((unsigned char)*s) || *s == '_') v.push_back(*s++);
+        a.idx.push_back(v);
+        while (*s && isspace((unsigned char)*s)) ++s;
+        if (*s == ',') { ++s; continue; }
+        if (*s == ')') { ++s; break; }
+        return false;
+    }
+    while (*s && isspace((unsigned char)*s)) ++s;
+    return true;
+}
+
+bool distinct(const std::vector<std::string>& v) {
+    for (size_t a = 0; a < v.size(); ++a)
+        for (size_t b = a + 1; b < v.size(); ++b)
+            if (v[a] == v[b]) return false;
+    return true;
+}
+
+// Accepts out(o_1..o_N) = x(o_1..o_{N-1}, r) * y(r, o_N), N = 2 or 3, with formats
+// (CSR, CSR, CSR) or (CSF3, CSF3, CSR): loop order o_1 -> .. -> r -> o_N, output order
+// o_1 -> .. -> o_N; they mismatch only by the reduction variable sitting one position from the
+// innermost index: a first-order scatter.  Returns the kind or -1.
+int classify_expression(const char* expr, const spws_format_t fmts[3]) {
+    const char* s = expr;
+    Access out, x, y;
+    if (!parse_access(s, out)) return -1;
+    if (*s == '+' && s[1] == '=') s += 2; else if (*s == '=') s += 1; else return -1;
+    if (!parse_access(s, x)) return -1;
+    if (*s != '*') return -1;
+    ++s;
+    if (!parse_access(s, y)) return -1;
+    if (*s != '\0') return -1;
+    const size_t N = out.idx.size();
+    if (N != 2 && N != 3) return -1;
+    if (x.idx.size() != N || y.idx.size() != 2) return -1;
+    if (!distinct(out.idx) || !distinct(x.idx) || !distinct(y.idx)) return -1;
+    const std::string& r = x.idx[N - 1];
+    for (size_t a = 0; a < N; ++a) if (out.idx[a] == r) return -1;           // r must be a reduction variable
+    for (size_t a = 0; a + 1 < N; ++a) if (x.idx[a] != out.idx[a]) return -1;
+    if (y.idx[0] != r || y.idx[1] != out.idx[N - 1]) return -1;
+    if (out.name == x.name || out.name == y.name) return -1;
+    if (N == 2) {
+        if (fmts[0] != SPWS_CSR || fmts[1] != SPWS_CSR || fmts[2] != SPWS_CSR) return -1;
+        return 0;
+    }
+    if (fmts[0] != SPWS_CSF3 || fmts[1] != SPWS_CSF3 || fmts[2] != SPWS_CSR) return -1;
+    return 1;
+}
+
+bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+// ---- scratch layout ------------------------------------------------------------------------
+struct Layout {
+    size_t ctl, ub, rowptr_raw, cnt, jmin, jmax, cls, perm, row_unit0, unit_row, unit_cnt, block_sums,
+        flags, fpos, sflags, spos, arena, fixed_end;
+    int unit_cap;
+};
+
+Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) {
+    Layout L{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
+    L.ctl = take(sizeof(DevCtl));
+    L.ub = take(8 * (size_t)m);
+    L.rowptr_raw = take(8 * ((size_t)m + 1));
+    L.cnt = take(4 * (size_t)m);
+    L.jmin = take(4 * (size_t)m);
+    L.jmax = take(4 * (size_t)m);
+    L.cls = take((size_t)m);
+    L.perm = take(4 * (size_t)m);
+    L.row_unit0 = take(4 * (size_t)m);
+    int64_t tiles_per_row = (ncols + p->opt.dense_tile_cols - 1) / p->opt.dense_tile_cols;
+    if (tiles_per_row > p->opt.max_dense_tiles) tiles_per_row = p->opt.max_dense_tiles;
+    if (tiles_per_row < 1) tiles_per_row = 1;
+    int64_t ucap = m * tiles_per_row;
+    if (ucap > 0x7fff0000ll) ucap = 0x7fff0000ll;
+    L.unit_cap = (int)ucap;
+    L.unit_row = take(4 * (size_t)ucap);
+    L.unit_cnt = take(4 * (size_t)ucap);
+    const size_t longest = (size_t)(m > n_i ? m : n_i);
+    L.block_sums = take(8 * (longest / 2048 + 2));
+    if (p->kind == 1) {
+        L.flags = take(4 * (size_t)m);
+        L.fpos = take(8 * ((size_t)m + 1));
+        L.sflags = take(4 * (size_t)n_i);
+        L.spos = take(8 * ((size_t)n_i + 1));
+    }
+    L.fixed_end = o;
+    L.arena = o;
+    return L;
+}
+
+// reserve for the global-memory ISM: room for a few slots of min(ncols, 2^22) components
+size_t global_reserve(const spws_plan_s* p, int64_t ncols) {
+    const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
+    const size_t comp = 4 + (p->is_f64 ? 8 : 4);
+    return align256(2 * (size_t)((elems + 63) & ~63ll) * comp) * 8;
+}
+
+struct Shapes {
+    int64_t m, k, ncols, nnzA, nnzB, n_i;
+    Csr A, B;
+};
+
+spws_status_t check_operands(const spws_plan_s* p, const spws_tensor_t* A, const spws_tensor_t* B, Shapes& S,
+                             bool need_pointers = true) {
+    if (!A || !B) return SPWS_INVALID_ARGUMENT;
+    if (B->order != 2) return SPWS_INVALID_ARGUMENT;
+    if (p->kind == 0) {
+        if (A->order != 2) return SPWS_INVALID_ARGUMENT;
+        S.m = A->dims[0]; S.k = A->dims[1]; S.nnzA = A->n[1]; S.n_i = 0;
+        S.A = Csr{LL(A->pos[1]), A->crd[1], A->val, (int)S.m, (int)S.k};
+    } else {
+        if (A->order != 3) return SPWS_INVALID_ARGUMENT;
+        S.m = A->n[1]; S.k = A->dims[2]; S.nnzA = A->n[2]; S.n_i = A->n[0];
+        S.A = Csr{LL(A->pos[2]), A->crd[2], A->val, (int)S.m, (int)S.k};
+        if (A->n[0] < 0 || A->n[0] > A->dims[0] || A->n[1] < A->n[0]) return SPWS_INVALID_ARGUMENT;
+    }
+    S.ncols = B->dims[1];
+    S.nnzB = B->n[1];
+    S.B = Csr{LL(B->pos[1]), B->crd[1], B->val, (int)B->dims[0], (int)S.ncols};
+    if (S.m < 0 || S.k < 0 || S.ncols < 0 || S.nnzA < 0 || S.nnzB < 0) return SPWS_INVALID_ARGUMENT;
+    if (S.m > 0x7ffffff0ll || S.k > 0x7ffffff0ll || S.ncols > 0x7ffffff0ll || B->dims[0] > 0x7ffffff0ll)
+        return SPWS_INVALID_ARGUMENT;
+    if (S.k != B->dims[0]) return SPWS_DIM_MISMATCH;
+    if (!need_pointers) return SPWS_OK;
+    if (S.m > 0 && (!S.A.pos)) return SPWS_INVALID_ARGUMENT;
+    if (S.nnzA > 0 && (!S.A.crd || !S.A.val)) return SPWS_INVALID_ARGUMENT;
+    if (B->dims[0] > 0 && !S.B.pos) return SPWS_INVALID_ARGUMENT;
+    if (S.nnzB > 0 && (!S.B.crd || !S.B.val)) return SPWS_INVALID_ARGUMENT;
+    return SPWS_OK;
+}
+
+spws_status_t check_output_dims(const spws_plan_s* p, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* C) {
+    if (!C) return SPWS_INVALID_ARGUMENT;
+    if (p->kind == 0) {
+        if (C->order != 2) return SPWS_INVALID_ARGUMENT;
+        if (C->dims[0] != A->dims[0] || C->dims[1] != B->dims[1]) return SPWS_DIM_MISMATCH;
+        if (!C->pos[1]) return SPWS_INVALID_ARGUMENT;
+    } else {
+        if (C->order != 3) return SPWS_INVALID_ARGUMENT;
+        if (C->dims[0] != A->dims[0] || C->dims[1] != A->dims[1] || C->dims[2] != B->dims[1]) return SPWS_DIM_MISMATCH;
+        if (!C->pos[0] || !C->pos[1] || !C->pos[2]) return SPWS_INVALID_ARGUMENT;
+        if (A->n[0] > 0 && !C->crd[0]) return SPWS_INVALID_ARGUMENT;
+        if (A->n[1] > 0 && !C->crd[1]) return SPWS_INVALID_ARGUMENT;
+    }
+    return SPWS_OK;
+}
+
+LaunchCtx make_ctx(const spws_plan_s* p, char* scratch, size_t scratch_bytes, const Layout& L) {
+    LaunchCtx c{};
+    c.stream = p->h->stream;
+    c.sm_count = p->h->sm_count;
+    c.ctl = reinterpret_cast<DevCtl*>(scratch + L.ctl);
+    c.prm.policy = p->policy;
+    c.prm.reg_cap = p->opt.ism_warp_cap;
+    c.prm.smem_cap = p->opt.ism_cta_cap;
+    c.prm.smem_small_cap = p->opt.ism_cta_cap >= 1024 ? 256 : (p->opt.ism_cta_cap >= 256 ? 64 : p->opt.ism_cta_cap);
+    c.prm.tile_cols = p->opt.dense_tile_cols;
+    c.prm.max_tiles = p->opt.max_dense_tiles;
+    c.prm.span_words_per_product = p->opt.dense_span_words_per_product;
+    c.prm.unit_cap = L.unit_cap;
+    c.tab.ub = reinterpret_cast<i64*>(scratch + L.ub);
+    c.tab.cnt = reinterpret_cast<int*>(scratch + L.cnt);
+    c.tab.jmin = reinterpret_cast<int*>(scratch + L.jmin);
+    c.tab.jmax = reinterpret_cast<int*>(scratch + L.jmax);
+    c.tab.cls = reinterpret_cast<unsigned char*>(scratch + L.cls);
+    c.tab.perm = reinterpret_cast<int*>(scratch + L.perm);
+    c.tab.row_unit0 = reinterpret_cast<int*>(scratch + L.row_unit0);
+    c.tab.unit_row = reinterpret_cast<int*>(scratch + L.unit_row);
+    c.tab.unit_cnt = reinterpret_cast<int*>(scratch + L.unit_cnt);
+    c.is_f64 = p->is_f64;
+    c.global_arena = scratch + L.arena;
+    c.global_arena_bytes = scratch_bytes > L.arena ? scratch_bytes - L.arena : 0;
+    c.global_cap = p->opt.fallback_cap;
+    return c;
+}
+
+spws_status_t from_dev_status(int s) {
+    switch (s) {
+        case DEV_OK: return SPWS_OK;
+        case DEV_NONCANONICAL: return SPWS_NONCANONICAL_INPUT;
+        case DEV_SCRATCH_TOO_SMALL: return SPWS_SCRATCH_TOO_SMALL;
+        case DEV_WORKSPACE_TOO_LARGE: return SPWS_WORKSPACE_TOO_LARGE;
+        default: return SPWS_INTERNAL_OVERFLOW;
+    }
+}
+
+#define CUDA_TRY(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return SPWS_CUDA_ERROR; } } while (0)
+
+}  // namespace
+
+extern "C" {
+
+spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3], int* kind) {
+    if (!expr || !fmts) return SPWS_INVALID_ARGUMENT;
+    for (int f = 0; f < 3; ++f)
+        if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3) return SPWS_INVALID_ARGUMENT;
+    const int k = classify_expression(expr, fmts);
+    if (k < 0) return SPWS_UNSUPPORTED_EXPRESSION;
+    if (kind) *kind = k;
+    return SPWS_OK;
+}
+
+spws_status_t spws_create(spws_handle_t* handle) {
+    if (!handle) return SPWS_INVALID_ARGUMENT;
+    spws_handle_s* h = new (std::nothrow) spws_handle_s;
+    if (!h) return SPWS_INVALID_ARGUMENT;
+    if (cudaGetDevice(&h->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) {
+        cudaGetLastError();
+        delete h;
+        return SPWS_CUDA_ERROR;
+    }
+    *handle = h;
+    return SPWS_OK;
+}
+
+spws_status_t spws_destroy(spws_handle_t handle) {
+    if (!handle) return SPWS_INVALID_ARGUMENT;
+    delete handle;
+    return SPWS_OK;
+}
+
+spws_status_t spws_set_stream(spws_handle_t handle, void* cuda_stream) {
+    if (!handle) return SPWS_INVALID_ARGUMENT;
+    handle->stream = static_cast<cudaStream_t>(cuda_stream);
+    return SPWS_OK;
+}
+
+spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spws_format_t fmts[3],
+                               spws_dtype_t value_type, spws_policy_t policy, const spws_options_t* options,
+                               spws_plan_t* plan) {
+    if (!handle || !expr || !fmts || !plan) return SPWS_INVALID_ARGUMENT;
+    if (value_type != SPWS_F32 && value_type != SPWS_F64) return SPWS_INVALID_ARGUMENT;
+    if (policy != SPWS_DENSE && policy != SPWS_SPARSE_ISM && policy != SPWS_AUTO) return SPWS_INVALID_ARGUMENT;
+    for (int f = 0; f < 3; ++f)
+        if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3) return SPWS_INVALID_ARGUMENT;
+    const int kind = classify_expression(expr, fmts);
+    if (kind < 0) return SPWS_UNSUPPORTED_EXPRESSION;
+    spws_options_t o{};
+    if (options) o = *options;
+    const bool f64 = value_type == SPWS_F64;
+    if (o.ism_warp_cap == 0) o.ism_warp_cap = 32;
+    if (o.ism_cta_cap == 0) o.ism_cta_cap = 4096;
+    if (o.dense_tile_cols == 0) o.dense_tile_cols = f64 ? 8192 : 16384;
+    if (o.max_dense_tiles == 0) o.max_dense_tiles = 64;
+    if (o.fallback_cap == 0) o.fallback_cap = 2048;
+    if (o.dense_span_words_per_product == 0.0f) o.dense_span_words_per_product = 4.0f;
+    if (o.validate != 0 && o.validate != 1) return SPWS_INVALID_ARGUMENT;
+    if (o.ism_warp_cap < 1 || o.ism_warp_cap > 32) return SPWS_INVALID_ARGUMENT;
+    if (!is_pow2(o.ism_cta_cap) || o.ism_cta_cap < 64 || o.ism_cta_cap > 4096) return SPWS_INVALID_ARGUMENT;
+    if (!is_pow2(o.dense_tile_cols) || o.dense_tile_cols < 256 || o.dense_tile_cols > 16384) return SPWS_INVALID_ARGUMENT;
+    if (o.max_dense_tiles < 1 || o.max_dense_tiles > 4096) return SPWS_INVALID_ARGUMENT;
+    if (!is_pow2(o.fallback_cap) || o.fallback_cap < 2 || o.fallback_cap > 2048) return SPWS_INVALID_ARGUMENT;
+    if (!(o.dense_span_words_per_product > 0.0f)) return SPWS_INVALID_ARGUMENT;
+    spws_plan_s* p = new (std::nothrow) spws_plan_s;
+    if (!p) return SPWS_INVALID_ARGUMENT;
+    p->h = handle;
+    p->kind = kind;
+    p->is_f64 = f64 ? 1 : 0;
+    p->policy = (int)policy;
+    p->opt = o;
+    if (cudaMallocHost(reinterpret_cast<void**>(&p->host_ctl), sizeof(DevCtl)) != cudaSuccess) {
+        cudaGetLastError();
+        delete p;
+        return SPWS_CUDA_ERROR;
+    }
+    memset(p->host_ctl, 0, sizeof(DevCtl));
+    *plan = p;
+    return SPWS_OK;
+}
+
+spws_status_t spws_plan_destroy(spws_plan_t plan) {
+    if (!plan) return SPWS_INVALID_ARGUMENT;
+    if (plan->host_ctl) cudaFreeHost(plan->host_ctl);
+    delete plan;
+    return SPWS_OK;
+}
+
+spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, size_t* bytes) {
+    if (!plan || !bytes) return SPWS_INVALID_ARGUMENT;
+    Shapes S{};
+    spws_status_t st = check_operands(plan, A, B, S, false);   // pointers may still be unset when sizing
+    if (st != SPWS_OK) return st;
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
+    *bytes = L.fixed_end + global_reserve(plan, S.ncols);
+    return SPWS_OK;
+}
+
+spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, spws_tensor_t* C,
+                            void* scratch, size_t scratch_bytes, int64_t* sizes_out) {
+    if (!plan) return SPWS_INVALID_ARGUMENT;
+    plan->symbolic_ok = false;
+    Shapes S{};
+    spws_status_t st = check_operands(plan, A, B, S);
+    if (st != SPWS_OK) return st;
+    if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
+    if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return SPWS_INVALID_ARGUMENT;
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
+    if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
+    cudaStream_t stream = c.stream;
+
+    CUDA_TRY(cudaMemsetAsync(c.ctl, 0, sizeof(DevCtl), stream));
+    if (plan->opt.validate) {
+        CUDA_TRY(launch_validate(c, S.A, S.B, S.nnzA, S.nnzB));
+        CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
+        CUDA_TRY(cudaStreamSynchronize(stream));
+        if (plan->host_ctl->status != 0) return from_dev_status(plan->host_ctl->status);
+    }
+    // a1: upper bounds + classes; a2: binning
+    CUDA_TRY(launch_row_bounds(c, S.A, S.B, S.nnzA));
+    CUDA_TRY(launch_bin_rows(c, (int)S.m));
+    // a3: exact count per row through the workspace of its class
+    i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<i64*>(sc + L.rowptr_raw);
+    if (S.m > 0) {
+        CUDA_TRY(launch_ism_reg(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        CUDA_TRY(launch_dense(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        if (plan->policy != SPWS_DENSE)
+            CUDA_TRY(launch_ism_global(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+    }
+    // a4: exclusive scan into the row pointer
+    CUDA_TRY(launch_scan_counts(c, c.tab.cnt, (int)S.m, rowptr, reinterpret_cast<i64*>(sc + L.block_sums), &c.ctl->nnz));
+    if (plan->kind == 1) {
+        CUDA_TRY(launch_ttm_compact(c, (int)S.n_i, (int)S.m, LL(A->pos[1]), A->crd[0], A->crd[1], rowptr,
+                                    reinterpret_cast<int*>(sc + L.flags), reinterpret_cast<i64*>(sc + L.fpos),
+                                    reinterpret_cast<int*>(sc + L.sflags), reinterpret_cast<i64*>(sc + L.spos),
+                                    reinterpret_cast<i64*>(sc + L.block_sums), LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
+    }
+    CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    const DevCtl& hc = *plan->host_ctl;
+    plan->stats = spws_stats_t{};
+    plan->stats.device_status = hc.status;
+    if (hc.status != 0) return from_dev_status(hc.status);
+    plan->stats.rows = S.m;
+    plan->stats.products = hc.products;
+    plan->stats.nnz = hc.nnz;
+    plan->stats.max_row_products = hc.max_ub;
+    for (int k = 0; k < NCLASS; ++k) plan->stats.rows_per_class[k] = hc.class_count[k];
+    plan->stats.dense_units = hc.n_units;
+    if (plan->kind == 0) {
+        C->n[0] = C->dims[0];
+        C->n[1] = hc.nnz;
+        C->n[2] = 0;
+    } else {
+        C->n[0] = hc.kept[0];
+        C->n[1] = hc.kept[1];
+        C->n[2] = hc.nnz;
+    }
+    if (sizes_out) { sizes_out[0] = C->n[0]; sizes_out[1] = C->n[1]; sizes_out[2] = C->n[2]; }
+    plan->symbolic_ok = true;
+    plan->m = S.m;
+    plan->scratch = scratch;
+    return SPWS_OK;
+}
+
+spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, spws_tensor_t* C,
+                           void* scratch, size_t scratch_bytes) {
+    if (!plan) return SPWS_INVALID_ARGUMENT;
+    if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
+    Shapes S{};
+    spws_status_t st = check_operands(plan, A, B, S);
+    if (st != SPWS_OK) return st;
+    if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
+    if (scratch != plan->scratch || S.m != plan->m) return SPWS_BAD_SEQUENCE;
+    const int last = plan->kind == 0 ? 1 : 2;
+    if (C->n[last] < plan->stats.nnz) return SPWS_OUTPUT_TOO_SMALL;
+    if (plan->stats.nnz > 0 && (!C->crd[last] || !C->val)) return SPWS_INVALID_ARGUMENT;
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
+    if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
+    const i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<const i64*>(sc + L.rowptr_raw);
+    CUDA_TRY(cudaMemsetAsync(c.ctl->work_counter, 0, sizeof(c.ctl->work_counter), c.stream));
+    const spws_stats_t& s = plan->stats;
+    int* crd = C->crd[last];
+    if (s.rows_per_class[CLS_ISM_REG] > 0)
+        CUDA_TRY(launch_ism_reg(c, true, (int)s.rows_per_class[CLS_ISM_REG], S.A, S.B, rowptr, crd, C->val));
+    if (s.rows_per_class[CLS_ISM_SMEM_S] > 0)
+        CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM_S, (int)s.rows_per_class[CLS_ISM_SMEM_S], S.A, S.B, rowptr, crd, C->val));
+    if (s.rows_per_class[CLS_ISM_SMEM] > 0)
+        CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM, (int)s.rows_per_class[CLS_ISM_SMEM], S.A, S.B, rowptr, crd, C->val));
+    if (s.dense_units > 0)
+        CUDA_TRY(launch_dense(c, true, (int)s.dense_units, S.A, S.B, rowptr, crd, C->val));
+    if (s.rows_per_class[CLS_ISM_GLOBAL] > 0)
+        CUDA_TRY(launch_ism_global(c, true, (int)s.rows_per_class[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));
+    return SPWS_OK;
+}
+
+spws_status_t spws_get_stats(spws_plan_t plan, spws_stats_t* stats) {
+    if (!plan || !stats) return SPWS_INVALID_ARGUMENT;
+    if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
+    DevCtl* ctl = reinterpret_cast<DevCtl*>(plan->scratch);
+    CUDA_TRY(cudaMemcpyAsync(&plan->host_ctl->status, &ctl->status, sizeof(int), cudaMemcpyDeviceToHost, plan->h->stream));
+    CUDA_TRY(cudaStreamSynchronize(plan->h->stream));
+    plan->stats.device_status = plan->host_ctl->status;
+    *stats = plan->stats;
+    return from_dev_status(plan->host_ctl->status);
+}
+
+spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, spws_tensor_t* C,
+                                void* arena, size_t arena_bytes, size_t* arena_needed) {
+    if (!plan || !A || !B || !C || !arena) return SPWS_INVALID_ARGUMENT;
+    if (reinterpret_cast<uintptr_t>(arena) & 255) return SPWS_INVALID_ARGUMENT;
+    Shapes S{};
+    spws_status_t st = check_operands(plan, A, B, S);
+    if (st != SPWS_OK) return st;
+    cudaStream_t stream = plan->h->stream;
+    const size_t V = plan->is_f64 ? 8 : 4;
+    char* base = static_cast<char*>(arena);
+    size_t o = 0;
+    bool fits = true;
+    auto carve = [&](size_t bytes) -> char* {
+        char* at = base + o;
+        o = align256(o + bytes);
+        if (o > arena_bytes) fits = false;
+        return at;
+    };
+    // device images of the operands
+    spws_tensor_t dA = *A, dB = *B, dC = *C;
+    const int lastA = plan->kind == 0 ? 1 : 2;
+    const bool same = (plan->kind == 0) && A->pos[1] == B->pos[1] && A->crd[1] == B->crd[1] && A->val == B->val;
+    struct Copy { void* dst; const void* src; size_t bytes; };
+    std::vector<Copy> h2d;
+    auto stage = [&](const void* src, size_t bytes) -> void* {
+        char* d = carve(bytes);
+        h2d.push_back(Copy{d, src, bytes});
+        return d;
+    };
+    if (plan->kind == 0) {
+        dA.pos[1] = (int64_t*)stage(A->pos[1], 8 * ((size_t)S.m + 1));
+        dA.crd[1] = (int32_t*)stage(A->crd[1], 4 * (size_t)S.nnzA);
+    } else {
+        dA.pos[0] = (int64_t*)stage(A->pos[0], 16);
+        dA.crd[0] = (int32_t*)stage(A->crd[0], 4 * (size_t)A->n[0]);
+        dA.pos[1] = (int64_t*)stage(A->pos[1], 8 * ((size_t)A->n[0] + 1));
+        dA.crd[1] = (int32_t*)stage(A->crd[1], 4 * (size_t)A->n[1]);
+        dA.pos[2] = (int64_t*)stage(A->pos[2], 8 * ((size_t)A->n[1] + 1));
+        dA.crd[2] = (int32_t*)stage(A->crd[2], 4 * (size_t)S.nnzA);
+    }
+    dA.val = stage(A->val, V * (size_t)S.nnzA);
+    if (same) {
+        dB.pos[1] = dA.pos[1]; dB.crd[1] = dA.crd[1]; dB.val = dA.val;
+    } else {
+        dB.pos[1] = (int64_t*)stage(B->pos[1], 8 * ((size_t)B->dims[0] + 1));
+        dB.crd[1] = (int32_t*)stage(B->crd[1], 4 * (size_t)S.nnzB);
+        dB.val = stage(B->val, V * (size_t)S.nnzB);
+    }
+    (void)lastA;
+    if (plan->kind == 0) {
+        dC.pos[1] = (int64_t*)carve(8 * ((size_t)S.m + 1));
+    } else {
+        dC.pos[0] = (int64_t*)carve(16);
+        dC.crd[0] = (int32_t*)carve(4 * (size_t)A->n[0]);
+        dC.pos[1] = (int64_t*)carve(8 * ((size_t)A->n[0] + 1));
+        dC.crd[1] = (int32_t*)carve(4 * (size_t)A->n[1]);
+        dC.pos[2] = (int64_t*)carve(8 * ((size_t)A->n[1] + 1));
+    }
+    size_t ws_bytes = 0;
+    if ((st = spws_workspace_size(plan, A, B, &ws_bytes)) != SPWS_OK) return st;
+    char* scratch = carve(ws_bytes);
+    if (!fits) {
+        if (arena_needed) *arena_needed = o;      // lower bound: C's entries are not counted yet
+        return SPWS_SCRATCH_TOO_SMALL;
+    }
+    for (const Copy& cp : h2d)
+        if (cp.bytes) CUDA_TRY(cudaMemcpyAsync(cp.dst, cp.src, cp.bytes, cudaMemcpyHostToDevice, stream));
+    int64_t cap[3] = {C->n[0], C->n[1], C->n[2]};
+    int64_t sizes[3];
+    if ((st = spws_symbolic(plan, &dA, &dB, &dC, scratch, ws_bytes, sizes)) != SPWS_OK) return st;
+    const int last = plan->kind == 0 ? 1 : 2;
+    const size_t nnz = (size_t)sizes[last];
+    dC.crd[last] = (int32_t*)carve(4 * nnz);
+    dC.val = carve(V * nnz);
+    if (arena_needed) *arena_needed = o;
+    C->n[0] = sizes[0]; C->n[1] = sizes[1]; C->n[2] = sizes[2];
+    if (!fits) return SPWS_SCRATCH_TOO_SMALL;
+    if ((int64_t)nnz > cap[last]) return SPWS_OUTPUT_TOO_SMALL;
+    if (plan->kind == 1 && (sizes[0] > cap[0] || sizes[1] > cap[1])) return SPWS_OUTPUT_TOO_SMALL;
+    if ((st = spws_numeric(plan, &dA, &dB, &dC, scratch, ws_bytes)) != SPWS_OK) return st;
+    if (plan->kind == 0) {
+        CUDA_TRY(cudaMemcpyAsync(C->pos[1], dC.pos[1], 8 * ((size_t)S.m + 1), cudaMemcpyDeviceToHost, stream));
+    } else {
+        CUDA_TRY(cudaMemcpyAsync(C->pos[0], dC.pos[0], 16, cudaMemcpyDeviceToHost, stream));
+        if (sizes[0]) CUDA_TRY(cudaMemcpyAsync(C->crd[0], dC.crd[0], 4 * (size_t)sizes[0], cudaMemcpyDeviceToHost, stream));
+        CUDA_TRY(cudaMemcpyAsync(C->pos[1], dC.pos[1], 8 * ((size_t)sizes[0] + 1), cudaMemcpyDeviceToHost, stream));
+        if (sizes[1]) CUDA_TRY(cudaMemcpyAsync(C->crd[1], dC.crd[1], 4 * (size_t)sizes[1], cudaMemcpyDeviceToHost, stream));
+        CUDA_TRY(cudaMemcpyAsync(C->pos[2], dC.pos[2], 8 * ((size_t)sizes[1] + 1), cudaMemcpyDeviceToHost, stream));
+    }
+    if (nnz) {
+        CUDA_TRY(cudaMemcpyAsync(C->crd[last], dC.crd[last], 4 * nnz, cudaMemcpyDeviceToHost, stream));
+        CUDA_TRY(cudaMemcpyAsync(C->val, dC.val, V * nnz, cudaMemcpyDeviceToHost, stream));
+    }
+    spws_stats_t stats;
+    return spws_get_stats(plan, &stats);
+}
+
+const char* spws_status_string(spws_status_t status) {
+    switch (status) {
+        case SPWS_OK: return "ok";
+        case SPWS_INVALID_ARGUMENT: return "invalid argument";
+        case SPWS_UNSUPPORTED_EXPRESSION: return "unsupported expression";
+        case SPWS_DIM_MISMATCH: return "dimension mismatch";
+        case SPWS_NONCANONICAL_INPUT: return "non-canonical input";
+        case SPWS_SCRATCH_TOO_SMALL: return "scratch too small";
+        case SPWS_WORKSPACE_TOO_LARGE: return "dense workspace too large";
+        case SPWS_CUDA_ERROR: return "CUDA error";
+        case SPWS_INTERNAL_OVERFLOW: return "internal overflow";
+        case SPWS_OUTPUT_TOO_SMALL: return "output too small";
+        case SPWS_BAD_SEQUENCE: return "bad call sequence";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

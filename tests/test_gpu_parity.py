@@ -1,0 +1,354 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI (ctypes binding).
+
+Structure (pos / crd) must match bit for bit; values within 1e-12 (f64) / 1e-5 (f32) relative
+per entry, or within that factor of sum|a*b| where mixed-sign products cancel.
+"""
+import numpy as np
+import pytest
+
+from helpers import TOL, read_hand_case, rows_of, values_close
+from workloads import (CSR, CSF3, config_inputs, random_csr, rmat_csr, stencil27_csr, uniform_csf3,
+                       uniform_rows_csr)
+
+pytestmark = pytest.mark.gpu
+
+POLICIES = ("dense", "ism", "auto")
+# thresholds that force every route on small inputs
+SMALL_ROUTES = dict(ism_warp_cap=8, ism_cta_cap=64, dense_tile_cols=256, max_dense_tiles=4096, fallback_cap=16)
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import torch
+    from paper_2404_04541_b200 import api
+    assert torch.cuda.is_available()
+    return api.Context("cuda")
+
+
+def run_spgemm(ctx, A, B, policy="auto", **options):
+    from paper_2404_04541_b200 import api
+    dA = api.DeviceCSR.from_host(A)
+    dB = dA if B is A else api.DeviceCSR.from_host(B)
+    C, stats = ctx.spgemm(dA, dB, policy=policy, **options)
+    return C.pos.cpu().numpy(), C.crd.cpu().numpy(), C.val.cpu().numpy(), stats
+
+
+def assert_matches(got, ref, dtype, rows=None, exact_values=False):
+    pos, crd, val = got
+    assert np.array_equal(pos, ref.pos), "row pointer differs"
+    assert np.array_equal(crd, ref.crd), "column indices differ"
+    if exact_values:
+        assert np.array_equal(val, ref.val.astype(dtype))
+        return 0
+    ok, second = values_close(val, ref.val_ref, ref.abs, TOL[np.dtype(dtype)])
+    assert ok.all(), f"{(~ok).sum()} of {ok.size} values out of tolerance"
+    return second
+
+
+def check_spgemm(ctx, oracle_mod, A, B, policy="auto", exact_values=False, threads=4, **options):
+    ref = oracle_mod.spgemm(A, B, threads=threads)
+    pos, crd, val, stats = run_spgemm(ctx, A, B, policy, **options)
+    assert stats["products"] == int(ref.products.sum())
+    assert stats["nnz"] == ref.nnz
+    assert_matches((pos, crd, val), ref, A.val.dtype, exact_values=exact_values)
+    return stats
+
+
+# ------------------------------------------------------------------ hand-worked cases
+@pytest.mark.parametrize("policy", POLICIES)
+@pytest.mark.parametrize("name", ["hand_dedupe_4x4.txt", "hand_cancel_4x4.txt", "hand_rect_3x5x4.txt"])
+def test_hand_cases(ctx, name, policy):
+    A, B, cr, cc, cv, products = read_hand_case(name)
+    pos, crd, val, stats = run_spgemm(ctx, A, B, policy)
+    assert np.array_equal(rows_of(pos), cr) and np.array_equal(crd, cc) and np.array_equal(val, cv)
+    assert stats["products"] == products.sum()
+
+
+# ------------------------------------------------------------------ random small, every route
+@pytest.mark.parametrize("policy", POLICIES)
+@pytest.mark.parametrize("m,k,n,dens,seed", [(1, 1, 1, 1.0, 0), (37, 64, 700, 0.08, 1), (200, 150, 1000, 0.05, 2),
+                                             (64, 64, 64, 0.5, 3), (129, 300, 5000, 0.02, 4)])
+def test_random_small_all_routes(ctx, oracle_mod, policy, m, k, n, dens, seed):
+    A = random_csr(m, k, dens, seed, empty_row_frac=0.1)
+    B = random_csr(k, n, dens, seed + 9, empty_row_frac=0.1)
+    check_spgemm(ctx, oracle_mod, A, B, policy)                      # default thresholds
+    stats = check_spgemm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
+    if policy == "ism" and m >= 37:
+        assert stats["rows_per_class"][5] > 0                        # the global-memory ISM ran
+    if policy == "dense" and n >= 700:
+        assert stats["dense_units"] > stats["rows_per_class"][4]      # some row used several tiles
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+@pytest.mark.parametrize("policy", POLICIES)
+def test_policy_equivalence_and_dtypes(ctx, oracle_mod, policy, dtype):
+    A = random_csr(300, 300, 0.03, 5, dtype=dtype, empty_row_frac=0.05)
+    check_spgemm(ctx, oracle_mod, A, A, policy, **SMALL_ROUTES)
+    check_spgemm(ctx, oracle_mod, A, A, policy)
+
+
+def _rows_with_products(targets, ncols, seed, dtype=np.float64):
+    """A (R x 2R), B (2R x ncols): row r of A*B has exactly targets[r] products, about half of
+    them colliding."""
+    rng = np.random.default_rng(seed)
+    R = len(targets)
+    rows, cols, vals = [], [], []
+    for r, P in enumerate(targets):
+        l0, l1 = (P + 1) // 2, P // 2
+        width = min(ncols, max(l0, int(1.5 * l0) + 1))
+        lo = int(rng.integers(0, ncols - width + 1))
+        for b, ln in ((2 * r, l0), (2 * r + 1, l1)):
+            c = np.sort(rng.choice(width, size=ln, replace=False)) + lo
+            rows.append(np.full(ln, b)); cols.append(c); vals.append(rng.uniform(-1, 1, ln))
+    Bm = CSR.from_coo(2 * R, ncols, np.concatenate(rows), np.concatenate(cols), np.concatenate(vals), dtype=dtype)
+    Am = CSR.from_coo(R, 2 * R, np.repeat(np.arange(R), 2), np.arange(2 * R), rng.uniform(-1, 1, 2 * R), dtype=dtype)
+    return Am, Bm
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_capacity_boundaries(ctx, oracle_mod, policy):
+    targets = [1, 2, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 255, 256, 257, 1023, 1024, 1025,
+               4095, 4096, 4097, 8191, 8192, 8193, 20000]
+    A, B = _rows_with_products(targets, 40000, 11)
+    stats = check_spgemm(ctx, oracle_mod, A, B, policy)
+    assert stats["max_row_products"] == 20000
+    if policy == "ism":
+        assert stats["rows_per_class"][5] == 5                       # rows above the shared-memory capacity
+    A, B = _rows_with_products(targets[:17], 3000, 12)
+    check_spgemm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_edge_cases(ctx, oracle_mod, policy):
+    # all-empty A, empty B rows, one huge row among empty ones
+    z = np.zeros(0)
+    A0 = CSR.from_coo(5, 6, z, z, z)
+    B0 = random_csr(6, 9, 0.5, 1)
+    check_spgemm(ctx, oracle_mod, A0, B0, policy)
+    A1 = random_csr(20, 30, 0.3, 2)
+    B1 = CSR.from_coo(30, 40, z, z, z)
+    check_spgemm(ctx, oracle_mod, A1, B1, policy)
+    rng = np.random.default_rng(3)
+    cols = np.sort(rng.choice(3000, 2000, replace=False))
+    A2 = CSR.from_coo(50, 3000, np.full(2000, 17), cols, rng.uniform(-1, 1, 2000))
+    B2 = uniform_rows_csr(3000, 5000, 40, 4)
+    stats = check_spgemm(ctx, oracle_mod, A2, B2, policy)
+    assert stats["max_row_products"] == 80000 and stats["rows_per_class"][0] == 49
+    # many A entries that pick empty B rows: a row with few products but a long A row
+    live = np.nonzero(rng.random(3000) < 0.01)[0]
+    B3 = CSR.from_coo(3000, 5000, np.repeat(live, 5),
+                      np.concatenate([np.sort(rng.choice(5000, 5, replace=False)) for _ in live]),
+                      rng.uniform(-1, 1, 5 * live.size))
+    check_spgemm(ctx, oracle_mod, A2, B3, policy)
+
+
+def test_ism_routes_reproduce_sequential_sum(ctx, oracle_mod):
+    """The ISM routes add each row's products in loop order with separate multiply and add, so
+    they give the oracle's plain double-precision sum bit for bit."""
+    A = random_csr(200, 200, 0.04, 8)
+    ref = oracle_mod.spgemm(A, A)
+    for opts in ({}, SMALL_ROUTES):
+        pos, crd, val, _ = run_spgemm(ctx, A, A, "ism", **opts)
+        assert np.array_equal(pos, ref.pos) and np.array_equal(crd, ref.crd) and np.array_equal(val, ref.val)
+
+
+# ------------------------------------------------------------------ benchmark configurations
+@pytest.mark.parametrize("policy", POLICIES)
+@pytest.mark.parametrize("cfg", ["uniform8", "rmat18", "stencil64"])
+def test_reduced_configs(ctx, oracle_mod, cfg, policy):
+    c = config_inputs(cfg, reduced=True)
+    check_spgemm(ctx, oracle_mod, c["A"], c["B"], policy)
+
+
+@pytest.mark.parametrize("policy", ["ism", "auto"])
+def test_wide_reduced(ctx, oracle_mod, policy):
+    c = config_inputs("wide26", reduced=True)
+    check_spgemm(ctx, oracle_mod, c["A"], c["B"], policy)
+
+
+def test_dense_policy_refuses_prohibitive_workspace(ctx):
+    from paper_2404_04541_b200 import binding
+    c = config_inputs("wide26", reduced=True)
+    with pytest.raises(binding.SpwsError) as e:
+        run_spgemm(ctx, c["A"], c["B"], "dense")
+    assert e.value.status == binding.SPWS_WORKSPACE_TOO_LARGE
+
+
+def test_full_uniform8(ctx, oracle_mod):
+    c = config_inputs("uniform8")
+    stats = check_spgemm(ctx, oracle_mod, c["A"], c["B"], "auto")
+    assert stats["products"] == 131072
+
+
+def test_full_stencil64(ctx, oracle_mod):
+    c = config_inputs("stencil64")
+    stats = check_spgemm(ctx, oracle_mod, c["A"], c["B"], "auto", threads=oracle_mod.hardware_threads())
+    assert stats["products"] == 566 ** 3 and stats["nnz"] == 314 ** 3
+
+
+def test_full_wide26(ctx, oracle_mod):
+    c = config_inputs("wide26")
+    A, B = c["A"], c["B"]
+    ref = oracle_mod.spgemm(A, B, threads=4)
+    pos, crd, val, stats = run_spgemm(ctx, A, B, "auto")
+    assert stats["rows_per_class"][1] == A.nrows                     # register ISM for every row
+    second = assert_matches((pos, crd, val), ref, np.float32)
+    single = np.repeat(ref.products == np.diff(ref.pos), np.diff(ref.pos))   # rows without any collision
+    assert np.array_equal(val[single], ref.val[single].astype(np.float32))   # one correctly rounded multiply
+    assert second <= ref.nnz - single.sum()
+
+
+def test_full_rmat18_sampled_rows_and_invariants(ctx, oracle_mod):
+    """Full-size power-law config in the launch configuration the benchmark times: the row
+    pointer is checked against properties that hold at any size, and sampled rows (the heaviest
+    ones included) against the oracle entry by entry."""
+    import torch
+    from paper_2404_04541_b200 import api
+    c = config_inputs("rmat18")
+    A = c["A"]
+    dA = api.DeviceCSR.from_host(A)
+    C, stats = ctx.spgemm(dA, dA, policy="auto")
+    lens = np.diff(A.pos)
+    ub = np.bincount(rows_of(A.pos), weights=lens[A.crd], minlength=A.nrows).astype(np.int64)
+    assert stats["products"] == ub.sum()
+    pos = C.pos.cpu().numpy()
+    cnt = np.diff(pos)
+    assert pos[0] == 0 and pos[-1] == stats["nnz"] == C.crd.shape[0]
+    assert (cnt <= np.minimum(ub, A.ncols)).all() and ((cnt == 0) == (ub == 0)).all()
+    # sorted and unique inside every row (checked on the device)
+    crd = C.crd
+    inc = torch.ones(crd.shape[0], dtype=torch.bool, device=crd.device)
+    inc[1:] = crd[1:] > crd[:-1]
+    starts = C.pos[:-1][torch.from_numpy(cnt > 0).to(crd.device)]
+    inc[starts] = True
+    assert bool(inc.all())
+    # C*1 = A*(B*1)
+    b1 = np.bincount(rows_of(A.pos), weights=A.val, minlength=A.nrows)
+    ab1 = np.bincount(rows_of(A.pos), weights=A.val * b1[A.crd], minlength=A.nrows)
+    absb1 = np.bincount(rows_of(A.pos), weights=np.abs(A.val), minlength=A.nrows)
+    scale = np.bincount(rows_of(A.pos), weights=np.abs(A.val) * absb1[A.crd], minlength=A.nrows)
+    rowid = torch.repeat_interleave(torch.arange(A.nrows, device=crd.device), torch.from_numpy(cnt).to(crd.device))
+    c1 = torch.zeros(A.nrows, dtype=torch.float64, device=crd.device).index_add_(0, rowid, C.val).cpu().numpy()
+    assert (np.abs(c1 - ab1) <= 1e-12 * scale + 1e-300).all()
+    # sampled rows against the oracle: the 3 heaviest, 3 around each class boundary, 300 random
+    order = np.argsort(ub)
+    rng = np.random.default_rng(0)
+    pick = set(order[-3:].tolist()) | set(rng.choice(A.nrows, 300, replace=False).tolist())
+    for edge in (32, 256, 4096):
+        near = np.argsort(np.abs(ub - edge))[:3]
+        pick |= set(near.tolist())
+    rows = np.array(sorted(pick))
+    ref = oracle_mod.spgemm(A, A, rows=rows, threads=oracle_mod.hardware_threads())
+    crd_h = None
+    for t, r in enumerate(rows):
+        s, e = int(pos[r]), int(pos[r + 1])
+        assert e - s == ref.pos[t + 1] - ref.pos[t]
+        got_c = C.crd[s:e].cpu().numpy()
+        got_v = C.val[s:e].cpu().numpy()
+        u = slice(ref.pos[t], ref.pos[t + 1])
+        assert np.array_equal(got_c, ref.crd[u])
+        ok, _ = values_close(got_v, ref.val_ref[u], ref.abs[u], 1e-12)
+        assert ok.all()
+
+
+# ------------------------------------------------------------------ TTM
+def run_ttm(ctx, A, B, policy="auto", **options):
+    from paper_2404_04541_b200 import api
+    C, stats = ctx.ttm(api.DeviceCSF3.from_host(A), api.DeviceCSR.from_host(B), policy=policy, **options)
+    f = lambda t: t.cpu().numpy()
+    return dict(pos0=f(C.pos0), crd0=f(C.crd0), pos1=f(C.pos1), crd1=f(C.crd1), pos2=f(C.pos2), crd2=f(C.crd2),
+                val=f(C.val)), stats
+
+
+def check_ttm(ctx, oracle_mod, A, B, policy="auto", **options):
+    ref = oracle_mod.ttm(A, B)
+    got, stats = run_ttm(ctx, A, B, policy, **options)
+    for name in ("pos0", "crd0", "pos1", "crd1", "pos2", "crd2"):
+        assert np.array_equal(got[name], getattr(ref, name)), name
+    ok, _ = values_close(got["val"], ref.val_ref, ref.abs, TOL[np.dtype(A.val.dtype)])
+    assert ok.all()
+    assert stats["products"] == ref.products.sum()
+    return stats
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_ttm_small_and_empty_fibres(ctx, oracle_mod, policy):
+    A = CSF3.from_coo((3, 3, 4), [0, 0, 1, 1, 2], [0, 2, 0, 1, 1], [1, 0, 1, 2, 3], [1.0, 2.0, 3.0, 4.0, 5.0])
+    B = CSR.from_coo(4, 5, [0, 0, 3], [4, 1, 2], [10.0, 20.0, 30.0])
+    got, _ = run_ttm(ctx, A, B, policy)
+    assert list(got["crd0"]) == [0, 2] and list(got["pos1"]) == [0, 1, 2] and list(got["crd1"]) == [2, 1]
+    assert list(got["pos2"]) == [0, 2, 3] and list(got["crd2"]) == [1, 4, 2] and list(got["val"]) == [40.0, 20.0, 150.0]
+    for dims, nnz, seed in (((8, 8, 8), 100, 1), ((20, 30, 40), 3000, 2), ((64, 64, 64), 20000, 3)):
+        A = uniform_csf3(dims, nnz, seed)
+        B = random_csr(dims[2], 300, 0.05, seed + 5, empty_row_frac=0.5)
+        check_ttm(ctx, oracle_mod, A, B, policy)
+        check_ttm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
+
+
+@pytest.mark.parametrize("reduced", [True, False])
+def test_ttm_config(ctx, oracle_mod, reduced):
+    c = config_inputs("ttm4096", reduced=reduced)
+    stats = check_ttm(ctx, oracle_mod, c["A"], c["B"], "auto")
+    assert stats["products"] == 8 * c["A"].nnz
+
+
+# ------------------------------------------------------------------ boundary behaviour
+def test_error_statuses(ctx):
+    import torch
+    from paper_2404_04541_b200 import api, binding
+    with pytest.raises(binding.SpwsError) as e:
+        ctx.plan("C(i,j) = A(k,i) * B(k,j)", (0, 0, 0), np.float64)
+    assert e.value.status == binding.SPWS_UNSUPPORTED_EXPRESSION
+    A = api.DeviceCSR.from_host(random_csr(10, 12, 0.3, 1))
+    Bm = api.DeviceCSR.from_host(random_csr(13, 9, 0.3, 2))
+    with pytest.raises(binding.SpwsError) as e:
+        ctx.spgemm(A, Bm)
+    assert e.value.status == binding.SPWS_DIM_MISMATCH
+    # scratch too small / numeric before symbolic
+    plan = ctx.plan(api.EXPR_SPGEMM, (0, 0, 0), np.float64)
+    Bok = api.DeviceCSR.from_host(random_csr(12, 9, 0.3, 2))
+    a, b = A.arrays(), Bok.arrays()
+    pos = torch.empty(11, dtype=torch.int64, device="cuda")
+    c = binding.csr_arrays(10, 9, pos, None, None)
+    sc = ctx.scratch(plan.workspace_size(a, b))
+    with pytest.raises(binding.SpwsError) as e:
+        plan.symbolic(a, b, c, ctx._aligned_ptr(sc), 64)
+    assert e.value.status == binding.SPWS_SCRATCH_TOO_SMALL
+    with pytest.raises(binding.SpwsError) as e:
+        plan.numeric(a, b, c, ctx._aligned_ptr(sc), plan.workspace_size(a, b))
+    assert e.value.status == binding.SPWS_BAD_SEQUENCE
+    plan.close()
+    # non-canonical input is reported when validation is on
+    bad = random_csr(12, 9, 0.6, 3)
+    bad.crd[0], bad.crd[1] = bad.crd[1], bad.crd[0]
+    with pytest.raises(binding.SpwsError) as e:
+        ctx.spgemm(A, api.DeviceCSR.from_host(bad), validate=1)
+    assert e.value.status == binding.SPWS_NONCANONICAL_INPUT
+    oob = random_csr(10, 12, 0.3, 1)
+    oob.crd[2] = 12
+    with pytest.raises(binding.SpwsError) as e:
+        ctx.spgemm(api.DeviceCSR.from_host(oob), Bok)
+    assert e.value.status == binding.SPWS_NONCANONICAL_INPUT
+
+
+def test_execute_host_matches(ctx, oracle_mod):
+    import torch
+    from paper_2404_04541_b200 import api, binding
+    A = rmat_csr(10, 8, 3)
+    ref = oracle_mod.spgemm(A, A)
+    plan = ctx.plan(api.EXPR_SPGEMM, (0, 0, 0), np.float64)
+    a = binding.csr_arrays(A.nrows, A.ncols, A.pos, A.crd, A.val)
+    cpos = np.empty(A.nrows + 1, dtype=np.int64)
+    ccrd = np.empty(ref.nnz + 10, dtype=np.int32)
+    cval = np.empty(ref.nnz + 10, dtype=np.float64)
+    c = binding.csr_arrays(A.nrows, A.ncols, cpos, ccrd, cval)
+    arena = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    st, sizes, need = plan.execute_host(a, a, c, ctx._aligned_ptr(arena), arena.numel() - 256)
+    assert st == 0 and sizes[1] == ref.nnz and 0 < need <= arena.numel()
+    assert np.array_equal(cpos, ref.pos) and np.array_equal(ccrd[:ref.nnz], ref.crd)
+    ok, _ = values_close(cval[:ref.nnz], ref.val_ref, ref.abs, 1e-12)
+    assert ok.all()
+    c.n = [A.nrows, 5, 0]                                              # capacity too small
+    st, sizes, _ = plan.execute_host(a, a, c, ctx._aligned_ptr(arena), arena.numel() - 256)
+    assert st == binding.SPWS_OUTPUT_TOO_SMALL and sizes[1] == ref.nnz
+    plan.close()
