@@ -111,7 +111,29 @@ typedef struct {
     int64_t dense_units;      /* (row, column tile) work units of the dense route                 */
     int32_t device_status;    /* last status word read back from the device                      */
     int32_t reserved;
+    int64_t products_per_class[8];
+    int64_t nnz_per_class[8];
+    int32_t launches_symbolic; /* kernels enqueued by the last spws_symbolic / spws_numeric       */
+    int32_t launches_numeric;
 } spws_stats_t;
+
+/* Kernel groups timed by spws_set_profiling (index into the array spws_get_timings fills). */
+enum {
+    SPWS_T_SYM_BOUNDS = 0,    /* per-row upper bound, span and class                               */
+    SPWS_T_SYM_BIN = 1,       /* binning + dense work units                                        */
+    SPWS_T_SYM_ISM_REG = 2,
+    SPWS_T_SYM_ISM_SMEM_S = 3,
+    SPWS_T_SYM_ISM_SMEM = 4,
+    SPWS_T_SYM_DENSE = 5,
+    SPWS_T_SYM_ISM_GLOBAL = 6,
+    SPWS_T_SYM_SCAN = 7,      /* exclusive scan (+ CSF level rebuild for the 3-tensor form)        */
+    SPWS_T_NUM_ISM_REG = 8,
+    SPWS_T_NUM_ISM_SMEM_S = 9,
+    SPWS_T_NUM_ISM_SMEM = 10,
+    SPWS_T_NUM_DENSE = 11,
+    SPWS_T_NUM_ISM_GLOBAL = 12,
+    SPWS_T_COUNT = 13
+};
 
 spws_status_t spws_create(spws_handle_t* handle);
 spws_status_t spws_destroy(spws_handle_t handle);
@@ -156,6 +178,14 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
 
 /* Synchronises the plan's stream and reports the last symbolic pass's statistics. */
 spws_status_t spws_get_stats(spws_plan_t plan, spws_stats_t* stats);
+
+/* Per-kernel timing for measurement (Sec. 7.1 reports kernel runtimes; the split by kernel is
+ * this library's).  With profiling on, both passes record a CUDA event on the plan's stream after
+ * every kernel group; spws_get_timings synchronises the stream and writes the milliseconds of
+ * each group of the last symbolic and numeric pass into ms[0 .. SPWS_T_COUNT) (0 for a group that
+ * did not run).  `n` is the capacity of `ms` and must be at least SPWS_T_COUNT. */
+spws_status_t spws_set_profiling(spws_plan_t plan, int enabled);
+spws_status_t spws_get_timings(spws_plan_t plan, float* ms, int n);
 
 /* Whole path with HOST tensors: copies A and B to the device, runs both passes, copies C back.
  * A, B, C hold host pointers; C's arrays must be allocated with capacities n[] (crd/val of the

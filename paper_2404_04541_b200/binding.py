@@ -33,7 +33,11 @@ POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPAR
 
 EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create", "spws_plan_destroy",
            "spws_check_expression", "spws_workspace_size", "spws_symbolic", "spws_numeric",
-           "spws_get_stats", "spws_execute_host", "spws_status_string")
+           "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host",
+           "spws_status_string")
+TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense",
+                 "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem", "num_dense",
+                 "num_ism_global")
 
 
 class spws_tensor_t(ctypes.Structure):
@@ -52,7 +56,9 @@ class spws_options_t(ctypes.Structure):
 class spws_stats_t(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int64), ("products", ctypes.c_int64), ("nnz", ctypes.c_int64),
                 ("max_row_products", ctypes.c_int64), ("rows_per_class", ctypes.c_int64 * 8),
-                ("dense_units", ctypes.c_int64), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("dense_units", ctypes.c_int64), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("products_per_class", ctypes.c_int64 * 8), ("nnz_per_class", ctypes.c_int64 * 8),
+                ("launches_symbolic", ctypes.c_int32), ("launches_numeric", ctypes.c_int32)]
 
 
 class SpwsError(RuntimeError):
@@ -84,6 +90,8 @@ def lib():
         L.spws_symbolic.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(ctypes.c_int64)]
         L.spws_numeric.argtypes = [vp, T, T, T, vp, sz]
         L.spws_get_stats.argtypes = [vp, ctypes.POINTER(spws_stats_t)]
+        L.spws_set_profiling.argtypes = [vp, i32]
+        L.spws_get_timings.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
         L.spws_execute_host.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(sz)]
         L.spws_status_string.argtypes = [i32]
         L.spws_status_string.restype = ctypes.c_char_p
@@ -218,9 +226,19 @@ class Plan:
         s = spws_stats_t()
         st = lib().spws_get_stats(self._p, ctypes.byref(s))
         d = dict(rows=s.rows, products=s.products, nnz=s.nnz, max_row_products=s.max_row_products,
-                 rows_per_class=list(s.rows_per_class), dense_units=s.dense_units, device_status=s.device_status)
+                 rows_per_class=list(s.rows_per_class), dense_units=s.dense_units, device_status=s.device_status,
+                 products_per_class=list(s.products_per_class), nnz_per_class=list(s.nnz_per_class),
+                 launches_symbolic=s.launches_symbolic, launches_numeric=s.launches_numeric)
         _check(st, "spws_get_stats")
         return d
+
+    def set_profiling(self, enabled: bool):
+        _check(lib().spws_set_profiling(self._p, int(bool(enabled))), "spws_set_profiling")
+
+    def get_timings(self) -> dict:
+        ms = (ctypes.c_float * len(TIMING_GROUPS))()
+        _check(lib().spws_get_timings(self._p, ms, len(TIMING_GROUPS)), "spws_get_timings")
+        return {name: float(ms[g]) for g, name in enumerate(TIMING_GROUPS)}
 
     def execute_host(self, A: TensorArrays, B: TensorArrays, C: TensorArrays, arena_ptr: int, arena_bytes: int):
         """A, B, C hold numpy (ideally pinned) host arrays; returns (status, sizes, arena_needed)."""

@@ -41,6 +41,8 @@ struct DevCtl {
     int work_counter[16];   // dynamic work distribution; cleared before each pass
     int global_slots;       // slots the global-memory ISM actually used
     int pad[7];
+    i64 class_products[NCLASS];
+    i64 class_nnz[NCLASS];
 };
 
 struct ClassParams {
@@ -140,12 +142,14 @@ struct LaunchCtx {
     char* global_arena;      // scratch for CLS_ISM_GLOBAL all arrays
     size_t global_arena_bytes;
     int global_cap;          // accumulation-array capacity of CLS_ISM_GLOBAL
+    mutable int launches;    // kernels enqueued through this context
 };
 
 // setup.cu
 cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA, i64 nnzB);
 cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA);
 cudaError_t launch_bin_rows(const LaunchCtx& c, int m);
+cudaError_t launch_class_nnz(const LaunchCtx& c, int m);
 cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out);
 cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
                                const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,

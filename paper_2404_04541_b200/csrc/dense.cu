@@ -141,6 +141,7 @@ static cudaError_t launch_t(const LaunchCtx& c, bool numeric, int n_units_host, 
         if (n_units_host >= 0 && n_units_host < grid) grid = n_units_host > 0 ? n_units_host : 1;
         k<<<(int)grid, DENSE_THREADS, smem, c.stream>>>(c.ctl, slot, W, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
     }
+    ++c.launches;
     return cudaGetLastError();
 }
 

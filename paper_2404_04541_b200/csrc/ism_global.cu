@@ -257,6 +257,7 @@ static cudaError_t launch_t(const LaunchCtx& c, bool numeric, int n_host, const 
         k<<<(int)grid, GL_THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, slot, c.global_cap, c.global_arena, c.global_arena_bytes,
                                                     A, B, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     }
+    ++c.launches;
     return cudaGetLastError();
 }
 

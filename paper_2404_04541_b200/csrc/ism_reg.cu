@@ -128,6 +128,7 @@ static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int n_host, const 
     else
         ism_reg_kernel<T, G, false><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, A, B,
                                                                   c.tab.jmin, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
+    ++c.launches;
     return cudaGetLastError();
 }
 

@@ -151,6 +151,7 @@ static cudaError_t launch_cap(const LaunchCtx& c, bool numeric, int cls, int n_h
         if (n_host >= 0 && n_host < grid) grid = n_host > 0 ? n_host : 1;
         k<<<(int)grid, THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, cls, slot, A, B, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     }
+    ++c.launches;
     return cudaGetLastError();
 }
 

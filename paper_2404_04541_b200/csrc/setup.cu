@@ -31,6 +31,7 @@ cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 
     const int grid = c.sm_count * 8;
     validate_csr_kernel<<<grid, 256, 0, c.stream>>>(A, nnzA, B.nrows, c.ctl);
     validate_csr_kernel<<<grid, 256, 0, c.stream>>>(B, nnzB, B.ncols, c.ctl);
+    c.launches += 2;
     return cudaGetLastError();
 }
 
@@ -68,8 +69,9 @@ __device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const Cl
 template <int G>
 __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl) {
     __shared__ int s_hist[NCLASS];
+    __shared__ i64 s_cprod[NCLASS];
     __shared__ i64 s_products, s_max_ub, s_max_ub_global;
-    if (threadIdx.x < NCLASS) s_hist[threadIdx.x] = 0;
+    if (threadIdx.x < NCLASS) { s_hist[threadIdx.x] = 0; s_cprod[threadIdx.x] = 0; }
     if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; }
     __syncthreads();
     const int gl = threadIdx.x % G;
@@ -112,6 +114,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             tab.cnt[row] = 0;
             tab.cls[row] = (unsigned char)cls;
             atomicAdd(&s_hist[cls], 1);
+            if (u) atomicAdd((u64*)&s_cprod[cls], (u64)u);
             my_products += u;
             my_max = max(my_max, u);
             if (cls == CLS_ISM_GLOBAL) my_max_global = max(my_max_global, u);
@@ -121,7 +124,10 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
     if (gl == 0 && my_max) atomicMax(&s_max_ub, my_max);
     if (gl == 0 && my_max_global) atomicMax(&s_max_ub_global, my_max_global);
     __syncthreads();
-    if (threadIdx.x < NCLASS && s_hist[threadIdx.x]) atomicAdd(&ctl->class_count[threadIdx.x], s_hist[threadIdx.x]);
+    if (threadIdx.x < NCLASS && s_hist[threadIdx.x]) {
+        atomicAdd(&ctl->class_count[threadIdx.x], s_hist[threadIdx.x]);
+        if (s_cprod[threadIdx.x]) atomicAdd((u64*)&ctl->class_products[threadIdx.x], (u64)s_cprod[threadIdx.x]);
+    }
     if (threadIdx.x == 0) {
         if (s_products) atomicAdd((u64*)&ctl->products, (u64)s_products);
         if (s_max_ub) atomicMax(&ctl->max_ub, s_max_ub);
@@ -141,6 +147,7 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
     if (avg <= 6.0) row_bounds_kernel<4><<<grid_for(4), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
     else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
     else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
+    ++c.launches;
     return cudaGetLastError();
 }
 
@@ -198,6 +205,29 @@ cudaError_t launch_bin_rows(const LaunchCtx& c, int m) {
     i64 want = ((i64)m + 1023) / 1024;
     i64 cap = (i64)c.sm_count * 8;
     bin_rows_kernel<<<(int)(want < cap ? want : cap), 256, 0, c.stream>>>(m, c.tab, c.prm, c.ctl);
+    ++c.launches;
+    return cudaGetLastError();
+}
+
+// Output entries per class (statistics for the per-kernel byte counts).
+__global__ void __launch_bounds__(256) class_nnz_kernel(int m, RowTables tab, DevCtl* ctl) {
+    __shared__ i64 s_nnz[NCLASS];
+    if (threadIdx.x < NCLASS) s_nnz[threadIdx.x] = 0;
+    __syncthreads();
+    for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < m; r += (i64)gridDim.x * blockDim.x) {
+        const int c = tab.cnt[r];
+        if (c) atomicAdd((u64*)&s_nnz[tab.cls[r]], (u64)c);
+    }
+    __syncthreads();
+    if (threadIdx.x < NCLASS && s_nnz[threadIdx.x]) atomicAdd((u64*)&ctl->class_nnz[threadIdx.x], (u64)s_nnz[threadIdx.x]);
+}
+
+cudaError_t launch_class_nnz(const LaunchCtx& c, int m) {
+    if (m == 0) return cudaSuccess;
+    i64 want = ((i64)m + 255) / 256;
+    i64 cap = (i64)c.sm_count * 8;
+    class_nnz_kernel<<<(int)(want < cap ? want : cap), 256, 0, c.stream>>>(m, c.tab, c.ctl);
+    ++c.launches;
     return cudaGetLastError();
 }
 
@@ -290,6 +320,7 @@ cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* o
     if (nblocks > 0) scan_reduce_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums);
     scan_block_sums_kernel<<<1, 1024, 0, c.stream>>>(block_sums, nblocks, out + n, total_out);
     if (nblocks > 0) scan_apply_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums, out);
+    c.launches += nblocks > 0 ? 3 : 1;
     return cudaGetLastError();
 }
 
@@ -350,6 +381,7 @@ cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64*
     e = launch_scan_counts(c, sflags, n_i, spos, block_sums, nullptr);
     if (e != cudaSuccess) return e;
     ttm_slice_compact_kernel<<<grid, 256, 0, c.stream>>>(n_i, n_ij, sflags, spos, Apos1, fpos, Acrd0, Ccrd0, Cpos1, Cpos0, c.ctl);
+    c.launches += 2 + (n_ij > 0) + (n_i > 0);
     return cudaGetLastError();
 }
 

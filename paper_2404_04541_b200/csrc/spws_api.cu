@@ -30,6 +30,12 @@ struct spws_plan_s {
     // what the last symbolic pass saw (numeric must be called with the same shapes and scratch)
     int64_t m = 0;
     void* scratch = nullptr;
+    // optional per-kernel timing: ev[g] is recorded after group g; ev_start[] before each pass
+    bool profiling = false;
+    cudaEvent_t ev[SPWS_T_COUNT] = {};
+    cudaEvent_t ev_start[2] = {};
+    bool ev_ran[SPWS_T_COUNT] = {};
+    bool ev_pass[2] = {};
 };
 
 namespace {
@@ -243,6 +249,19 @@ spws_status_t from_dev_status(int s) {
 
 #define CUDA_TRY(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return SPWS_CUDA_ERROR; } } while (0)
 
+inline void mark(spws_plan_s* p, int group) {
+    if (!p->profiling) return;
+    cudaEventRecord(p->ev[group], p->h->stream);
+    p->ev_ran[group] = true;
+}
+inline void mark_start(spws_plan_s* p, int pass) {
+    if (!p->profiling) return;
+    const int g0 = pass == 0 ? 0 : SPWS_T_NUM_ISM_REG, g1 = pass == 0 ? SPWS_T_NUM_ISM_REG : SPWS_T_COUNT;
+    for (int g = g0; g < g1; ++g) p->ev_ran[g] = false;
+    cudaEventRecord(p->ev_start[pass], p->h->stream);
+    p->ev_pass[pass] = true;
+}
+
 }  // namespace
 
 extern "C" {
@@ -326,8 +345,40 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
     return SPWS_OK;
 }
 
+spws_status_t spws_set_profiling(spws_plan_t plan, int enabled) {
+    if (!plan) return SPWS_INVALID_ARGUMENT;
+    if (enabled && !plan->ev[0]) {
+        for (int g = 0; g < SPWS_T_COUNT; ++g) CUDA_TRY(cudaEventCreate(&plan->ev[g]));
+        for (int g = 0; g < 2; ++g) CUDA_TRY(cudaEventCreate(&plan->ev_start[g]));
+    }
+    plan->profiling = enabled != 0;
+    return SPWS_OK;
+}
+
+spws_status_t spws_get_timings(spws_plan_t plan, float* ms, int n) {
+    if (!plan || !ms || n < SPWS_T_COUNT) return SPWS_INVALID_ARGUMENT;
+    for (int g = 0; g < SPWS_T_COUNT; ++g) ms[g] = 0.0f;
+    if (!plan->ev[0]) return SPWS_BAD_SEQUENCE;
+    CUDA_TRY(cudaStreamSynchronize(plan->h->stream));
+    for (int pass = 0; pass < 2; ++pass) {
+        if (!plan->ev_pass[pass]) continue;
+        cudaEvent_t prev = plan->ev_start[pass];
+        const int g0 = pass == 0 ? 0 : SPWS_T_NUM_ISM_REG, g1 = pass == 0 ? SPWS_T_NUM_ISM_REG : SPWS_T_COUNT;
+        for (int g = g0; g < g1; ++g) {
+            if (!plan->ev_ran[g]) continue;
+            CUDA_TRY(cudaEventElapsedTime(&ms[g], prev, plan->ev[g]));
+            prev = plan->ev[g];
+        }
+    }
+    return SPWS_OK;
+}
+
 spws_status_t spws_plan_destroy(spws_plan_t plan) {
     if (!plan) return SPWS_INVALID_ARGUMENT;
+    if (plan->ev[0]) {
+        for (int g = 0; g < SPWS_T_COUNT; ++g) cudaEventDestroy(plan->ev[g]);
+        for (int g = 0; g < 2; ++g) cudaEventDestroy(plan->ev_start[g]);
+    }
     if (plan->host_ctl) cudaFreeHost(plan->host_ctl);
     delete plan;
     return SPWS_OK;
@@ -366,17 +417,30 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
         if (plan->host_ctl->status != 0) return from_dev_status(plan->host_ctl->status);
     }
     // a1: upper bounds + classes; a2: binning
+    mark_start(plan, 0);
     CUDA_TRY(launch_row_bounds(c, S.A, S.B, S.nnzA));
+    mark(plan, SPWS_T_SYM_BOUNDS);
     CUDA_TRY(launch_bin_rows(c, (int)S.m));
+    mark(plan, SPWS_T_SYM_BIN);
     // a3: exact count per row through the workspace of its class
     i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<i64*>(sc + L.rowptr_raw);
     if (S.m > 0) {
-        CUDA_TRY(launch_ism_reg(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
-        CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
-        CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, -1, S.A, S.B, rowptr, nullptr, nullptr));
-        CUDA_TRY(launch_dense(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
-        if (plan->policy != SPWS_DENSE)
+        if (plan->policy != SPWS_DENSE) {
+            CUDA_TRY(launch_ism_reg(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            mark(plan, SPWS_T_SYM_ISM_REG);
+            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            mark(plan, SPWS_T_SYM_ISM_SMEM_S);
+            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            mark(plan, SPWS_T_SYM_ISM_SMEM);
+        }
+        if (plan->policy != SPWS_SPARSE_ISM) {
+            CUDA_TRY(launch_dense(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            mark(plan, SPWS_T_SYM_DENSE);
+        }
+        if (plan->policy != SPWS_DENSE) {
             CUDA_TRY(launch_ism_global(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            mark(plan, SPWS_T_SYM_ISM_GLOBAL);
+        }
     }
     // a4: exclusive scan into the row pointer
     CUDA_TRY(launch_scan_counts(c, c.tab.cnt, (int)S.m, rowptr, reinterpret_cast<i64*>(sc + L.block_sums), &c.ctl->nnz));
@@ -386,6 +450,8 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
                                     reinterpret_cast<int*>(sc + L.sflags), reinterpret_cast<i64*>(sc + L.spos),
                                     reinterpret_cast<i64*>(sc + L.block_sums), LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
     }
+    CUDA_TRY(launch_class_nnz(c, (int)S.m));
+    mark(plan, SPWS_T_SYM_SCAN);
     CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
     CUDA_TRY(cudaStreamSynchronize(stream));
     const DevCtl& hc = *plan->host_ctl;
@@ -396,8 +462,13 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     plan->stats.products = hc.products;
     plan->stats.nnz = hc.nnz;
     plan->stats.max_row_products = hc.max_ub;
-    for (int k = 0; k < NCLASS; ++k) plan->stats.rows_per_class[k] = hc.class_count[k];
+    for (int k = 0; k < NCLASS; ++k) {
+        plan->stats.rows_per_class[k] = hc.class_count[k];
+        plan->stats.products_per_class[k] = hc.class_products[k];
+        plan->stats.nnz_per_class[k] = hc.class_nnz[k];
+    }
     plan->stats.dense_units = hc.n_units;
+    plan->stats.launches_symbolic = c.launches;
     if (plan->kind == 0) {
         C->n[0] = C->dims[0];
         C->n[1] = hc.nnz;
@@ -432,18 +503,30 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
     const i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<const i64*>(sc + L.rowptr_raw);
     CUDA_TRY(cudaMemsetAsync(c.ctl->work_counter, 0, sizeof(c.ctl->work_counter), c.stream));
+    mark_start(plan, 1);
     const spws_stats_t& s = plan->stats;
     int* crd = C->crd[last];
-    if (s.rows_per_class[CLS_ISM_REG] > 0)
+    if (s.rows_per_class[CLS_ISM_REG] > 0) {
         CUDA_TRY(launch_ism_reg(c, true, (int)s.rows_per_class[CLS_ISM_REG], S.A, S.B, rowptr, crd, C->val));
-    if (s.rows_per_class[CLS_ISM_SMEM_S] > 0)
+        mark(plan, SPWS_T_NUM_ISM_REG);
+    }
+    if (s.rows_per_class[CLS_ISM_SMEM_S] > 0) {
         CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM_S, (int)s.rows_per_class[CLS_ISM_SMEM_S], S.A, S.B, rowptr, crd, C->val));
-    if (s.rows_per_class[CLS_ISM_SMEM] > 0)
+        mark(plan, SPWS_T_NUM_ISM_SMEM_S);
+    }
+    if (s.rows_per_class[CLS_ISM_SMEM] > 0) {
         CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM, (int)s.rows_per_class[CLS_ISM_SMEM], S.A, S.B, rowptr, crd, C->val));
-    if (s.dense_units > 0)
+        mark(plan, SPWS_T_NUM_ISM_SMEM);
+    }
+    if (s.dense_units > 0) {
         CUDA_TRY(launch_dense(c, true, (int)s.dense_units, S.A, S.B, rowptr, crd, C->val));
-    if (s.rows_per_class[CLS_ISM_GLOBAL] > 0)
+        mark(plan, SPWS_T_NUM_DENSE);
+    }
+    if (s.rows_per_class[CLS_ISM_GLOBAL] > 0) {
         CUDA_TRY(launch_ism_global(c, true, (int)s.rows_per_class[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));
+        mark(plan, SPWS_T_NUM_ISM_GLOBAL);
+    }
+    plan->stats.launches_numeric = c.launches;
     return SPWS_OK;
 }
 
