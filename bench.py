@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse-workspace SpGEMM path on B200.
+
+One step = one whole pass of the hot path (symbolic + numeric, policy auto) over one synthetic
+operand set already resident in HBM.  Default workload: the power-law configuration (R-MAT,
+2^18 vertices, average degree 16, C = A*A, fp64).  Prints ONE JSON line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+N > 1 (under torchrun): every rank runs its own seeded problem of the same shape (output rows
+are independent, so ranks share nothing on the data path); value = all ranks' flops over the
+slowest rank's device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC, UNIT = "spgemm_gflops_2_per_product", "GFLOP/s"
+WORKLOAD_TEXT = {
+    "rmat18": "power-law SpGEMM C=A*A, R-MAT 2^18 vertices, degree 16, (0.57,0.19,0.19,0.05), fp64",
+    "stencil64": "FEM-like SpGEMM C=A*A, 27-point stencil on 64^3, fp64",
+    "uniform8": "SpGEMM C=A*A, 2048x2048, 8 nnz/row, fp64",
+    "wide26": "wide-output SpGEMM, A 65536 x 2^26, B 2^26 x 2^26, 4 nnz/row, fp32",
+}
+NOMINAL_HBM_GBS = 8000.0
+
+
+def algorithmic_bytes(m, nnzA, products, nnzC, V):
+    """Bytes the method itself must move, counted once: A read, gathered B rows (two offsets per
+    A entry + index and value per product), C written."""
+    return ((m + 1) * 8 + nnzA * (4 + V)) + (nnzA * 16 + products * (4 + V)) + ((m + 1) * 8 + nnzC * (4 + V))
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample(A, B, budget_products: float, seed: int = 0):
+    """Rows of the workload drawn at random until their products reach the budget."""
+    rng = np.random.default_rng(seed)
+    lens = np.diff(B.pos)
+    rows_of_nz = np.repeat(np.arange(A.nrows), np.diff(A.pos))
+    ub = np.bincount(rows_of_nz, weights=lens[A.crd], minlength=A.nrows).astype(np.int64)
+    order = rng.permutation(A.nrows)
+    csum = np.cumsum(ub[order])
+    n = int(np.searchsorted(csum, budget_products) + 1)
+    n = max(1, min(n, A.nrows))
+    rows = np.sort(order[:n])
+    return rows, int(ub[rows].sum()), int(ub.sum())
+
+
+def time_oracle(A, B, rows, threads):
+    import oracle
+    t0 = time.perf_counter()
+    res = oracle.spgemm(A, B, rows=rows, threads=threads)
+    dt = time.perf_counter() - t0
+    return dt, int(res.products.sum())
+
+
+def sized_oracle_sample(A, B, threads, seconds):
+    """Calibrate on a small sample, then size a sample for about `seconds` of CPU work."""
+    rows0, p0, total = oracle_sample(A, B, 2e7)
+    dt0, _ = time_oracle(A, B, rows0, threads)
+    budget = min(total, max(2e7, p0 / max(dt0, 1e-6) * seconds))
+    rows, psample, _ = oracle_sample(A, B, budget)
+    return rows, psample, total
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores, on a bounded sample."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    from workloads import config_inputs
+    oracle.build()
+    cfg = config_inputs(args.workload, seed=args.seed)
+    A, B = cfg["A"], cfg["B"]
+    threads = oracle.hardware_threads()
+    rows, psample, total = sized_oracle_sample(A, B, threads, 6.0)
+    for _ in range(args.warmup):
+        time_oracle(A, B, rows, threads)
+    times = [time_oracle(A, B, rows, threads)[0] for _ in range(args.steps)]
+    ms = 1e3 * float(np.mean(times))
+    value = 2.0 * psample / (ms * 1e-3) / 1e9
+    sample = f"{rows.size} random rows of {A.nrows}, {psample} of {total} products per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "seed": args.seed,
+                       "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="rmat18", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--policy", default="auto")
+    ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2404_04541_b200 import api, binding
+    from workloads import config_inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = config_inputs(args.workload, seed=args.seed + rank)
+    A, B = cfg["A"], cfg["B"]
+    V = 8 if cfg["dtype"] == np.float64 else 4
+    vt = torch.float64 if V == 8 else torch.float32
+    ctx = api.Context(dev)
+    dA = api.DeviceCSR.from_host(A, device=dev)
+    dB = dA if B is A else api.DeviceCSR.from_host(B, device=dev)
+    plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, cfg["dtype"], args.policy)
+    plan.set_profiling(True)
+
+    # a first pass sizes C; its buffers are reused by every step (allocation is outside the timed region)
+    c, state = ctx.spgemm_symbolic(plan, dA, dB)
+    nnzC = c.n[1]
+    crd = torch.empty(nnzC, dtype=torch.int32, device=dev)
+    val = torch.empty(nnzC, dtype=vt, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)       # > L2 (126 MB)
+
+    def step():
+        cc, st = ctx.spgemm_symbolic(plan, dA, dB)
+        ctx.spgemm_numeric(plan, cc, st, crd=crd, val=val)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    stats = plan.get_stats()
+    products = stats["products"]
+
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    group_ms = {g: 0.0 for g in binding.TIMING_GROUPS}
+    for s in range(args.steps):
+        flush.fill_(s & 0xff)                                            # L2 flush between timed steps
+        ev[s][0].record()
+        step()
+        ev[s][1].record()
+        for g, ms in plan.get_timings().items():                         # synchronises the stream
+            group_ms[g] += ms
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    t = torch.tensor([total_ms, float(products), float(nnzC), float(A.nnz), float(A.nrows)], dtype=torch.float64, device=dev)
+    if world > 1:
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        total_ms = float(tmax[0])
+    all_products, all_nnzC, all_nnzA, all_m = float(t[1]), float(t[2]), float(t[3]), float(t[4])
+    ms_per_step = total_ms / args.steps
+    value = 2.0 * all_products / (ms_per_step * 1e-3) / 1e9
+    abytes = algorithmic_bytes(all_m, all_nnzA, all_products, all_nnzC, V)
+    eff_gbs = abytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (this rank's launches)
+    peak, peak_kind = measured_peak()
+    avg = {g: v / args.steps for g, v in group_ms.items()}
+    top = max(avg, key=avg.get)
+    cls_of = {"ism_reg": 1, "ism_smem_s": 2, "ism_smem": 3, "dense": 4, "ism_global": 5}
+    kname = top.split("_", 1)[1]
+    kbytes = 0
+    if kname in cls_of:
+        pc, nc = stats["products_per_class"][cls_of[kname]], stats["nnz_per_class"][cls_of[kname]]
+        # numeric: index + value per product gathered, index + value per output written;
+        # symbolic: index per product gathered
+        kbytes = pc * (4 + V) + nc * (4 + V) if top.startswith("num_") else pc * 4
+    achieved = kbytes / (avg[top] * 1e-3) / 1e9 if avg[top] > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "kernel_ms": avg[top], "algorithmic_bytes": kbytes}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64" if V == 8 else "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "policy": args.policy,
+                       "seed": args.seed, "rows": int(A.nrows), "nnzA": int(A.nnz), "products": int(products),
+                       "nnzC": int(nnzC), "l2": "512 MiB buffer written between timed steps",
+                       "timed": "spws_symbolic + spws_numeric; C buffers preallocated"},
+            "effective_gbs": eff_gbs, "algorithmic_bytes_per_step": abytes,
+            "hbm_frac_nominal_8tbs": eff_gbs / NOMINAL_HBM_GBS, "hbm_frac_measured": eff_gbs / peak,
+            "roofline": roofline, "kernel_ms": avg, "rows_per_class": stats["rows_per_class"],
+            "products_per_class": stats["products_per_class"], "nnz_per_class": stats["nnz_per_class"],
+            "dense_units": stats["dense_units"],
+            "gpu_launches": (stats["launches_symbolic"] + stats["launches_numeric"]) * args.steps,
+            "clocks": clocks}
+
+    # ---- end to end through the host-buffer entry point (H2D of A, D2H of C inside the timed region)
+    if not args.no_e2e and B is A:
+        try:
+            pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+            hp, hc, hv = pin(A.pos), pin(A.crd), pin(A.val)
+            cpos = torch.empty(A.nrows + 1, dtype=torch.int64).pin_memory()
+            ccrd = torch.empty(nnzC, dtype=torch.int32).pin_memory()
+            cval = torch.empty(nnzC, dtype=vt).pin_memory()
+            a = binding.csr_arrays(A.nrows, A.ncols, hp.numpy(), hc.numpy(), hv.numpy())
+            cc = binding.csr_arrays(A.nrows, A.ncols, cpos.numpy(), ccrd.numpy(), cval.numpy())
+            in_bytes = hp.numel() * 8 + hc.numel() * 4 + hv.numel() * V
+            ws = plan.workspace_size(dA.arrays(), dA.arrays())
+            arena_bytes = in_bytes + (A.nrows + 1) * 8 + ws + nnzC * (4 + V) + (1 << 20)
+            arena = torch.empty(arena_bytes + 256, dtype=torch.uint8, device=dev)
+            aptr = ctx._aligned_ptr(arena)
+            plan.set_profiling(False)
+            for _ in range(2):
+                st, sizes, need = plan.execute_host(a, a, cc, aptr, arena_bytes)
+                if st != 0:
+                    raise RuntimeError(f"execute_host: {binding.status_string(st)} (needs {need} bytes)")
+            n_e2e = max(1, min(args.steps, 3))
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n_e2e):
+                st, sizes, need = plan.execute_host(a, a, cc, aptr, arena_bytes)
+            e1.record()
+            torch.cuda.synchronize()
+            e2e_ms = torch.tensor([e0.elapsed_time(e1) / n_e2e], dtype=torch.float64, device=dev)
+            if world > 1:
+                dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+            out_bytes = (A.nrows + 1) * 8 + nnzC * (4 + V)
+            line["e2e"] = {"value": 2.0 * all_products / (float(e2e_ms[0]) * 1e-3) / 1e9, "unit": UNIT,
+                           "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
+                           "ms_per_step": float(e2e_ms[0]), "steps": n_e2e,
+                           "call": "spws_execute_host, pinned host buffers"}
+        except Exception as exc:  # report, do not hide
+            line["e2e"] = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
+
+    # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        threads = oracle.hardware_threads()
+        rows, psample, total = sized_oracle_sample(A, B, threads, 12.0)
+        dt, _ = time_oracle(A, B, rows, threads)
+        line["cpu_baseline"] = {"value": 2.0 * psample / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{rows.size} random rows of {A.nrows}, {psample} of {total} products, {dt:.1f} s"}
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
