@@ -197,6 +197,32 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
                                 spws_tensor_t* C, void* arena, size_t arena_bytes,
                                 size_t* arena_needed);
 
+/* Row pointer from per-row counts, without any scratch argument (the paper has no counterpart:
+ * this entry exists for the sake of callers, not of the method).
+ *
+ * Some code that wants the symbolic pass's last step -- pos[0] = 0, pos[i+1] = pos[i] + counts[i]
+ * -- is not in a position to obtain device memory: a plug-in running inside a host whose
+ * allocator already owns the whole GPU, a component that must not trigger the device-wide
+ * synchronisation cudaMalloc / cudaFree imply, or a context (a host callback, a start-up path
+ * before any pool exists) where allocation calls are simply off limits.  spws_symbolic needs a
+ * caller-supplied scratch buffer for its scan; this variant keeps the scan's partial sums in a
+ * fixed 64 KiB array that is part of the library image and therefore sits on every GPU that
+ * loads the library until the process exits.  It calls no allocation routine of any kind.
+ *
+ * counts : DEVICE, int32, n entries (row i's number of stored outputs).
+ * pos    : DEVICE, int64, n+1 entries, written by the call; pos[n] is the total.
+ * n      : 0 <= n <= SPWS_STATIC_MAX_ROWS; a larger n is refused with SPWS_SCRATCH_TOO_SMALL and
+ *          nothing is launched.
+ * Work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default stream); the call does not
+ * synchronise.  The first call on each device looks up the array's address on that device
+ * (with that device current) and caches it, so make that first call outside any stream capture.
+ * All calls on one GPU share the one array: two calls whose kernels can overlap on that GPU
+ * (different streams, no ordering between them) race on it; order them.  The array keeps
+ * whatever the last call left there, which is harmless because each call writes every partial
+ * sum before reading it. */
+#define SPWS_STATIC_MAX_ROWS 16777216
+spws_status_t spws_row_pointer_static(const int32_t* counts, int64_t n, int64_t* pos, void* cuda_stream);
+
 const char* spws_status_string(spws_status_t status);
 
 #ifdef __cplusplus

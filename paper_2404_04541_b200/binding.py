@@ -34,7 +34,8 @@ POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPAR
 EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create", "spws_plan_destroy",
            "spws_check_expression", "spws_workspace_size", "spws_symbolic", "spws_numeric",
            "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host",
-           "spws_status_string")
+           "spws_row_pointer_static", "spws_status_string")
+STATIC_MAX_ROWS = 16777216
 TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense",
                  "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem", "num_dense",
                  "num_ism_global")
@@ -93,6 +94,7 @@ def lib():
         L.spws_set_profiling.argtypes = [vp, i32]
         L.spws_get_timings.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
         L.spws_execute_host.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(sz)]
+        L.spws_row_pointer_static.argtypes = [vp, ctypes.c_int64, vp, vp]
         L.spws_status_string.argtypes = [i32]
         L.spws_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -116,6 +118,13 @@ def check_expression(expr: str, fmts) -> int:
     arr = (ctypes.c_int * 3)(*fmts)
     kind = ctypes.c_int(-1)
     return lib().spws_check_expression(expr.encode(), arr, ctypes.byref(kind))
+
+
+def row_pointer_static(counts_ptr: int, n: int, pos_ptr: int, stream_ptr: int | None = None) -> int:
+    """spws_row_pointer_static: device pointers in, status out (does not raise).  The scan's
+    scratch is a fixed array inside the library, so this call allocates nothing."""
+    return lib().spws_row_pointer_static(ctypes.c_void_p(counts_ptr), int(n), ctypes.c_void_p(pos_ptr),
+                                         ctypes.c_void_p(stream_ptr))
 
 
 # ---------------------------------------------------------------------------- tensors

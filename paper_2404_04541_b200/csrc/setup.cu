@@ -386,3 +386,64 @@ cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64*
 }
 
 }  // namespace spws
+
+// ---------------------------------------------------------------------------------------
+// spws_row_pointer_static: the exclusive scan of the symbolic pass for callers that cannot
+// allocate device memory.  The scan's block sums -- the one piece of scratch it needs -- live
+// in a fixed array inside the library image instead of a caller-supplied buffer.
+// ---------------------------------------------------------------------------------------
+#include <mutex>
+
+#include "../../include/spws.h"
+
+namespace {
+
+constexpr long long STATIC_BLOCK_SUMS = SPWS_STATIC_MAX_ROWS / spws::SCAN_TILE;   // 8192 partial sums
+static_assert(SPWS_STATIC_MAX_ROWS % spws::SCAN_TILE == 0, "row limit must be a whole number of scan tiles");
+
+// 64 KiB resident on every GPU that loads the library, until the process exits.
+static __device__ __align__(256) long long g_static_block_sums[STATIC_BLOCK_SUMS + 2];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+void* g_static_addr[MAX_DEVICES] = {};
+
+// The array's name is only a host-side handle; kernels need its device address, which differs
+// per GPU and is looked up once per device with that device current.
+spws_status_t static_scratch_address(spws::i64** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+        cudaGetLastError();
+        return SPWS_CUDA_ERROR;
+    }
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_block_sums) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return SPWS_CUDA_ERROR;
+        }
+        g_static_addr[dev] = p;
+    }
+    *out = static_cast<spws::i64*>(g_static_addr[dev]);
+    return SPWS_OK;
+}
+
+}  // namespace
+
+extern "C" spws_status_t spws_row_pointer_static(const int32_t* counts, int64_t n, int64_t* pos, void* cuda_stream) {
+    if (n < 0 || !pos || (n > 0 && !counts)) return SPWS_INVALID_ARGUMENT;
+    if (n > SPWS_STATIC_MAX_ROWS) return SPWS_SCRATCH_TOO_SMALL;
+    spws::i64* block_sums = nullptr;
+    const spws_status_t st = static_scratch_address(&block_sums);
+    if (st != SPWS_OK) return st;
+    spws::LaunchCtx c{};
+    c.stream = static_cast<cudaStream_t>(cuda_stream);
+    // Every partial sum the scan reads is written earlier in the same call, so nothing left
+    // behind by a previous call has to be cleared.
+    if (spws::launch_scan_counts(c, counts, (int)n, reinterpret_cast<spws::i64*>(pos), block_sums, nullptr) != cudaSuccess) {
+        cudaGetLastError();
+        return SPWS_CUDA_ERROR;
+    }
+    return SPWS_OK;
+}
