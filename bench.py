@@ -169,13 +169,15 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="rmat18", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--workload", default="rmat18",
+                    help="rmat18 (default), stencil64, uniform8, wide26, or rmatNN / stencilNN at another size")
     ap.add_argument("--policy", default="auto")
     ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    WORKLOAD_TEXT.setdefault(args.workload, f"{args.workload} (same recipe as the named configuration, other size), fp64")
     if args.impl == "reference":
         run_reference(args)
         return

@@ -167,4 +167,11 @@ def config_inputs(name: str, seed: int = 1, reduced: bool = False) -> dict:
         A = uniform_csf3((d, d, d), nnz, seed)
         B = uniform_rows_csr(d, d, 8, seed + 1000)
         return dict(kind="ttm", A=A, B=B, dtype=np.float64, name=name)
+    # same recipes at other sizes (profiling captures need a smaller case): "rmat16", "stencil40"
+    if name.startswith("rmat") and name[4:].isdigit():
+        A = rmat_csr(int(name[4:]), 16, seed)
+        return dict(kind="spgemm", A=A, B=A, dtype=np.float64, name=name)
+    if name.startswith("stencil") and name[7:].isdigit():
+        A = stencil27_csr(int(name[7:]), seed)
+        return dict(kind="spgemm", A=A, B=A, dtype=np.float64, name=name)
     raise ValueError(f"unknown config {name!r}; choose from {CONFIG_NAMES}")
