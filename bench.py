@@ -259,14 +259,25 @@ def main():
     peak, peak_kind = measured_peak()
     avg = {g: v / args.steps for g, v in group_ms.items()}
     top = max(avg, key=avg.get)
-    cls_of = {"ism_reg": 1, "ism_smem_s": 2, "ism_smem": 3, "dense": 4, "ism_global": 5}
+    # algorithmic bytes of each per-class kernel group: numeric = index + value per product
+    # gathered and per output written; symbolic = index per product gathered
+    pc, nc = stats["products_per_class"], stats["nnz_per_class"]
+    dw_p, dw_n = stats["dense_warp_products"], stats["dense_warp_nnz"]
+    dense_p, dense_n = sum(pc[4:7]), sum(nc[4:7])
+    group_units = {"ism_reg": (pc[1], nc[1]), "ism_smem_s": (pc[2], nc[2]), "ism_smem": (pc[3], nc[3]),
+                   "ism_global": (pc[7], nc[7])}
     kname = top.split("_", 1)[1]
-    kbytes = 0
-    if kname in cls_of:
-        pc, nc = stats["products_per_class"][cls_of[kname]], stats["nnz_per_class"][cls_of[kname]]
-        # numeric: index + value per product gathered, index + value per output written;
-        # symbolic: index per product gathered
-        kbytes = pc * (4 + V) + nc * (4 + V) if top.startswith("num_") else pc * 4
+    if top == "num_dense_warp":
+        gp, gn = dw_p, dw_n
+    elif top == "num_dense_cta":
+        gp, gn = dense_p - dw_p, dense_n - dw_n
+    elif top == "sym_dense_warp":
+        gp, gn = pc[4], nc[4]
+    elif top == "sym_dense_cta":
+        gp, gn = pc[5] + pc[6], nc[5] + nc[6]
+    else:
+        gp, gn = group_units.get(kname, (0, 0))
+    kbytes = gp * (4 + V) + gn * (4 + V) if top.startswith("num_") else gp * 4
     achieved = kbytes / (avg[top] * 1e-3) / 1e9 if avg[top] > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
@@ -283,7 +294,8 @@ def main():
             "hbm_frac_nominal_8tbs": eff_gbs / NOMINAL_HBM_GBS, "hbm_frac_measured": eff_gbs / peak,
             "roofline": roofline, "kernel_ms": avg, "rows_per_class": stats["rows_per_class"],
             "products_per_class": stats["products_per_class"], "nnz_per_class": stats["nnz_per_class"],
-            "dense_units": stats["dense_units"],
+            "dense_units": stats["dense_units"], "dense_warp_rows": stats["dense_warp_rows"],
+            "bitmap_bytes": stats["bitmap_bytes"],
             "gpu_launches": (stats["launches_symbolic"] + stats["launches_numeric"]) * args.steps,
             "clocks": clocks}
 

@@ -47,7 +47,7 @@ enum {
     SPWS_DIM_MISMATCH = 3,           /* contracted dimension or output dimensions disagree          */
     SPWS_NONCANONICAL_INPUT = 4,     /* unsorted / duplicate / out-of-range coordinate, bad pos     */
     SPWS_SCRATCH_TOO_SMALL = 5,      /* scratch (or arena) smaller than this call needs             */
-    SPWS_WORKSPACE_TOO_LARGE = 6,    /* policy DENSE forced on a row needing > max_dense_tiles tiles*/
+    SPWS_WORKSPACE_TOO_LARGE = 6,    /* policy DENSE forced on a row wider than dense_max_span      */
     SPWS_CUDA_ERROR = 7,             /* a CUDA runtime call failed                                  */
     SPWS_INTERNAL_OVERFLOW = 8,      /* a bounded device loop hit its limit                         */
     SPWS_OUTPUT_TOO_SMALL = 9,       /* C's capacity (n[]) is smaller than the result               */
@@ -61,7 +61,7 @@ typedef struct spws_plan_s* spws_plan_t;
 typedef enum { SPWS_CSR = 0, SPWS_CSF3 = 1 } spws_format_t;
 typedef enum { SPWS_F32 = 0, SPWS_F64 = 1 } spws_dtype_t;
 /* Workspace policy.  DENSE: value array + occupancy bitmap along the last index (Gustavson's
- * workspace, Table 2), column-tiled in shared memory.  SPARSE_ISM: insert-sort-merge with the
+ * workspace, Table 2), held in shared memory.  SPARSE_ISM: insert-sort-merge with the
  * coordinate-sort policy (Algorithm 1, Sec. 5.2).  AUTO: chosen per row bin from the product
  * count and the column span.  The policy changes the route, never the result. */
 typedef enum { SPWS_DENSE = 0, SPWS_SPARSE_ISM = 1, SPWS_AUTO = 2 } spws_policy_t;
@@ -91,12 +91,15 @@ typedef struct {
     int32_t ism_warp_cap;     /* rows with <= this many products use the register ISM (<= 32)    */
     int32_t ism_cta_cap;      /* accumulation-array capacity of the shared-memory ISM, power of
                                  two in [64, 4096]; default 4096                                  */
-    int32_t dense_tile_cols;  /* columns per dense tile, power of two in [256, 16384];
-                                 default 8192 (f64) / 16384 (f32)                                 */
-    int32_t max_dense_tiles;  /* a row may use at most this many tiles; default 64               */
+    int32_t dense_unit_outputs;/* outputs one CTA unit of the dense workspace accumulates (a long
+                                 row is cut into units of this many consecutive outputs), power
+                                 of two in [64, 8192]; default 4096                               */
+    int32_t dense_max_span;   /* widest column span (jmax - jmin + 1) a dense workspace may cover,
+                                 in [32, 2^20]; default 2^20.  Wider rows go to ISM (AUTO) or
+                                 fail with SPWS_WORKSPACE_TOO_LARGE (DENSE)                       */
     int32_t fallback_cap;     /* accumulation-array capacity (the paper's `cap`) of the global-
                                  memory ISM, power of two in [2, 2048]; default 2048              */
-    float dense_span_words_per_product; /* AUTO picks DENSE for a single-tile row when
+    float dense_span_words_per_product; /* AUTO prefers DENSE over the shared-memory ISM when
                                  span/32 <= this * products; default 4                            */
     int32_t reserved[5];
 } spws_options_t;
@@ -106,15 +109,19 @@ typedef struct {
     int64_t products;         /* intermediate products = sum of the per-row upper bounds          */
     int64_t nnz;              /* stored entries of C                                              */
     int64_t max_row_products;
-    int64_t rows_per_class[8];/* empty, ISM-register, ISM-shared(small), ISM-shared, dense,
-                                 ISM-global, reserved, reserved                                   */
-    int64_t dense_units;      /* (row, column tile) work units of the dense route                 */
+    int64_t rows_per_class[8];/* empty, ISM-register, ISM-shared(small), ISM-shared, dense-warp,
+                                 dense-CTA(hub), dense-CTA, ISM-global                            */
+    int64_t dense_units;      /* CTA work units (row, output range) of the dense numeric pass     */
     int32_t device_status;    /* last status word read back from the device                      */
     int32_t reserved;
     int64_t products_per_class[8];
     int64_t nnz_per_class[8];
     int32_t launches_symbolic; /* kernels enqueued by the last spws_symbolic / spws_numeric       */
     int32_t launches_numeric;
+    int64_t dense_warp_rows;  /* dense rows the warp-per-row numeric kernel takes ...             */
+    int64_t dense_warp_products; /* ... and their products and outputs                            */
+    int64_t dense_warp_nnz;
+    int64_t bitmap_bytes;     /* bytes of the bitmap arena in use                                 */
 } spws_stats_t;
 
 /* Kernel groups timed by spws_set_profiling (index into the array spws_get_timings fills). */
@@ -124,15 +131,18 @@ enum {
     SPWS_T_SYM_ISM_REG = 2,
     SPWS_T_SYM_ISM_SMEM_S = 3,
     SPWS_T_SYM_ISM_SMEM = 4,
-    SPWS_T_SYM_DENSE = 5,
-    SPWS_T_SYM_ISM_GLOBAL = 6,
-    SPWS_T_SYM_SCAN = 7,      /* exclusive scan (+ CSF level rebuild for the 3-tensor form)        */
-    SPWS_T_NUM_ISM_REG = 8,
-    SPWS_T_NUM_ISM_SMEM_S = 9,
-    SPWS_T_NUM_ISM_SMEM = 10,
-    SPWS_T_NUM_DENSE = 11,
-    SPWS_T_NUM_ISM_GLOBAL = 12,
-    SPWS_T_COUNT = 13
+    SPWS_T_SYM_DENSE_WARP = 5,
+    SPWS_T_SYM_DENSE_CTA = 6,
+    SPWS_T_SYM_ISM_GLOBAL = 7,
+    SPWS_T_SYM_SCAN = 8,      /* exclusive scan, numeric routing of dense rows (+ CSF level
+                                 rebuild for the 3-tensor form)                                    */
+    SPWS_T_NUM_ISM_REG = 9,
+    SPWS_T_NUM_ISM_SMEM_S = 10,
+    SPWS_T_NUM_ISM_SMEM = 11,
+    SPWS_T_NUM_DENSE_WARP = 12,
+    SPWS_T_NUM_DENSE_CTA = 13,
+    SPWS_T_NUM_ISM_GLOBAL = 14,
+    SPWS_T_COUNT = 15
 };
 
 spws_status_t spws_create(spws_handle_t* handle);
@@ -157,8 +167,11 @@ spws_status_t spws_plan_destroy(spws_plan_t plan);
 spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3], int* kind);
 
 /* Upper bound of the scratch bytes spws_symbolic + spws_numeric need for these operands (reads
- * only dims and n[] of A and B; host-side, launches nothing).  256-byte alignment is required of
- * the scratch pointer. */
+ * only dims and n[] of A and B; host-side, launches nothing).  It always suffices; the largest
+ * part is room for one occupancy bitmap per row (rows x min(columns, dense_max_span) / 8 bytes),
+ * of which only the rows routed to the dense workspace use their exact span, so a smaller buffer
+ * works for narrow rows and spws_symbolic reports SPWS_SCRATCH_TOO_SMALL when it does not.
+ * 256-byte alignment is required of the scratch pointer. */
 spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
                                   size_t* bytes);
 

@@ -36,9 +36,11 @@ EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create",
            "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host",
            "spws_row_pointer_static", "spws_status_string")
 STATIC_MAX_ROWS = 16777216
-TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense",
-                 "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem", "num_dense",
-                 "num_ism_global")
+TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense_warp",
+                 "sym_dense_cta", "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem",
+                 "num_dense_warp", "num_dense_cta", "num_ism_global")
+# class index of each per-class kernel group (rows_per_class / products_per_class / nnz_per_class)
+CLASS_NAMES = ("empty", "ism_reg", "ism_smem_s", "ism_smem", "dense_warp", "dense_hub", "dense_cta", "ism_global")
 
 
 class spws_tensor_t(ctypes.Structure):
@@ -49,7 +51,7 @@ class spws_tensor_t(ctypes.Structure):
 
 class spws_options_t(ctypes.Structure):
     _fields_ = [("validate", ctypes.c_int32), ("ism_warp_cap", ctypes.c_int32), ("ism_cta_cap", ctypes.c_int32),
-                ("dense_tile_cols", ctypes.c_int32), ("max_dense_tiles", ctypes.c_int32),
+                ("dense_unit_outputs", ctypes.c_int32), ("dense_max_span", ctypes.c_int32),
                 ("fallback_cap", ctypes.c_int32), ("dense_span_words_per_product", ctypes.c_float),
                 ("reserved", ctypes.c_int32 * 5)]
 
@@ -59,7 +61,9 @@ class spws_stats_t(ctypes.Structure):
                 ("max_row_products", ctypes.c_int64), ("rows_per_class", ctypes.c_int64 * 8),
                 ("dense_units", ctypes.c_int64), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("products_per_class", ctypes.c_int64 * 8), ("nnz_per_class", ctypes.c_int64 * 8),
-                ("launches_symbolic", ctypes.c_int32), ("launches_numeric", ctypes.c_int32)]
+                ("launches_symbolic", ctypes.c_int32), ("launches_numeric", ctypes.c_int32),
+                ("dense_warp_rows", ctypes.c_int64), ("dense_warp_products", ctypes.c_int64),
+                ("dense_warp_nnz", ctypes.c_int64), ("bitmap_bytes", ctypes.c_int64)]
 
 
 class SpwsError(RuntimeError):
@@ -237,7 +241,9 @@ class Plan:
         d = dict(rows=s.rows, products=s.products, nnz=s.nnz, max_row_products=s.max_row_products,
                  rows_per_class=list(s.rows_per_class), dense_units=s.dense_units, device_status=s.device_status,
                  products_per_class=list(s.products_per_class), nnz_per_class=list(s.nnz_per_class),
-                 launches_symbolic=s.launches_symbolic, launches_numeric=s.launches_numeric)
+                 launches_symbolic=s.launches_symbolic, launches_numeric=s.launches_numeric,
+                 dense_warp_rows=s.dense_warp_rows, dense_warp_products=s.dense_warp_products,
+                 dense_warp_nnz=s.dense_warp_nnz, bitmap_bytes=s.bitmap_bytes)
         _check(st, "spws_get_stats")
         return d
 

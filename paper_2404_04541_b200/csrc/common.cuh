@@ -9,15 +9,24 @@ typedef long long i64;
 typedef unsigned long long u64;
 
 constexpr int NCLASS = 8;
-// Row classes = the workspace a row (or (i,j) fibre) is routed to.
+// Row classes = the workspace a row (or (i,j) fibre) is routed to in the symbolic pass.
 enum RowClass : int {
-    CLS_EMPTY = 0,     // no intermediate product
-    CLS_ISM_REG = 1,   // insert-sort-merge in registers, one lane group per row
-    CLS_ISM_SMEM_S = 2,// insert-sort-merge in shared memory, small CTA
-    CLS_ISM_SMEM = 3,  // insert-sort-merge in shared memory, full CTA
-    CLS_DENSE = 4,     // dense accumulator + occupancy bitmap, (row, column tile) units
-    CLS_ISM_GLOBAL = 5 // accumulation array in shared memory, all array in global memory
+    CLS_EMPTY = 0,      // no intermediate product
+    CLS_ISM_REG = 1,    // insert-sort-merge in registers, one lane group per row
+    CLS_ISM_SMEM_S = 2, // insert-sort-merge in shared memory, small CTA
+    CLS_ISM_SMEM = 3,   // insert-sort-merge in shared memory, full CTA
+    CLS_DENSE_WARP = 4, // dense workspace (occupancy bitmap), one warp per row
+    CLS_DENSE_HUB = 5,  // dense workspace, one CTA per row, heaviest rows (scheduled first)
+    CLS_DENSE_CTA = 6,  // dense workspace, one CTA per row
+    CLS_ISM_GLOBAL = 7  // accumulation array in shared memory, all array in global memory
 };
+
+// Capacities fixed at compile time.
+constexpr int DENSE_WARP_BM_WORDS = 1024;  // bitmap words a warp-per-row workspace may span (32768 columns)
+constexpr int DENSE_WARP_ACC = 256;        // outputs a warp-per-row numeric workspace may hold
+constexpr int DENSE_WARP_MAX_UB = 4096;    // products a single warp is given at most
+constexpr i64 DENSE_HUB_UB = 1ll << 17;    // rows with at least this many products are scheduled first
+constexpr int DENSE_MAX_SPAN_WORDS = 32768;// 2^20 columns: the widest bitmap one CTA can hold
 
 enum DevStatus : int {
     DEV_OK = 0,
@@ -34,15 +43,17 @@ struct DevCtl {
     i64 max_ub;
     i64 max_ub_global;      // largest product count among CLS_ISM_GLOBAL rows
     i64 kept[2];            // TTM: surviving slices (level 0) and fibres (level 1)
+    u64 bm_words_used;      // words handed out of the bitmap arena
     int status;
-    int n_units;
+    int n_units;            // numeric dense CTA units (row, rank range)
+    int n_warp_rows;        // numeric dense warp rows
+    int max_span_words;     // widest bitmap among CTA-class dense rows
     int class_count[NCLASS];
     int class_cursor[NCLASS];
     int work_counter[16];   // dynamic work distribution; cleared before each pass
-    int global_slots;       // slots the global-memory ISM actually used
-    int pad[7];
     i64 class_products[NCLASS];
     i64 class_nnz[NCLASS];
+    i64 dense_warp_products, dense_warp_nnz;   // share of the dense rows the warp numeric kernel takes
 };
 
 struct ClassParams {
@@ -50,10 +61,11 @@ struct ClassParams {
     int reg_cap;            // CLS_ISM_REG: products <= reg_cap
     int smem_small_cap;     // CLS_ISM_SMEM_S
     int smem_cap;           // CLS_ISM_SMEM
-    int tile_cols;          // W
-    int max_tiles;
+    int unit_outputs;       // accumulator capacity of a dense CTA unit
+    int max_span_words;     // dense allowed up to this many bitmap words
     float span_words_per_product;
-    int unit_cap;           // entries available in the unit tables
+    int unit_cap;           // entries available in the unit table
+    u64 bm_arena_words;     // capacity of the bitmap arena
 };
 
 struct Csr {
@@ -72,9 +84,11 @@ struct RowTables {
     int* jmax;
     unsigned char* cls;
     int* perm;
-    int* row_unit0;
-    int* unit_row;
-    int* unit_cnt;
+    i64* bm_off;        // word offset of the row's bitmap in the arena (dense classes)
+    unsigned* bm_arena;
+    int* warp_rows;     // numeric: rows handled by the warp-per-row dense kernel
+    int* row_unit0;     // numeric: first CTA unit of a row
+    int* unit_row;      // numeric: row of a CTA unit
 };
 
 __device__ __forceinline__ void raise_status(DevCtl* ctl, int s) { atomicCAS(&ctl->status, 0, s); }
@@ -116,16 +130,16 @@ __device__ __forceinline__ int block_excl_scan(int v, int* ws, int& total) {
 }
 
 // First position in crd[lo, hi) whose coordinate is >= c (rows are sorted).
-__device__ __forceinline__ i64 lower_bound_crd(const int* __restrict__ crd, i64 lo, i64 hi, int c) {
+__device__ __forceinline__ i64 lower_bound_crd(const int* __restrict__ crd, i64 lo, i64 hi, i64 c) {
     while (lo < hi) {
         const i64 mid = (lo + hi) >> 1;
-        if (__ldg(crd + mid) < c) lo = mid + 1; else hi = mid;
+        if ((i64)__ldg(crd + mid) < c) lo = mid + 1; else hi = mid;
     }
     return lo;
 }
 
 // Products are formed as a rounded multiply followed by rounded adds (no contraction), so the
-// ISM routes, which sum in product order, reproduce a plain sequential sum bit for bit.
+// routes that sum in product order reproduce a plain sequential sum bit for bit.
 __device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
 __device__ __forceinline__ float mul_rn(float a, float b) { return __fmul_rn(a, b); }
 __device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
@@ -139,8 +153,9 @@ struct LaunchCtx {
     ClassParams prm;
     RowTables tab;
     int is_f64;
-    char* global_arena;      // scratch for CLS_ISM_GLOBAL all arrays
-    size_t global_arena_bytes;
+    int dense_smem_words;    // bitmap words the CTA dense kernels reserve (from ncols)
+    char* rest;              // scratch after the fixed tables: bitmap arena, then the ISM-global arena
+    size_t rest_bytes;
     int global_cap;          // accumulation-array capacity of CLS_ISM_GLOBAL
     mutable int launches;    // kernels enqueued through this context
 };
@@ -149,20 +164,24 @@ struct LaunchCtx {
 cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA, i64 nnzB);
 cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA);
 cudaError_t launch_bin_rows(const LaunchCtx& c, int m);
+cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr);
 cudaError_t launch_class_nnz(const LaunchCtx& c, int m);
 cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out);
 cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
                                const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
                                i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2);
-// ism_reg.cu / ism_smem.cu / dense.cu / ism_global.cu: n_host < 0 means "read the count from ctl".
+// class kernels: n_host < 0 means "size the grid for any count"
 cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
                            const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_ism_smem(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                             const i64* rowptr, int* Ccrd, void* Cval);
-cudaError_t launch_dense(const LaunchCtx& c, bool numeric, int n_units_host, const Csr& A, const Csr& B,
-                         const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B);
+cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B);
+cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B,
+                                  const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, const Csr& A, const Csr& B,
+                                 const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
                               const i64* rowptr, int* Ccrd, void* Cval);
-size_t dense_smem_bytes(int tile_cols, int is_f64);
 
 }  // namespace spws

@@ -1,154 +1,435 @@
-// Dense workspace in shared memory: a value array plus an occupancy bitmap along the last
-// index (Gustavson's workspace, Table 2: a flag marks positions that hold a component, so a
-// product deduplicates on insertion; position = coordinate, so the workspace is bucket-sorted;
-// the flagged positions are copied out in order = boolean indexing).  A row's column span
-// [jmin, jmax] is cut into tiles of W columns; one work unit = (row, tile).  Units of one row
-// write disjoint, ordered pieces of the row's output, so hub rows spread over many CTAs
-// without atomics between CTAs.
-//   symbolic : bitmap only; unit_cnt[u] = popcount; cnt[row] += unit_cnt[u].
-//   numeric  : acc[j - c0] += a*b (shared-memory atomics, CTA-wide), then the bitmap is scanned
-//              word by word and (j, acc) is written at row_ptr[i] + (outputs of earlier tiles)
-//              + rank; touched positions are cleared on the way out.
+// Dense workspace: an occupancy bitmap along the last index plus a value array (Gustavson's
+// workspace, Table 2: the flag marks positions that already hold a component, so a product
+// deduplicates on insertion; position = coordinate, so the workspace is bucket-sorted; the
+// flagged positions are copied out in order = boolean indexing).
+//
+// The bitmap covers the row's exact column span [jmin, jmax] and lives in shared memory.  The
+// value array is NOT indexed by column but by the RANK of the column among the row's set bits
+// (rank = prefix popcount), so it holds only as many entries as the row has outputs and is
+// already in output order:
+//   symbolic : gather the column indices of the row's products, set bits; cnt = popcount; the
+//              bitmap is saved to the arena in scratch so the numeric pass need not rebuild it.
+//   numeric  : reload the bitmap, prefix-sum its words, then acc[rank(j)] += a*b for every
+//              product; acc is copied straight to the row's value segment and the set bits give
+//              the column indices.
+// Two granularities:
+//   warp per row : bitmap <= 1024 words, <= 256 outputs.  A warp walks the A entries one at a
+//              time with its lanes across the B row, so no two lanes ever hit the same slot and
+//              the accumulator needs no atomics; sums are in loop order.
+//   CTA units    : any span up to 2^20 columns.  A row is cut into units of `unit_outputs`
+//              consecutive outputs (rank ranges), so units carry equal output counts however
+//              skewed the columns are; hub rows spread over many CTAs and write disjoint,
+//              ordered pieces of the row.  Shared-memory atomics combine the CTA's warps.
 #include "common.cuh"
 
 namespace spws {
 
-constexpr int DENSE_THREADS = 256;
+constexpr int DW_THREADS = 256;            // warp-per-row kernels: 8 warps per CTA
+constexpr int DW_WARPS = DW_THREADS / 32;
+constexpr int DC_THREADS = 256;            // CTA kernels
 
-size_t dense_smem_bytes(int tile_cols, int is_f64) {
-    return (size_t)tile_cols * (is_f64 ? 8 : 4) + (size_t)tile_cols / 8 + 16;
+__device__ __forceinline__ int pick_group_size(i64 ub, i64 entries) {
+    // lanes per A entry: the smallest power of two >= the mean B-row segment length
+    const i64 avg = ub / (entries > 0 ? entries : 1);
+    int gs = 32;
+    while (gs > 1 && (gs >> 1) >= avg) gs >>= 1;
+    return gs;
 }
 
-template <typename T, bool NUMERIC>
-__global__ void __launch_bounds__(DENSE_THREADS) dense_unit_kernel(DevCtl* __restrict__ ctl, int counter_slot, int W,
-                                                                   Csr A, Csr B, RowTables tab,
-                                                                   const i64* __restrict__ rowptr, int* __restrict__ Ccrd, T* __restrict__ Cval) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    T* acc = reinterpret_cast<T*>(smem_raw);                               // W (numeric only)
-    unsigned* bm = reinterpret_cast<unsigned*>(smem_raw + (NUMERIC ? sizeof(T) * (size_t)W : 0));   // W/32
-    __shared__ int s_next, s_tile_off;
-    __shared__ int ws[33];
-    const int tid = threadIdx.x;
+// ---------------------------------------------------------------------------------------
+// symbolic, warp per row
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __restrict__ ctl, Csr A, Csr B, RowTables tab) {
+    __shared__ unsigned s_bm[DW_WARPS][DENSE_WARP_BM_WORDS];
     if (ctl->status != 0) return;
-    const int n_units = ctl->n_units;
+    int off, n;
+    class_range(ctl, CLS_DENSE_WARP, off, n);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned* bm = s_bm[warp];
+    for (;;) {
+        int r = 0;
+        if (lane == 0) r = atomicAdd(&ctl->work_counter[CLS_DENSE_WARP], 1);
+        r = __shfl_sync(0xffffffffu, r, 0);
+        if (r >= n) break;
+        const int row = tab.perm[off + r];
+        const int base = tab.jmin[row];
+        const int nw = (tab.jmax[row] - base) / 32 + 1;
+        const unsigned span = (unsigned)nw * 32u;
+        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        for (int w = lane; w < nw; w += 32) bm[w] = 0;
+        __syncwarp();
+        const int gs = pick_group_size(tab.ub[row], pe - ps);
+        const int g = lane / gs, gl = lane % gs, ng = 32 / gs;
+        for (i64 p = ps + g; p < pe; p += ng) {
+            const int k = __ldg(A.crd + p);
+            if ((unsigned)k >= (unsigned)B.nrows) continue;
+            const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+            for (i64 q = qs + gl; q < qe; q += gs) {
+                const unsigned rel = (unsigned)(__ldg(B.crd + q) - base);
+                if (rel < span) atomicOr(&bm[rel >> 5], 1u << (rel & 31));
+            }
+        }
+        __syncwarp();
+        unsigned* out = tab.bm_arena + tab.bm_off[row];
+        int c = 0;
+        for (int w = lane; w < nw; w += 32) {
+            const unsigned word = bm[w];
+            c += __popc(word);
+            out[w] = word;
+        }
+        for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
+        if (lane == 0) tab.cnt[row] = c;
+        __syncwarp();
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// symbolic, CTA per row (hub rows first: classes HUB and CTA are adjacent in perm)
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, Csr A, Csr B, RowTables tab) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned* bm = reinterpret_cast<unsigned*>(smem_raw);
+    __shared__ int s_next;
+    __shared__ int ws[33];
+    if (ctl->status != 0) return;
+    int off, n_hub, o6, n_cta;
+    class_range(ctl, CLS_DENSE_HUB, off, n_hub);
+    class_range(ctl, CLS_DENSE_CTA, o6, n_cta);
+    const int n = n_hub + n_cta;
+    const int tid = threadIdx.x;
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[CLS_DENSE_CTA], 1);
+        __syncthreads();
+        const int r = s_next;
+        if (r >= n) break;
+        const int row = tab.perm[off + r];
+        const int base = tab.jmin[row];
+        const int nw = min((tab.jmax[row] - base) / 32 + 1, smem_words);
+        const unsigned span = (unsigned)nw * 32u;
+        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        for (int w = tid; w < nw; w += DC_THREADS) bm[w] = 0;
+        __syncthreads();
+        const int gs = pick_group_size(tab.ub[row], pe - ps);
+        const int g = tid / gs, gl = tid % gs, ng = DC_THREADS / gs;
+        for (i64 p = ps + g; p < pe; p += ng) {
+            const int k = __ldg(A.crd + p);
+            if ((unsigned)k >= (unsigned)B.nrows) continue;
+            const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+            i64 q = qs + gl;
+            for (; q + gs < qe; q += 2 * gs) {          // two loads in flight per lane
+                const unsigned r0 = (unsigned)(__ldg(B.crd + q) - base);
+                const unsigned r1 = (unsigned)(__ldg(B.crd + q + gs) - base);
+                if (r0 < span) atomicOr(&bm[r0 >> 5], 1u << (r0 & 31));
+                if (r1 < span) atomicOr(&bm[r1 >> 5], 1u << (r1 & 31));
+            }
+            if (q < qe) {
+                const unsigned r0 = (unsigned)(__ldg(B.crd + q) - base);
+                if (r0 < span) atomicOr(&bm[r0 >> 5], 1u << (r0 & 31));
+            }
+        }
+        __syncthreads();
+        unsigned* out = tab.bm_arena + tab.bm_off[row];
+        int c = 0;
+        for (int w = tid; w < nw; w += DC_THREADS) {
+            const unsigned word = bm[w];
+            c += __popc(word);
+            out[w] = word;
+        }
+        int total;
+        block_excl_scan<DC_THREADS>(c, ws, total);
+        if (tid == 0) tab.cnt[row] = total;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// numeric, warp per row
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __restrict__ ctl, Csr A, Csr B, RowTables tab,
+                                                                    const i64* __restrict__ rowptr, int* __restrict__ Ccrd,
+                                                                    T* __restrict__ Cval) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (ctl->status != 0) return;
+    const int n = ctl->n_warp_rows;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    T* acc = reinterpret_cast<T*>(smem_raw) + warp * DENSE_WARP_ACC;
+    unsigned* bm = reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) + warp * DENSE_WARP_BM_WORDS;
+    unsigned short* pre = reinterpret_cast<unsigned short*>(reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) +
+                                                            DW_WARPS * DENSE_WARP_BM_WORDS) + warp * DENSE_WARP_BM_WORDS;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
+    for (;;) {
+        int r = 0;
+        if (lane == 0) r = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_WARP], 1);
+        r = __shfl_sync(0xffffffffu, r, 0);
+        if (r >= n) break;
+        const int row = tab.warp_rows[r];
+        const int base = tab.jmin[row];
+        const int nw = (tab.jmax[row] - base) / 32 + 1;
+        const unsigned span = (unsigned)nw * 32u;
+        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        const i64 out0 = rowptr[row];
+        const int cnt = (int)(rowptr[row + 1] - out0);
+        // reload the bitmap and prefix-sum its words (rank of each word's first bit)
+        const unsigned* src = tab.bm_arena + tab.bm_off[row];
+        int carry = 0;
+        for (int w0 = 0; w0 < nw; w0 += 32) {
+            const int w = w0 + lane;
+            const unsigned word = (w < nw) ? src[w] : 0u;
+            const int c = __popc(word);
+            const int incl = warp_incl_scan(c);
+            if (w < nw) { bm[w] = word; pre[w] = (unsigned short)(carry + incl - c); }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        for (int x = lane; x < cnt; x += 32) acc[x] = 0;
+        __syncwarp();
+        const int gs = pick_group_size(tab.ub[row], pe - ps);
+        if (gs == 32) {
+            // one A entry at a time, lanes across its B row: distinct columns, no atomics,
+            // every output summed in loop order
+            for (i64 p = ps; p < pe; ++p) {
+                const int k = __ldg(A.crd + p);
+                if ((unsigned)k >= (unsigned)B.nrows) continue;
+                const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                const T a = __ldg(Aval + p);
+                for (i64 q = qs + lane; q < qe; q += 32) {
+                    const unsigned rel = (unsigned)(__ldg(B.crd + q) - base);
+                    if (rel < span) {
+                        const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
+                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a, __ldg(Bval + q)));
+                    }
+                }
+                __syncwarp();
+            }
+        } else {
+            // short B rows: several A entries in flight, so slots can collide -> atomics
+            const int g = lane / gs, gl = lane % gs, ng = 32 / gs;
+            for (i64 p = ps + g; p < pe; p += ng) {
+                const int k = __ldg(A.crd + p);
+                if ((unsigned)k >= (unsigned)B.nrows) continue;
+                const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                const T a = __ldg(Aval + p);
+                for (i64 q = qs + gl; q < qe; q += gs) {
+                    const unsigned rel = (unsigned)(__ldg(B.crd + q) - base);
+                    if (rel < span) {
+                        const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
+                        if (slot < DENSE_WARP_ACC) atomicAdd(&acc[slot], mul_rn(a, __ldg(Bval + q)));
+                    }
+                }
+            }
+            __syncwarp();
+        }
+        // copy out: values are already in output order; set bits give the coordinates
+        for (int x = lane; x < cnt; x += 32) Cval[out0 + x] = acc[x];
+        for (int w = lane; w < nw; w += 32) {
+            unsigned word = bm[w];
+            i64 o = out0 + pre[w];
+            while (word) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+                Ccrd[o++] = base + (w << 5) + b;
+            }
+        }
+        __syncwarp();
+    }
+}
 
-    if (NUMERIC)
-        for (int x = tid; x < W; x += DENSE_THREADS) acc[x] = 0;
-    for (int x = tid; x < W / 32; x += DENSE_THREADS) bm[x] = 0;
+// ---------------------------------------------------------------------------------------
+// numeric, CTA units (row, rank range)
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int nth_set_bit(unsigned word, int nth) {   // position of the nth (0-based) set bit
+    for (int x = 0; x < nth; ++x) word &= word - 1;
+    return __ffs(word) - 1;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(DC_THREADS) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, Csr A, Csr B,
+                                                                   RowTables tab, const i64* __restrict__ rowptr,
+                                                                   int* __restrict__ Ccrd, T* __restrict__ Cval) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
+    unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
+    short* pre = reinterpret_cast<short*>(bm + smem_words);                          // smem_words: rank of word start - r0
+    __shared__ int s_next, s_w0, s_w1;
+    __shared__ i64 s_c0, s_c1;
+    __shared__ int ws[33];
+    if (ctl->status != 0) return;
+    const int n_units = ctl->n_units;
+    const int tid = threadIdx.x;
+    const T* __restrict__ Aval = (const T*)A.val;
+    const T* __restrict__ Bval = (const T*)B.val;
+    for (int x = tid; x < CAP; x += DC_THREADS) acc[x] = 0;
 
     for (;;) {
         __syncthreads();
-        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[counter_slot], 1);
+        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_CTA], 1);
         __syncthreads();
         const int u = s_next;
         if (u >= n_units) break;
         const int row = tab.unit_row[u];
-        const int u0 = tab.row_unit0[row];
-        const int t = u - u0;
+        const int uidx = u - tab.row_unit0[row];
         const int base = tab.jmin[row], last = tab.jmax[row];
-        const int ntiles = (last - base) / W + 1;
-        const i64 c0 = (i64)base + (i64)t * W;
-        const unsigned width = (unsigned)min((i64)W, (i64)last + 1 - c0);
+        const int nw = min((last - base) / 32 + 1, smem_words);
+        const i64 out0 = rowptr[row];
+        const int cnt = (int)(rowptr[row + 1] - out0);
+        const int r0 = uidx * CAP;
+        const int nout = min(CAP, cnt - r0);
+        const int r1 = r0 + nout;
+        const bool whole = (r0 == 0 && r1 == cnt);
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        if (tid == 0) { s_w0 = 0; s_w1 = nw - 1; s_c0 = base; s_c1 = (i64)last + 1; }
+        __syncthreads();
 
-        if (NUMERIC && tid < 32) {          // outputs of the earlier tiles of this row
-            int s = 0;
-            for (int x = tid; x < t; x += 32) s += tab.unit_cnt[u0 + x];
-            for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-            if (tid == 0) s_tile_off = s;
+        // bitmap + word prefix; the words holding ranks r0 and r1 give the unit's column range
+        const unsigned* src = tab.bm_arena + tab.bm_off[row];
+        int carry = 0;
+        for (int w0 = 0; w0 < nw; w0 += DC_THREADS) {
+            const int w = w0 + tid;
+            const unsigned word = (w < nw) ? src[w] : 0u;
+            const int c = __popc(word);
+            int chunk_total;
+            const int start = carry + block_excl_scan<DC_THREADS>(c, ws, chunk_total);   // rank of the word's first bit
+            if (w < nw) {
+                bm[w] = word;
+                const int rel = start - r0;
+                pre[w] = (short)max(-32768, min(32767, rel));
+                if (start <= r0 && r0 < start + c) { s_w0 = w; s_c0 = (i64)base + (w << 5) + nth_set_bit(word, r0 - start); }
+                if (r1 < cnt && start <= r1 && r1 < start + c) { s_w1 = w; s_c1 = (i64)base + (w << 5) + nth_set_bit(word, r1 - start); }
+            }
+            carry += chunk_total;
         }
+        __syncthreads();
+        const i64 c0 = s_c0, c1 = s_c1;               // the unit owns columns [c0, c1)
+        const unsigned lo_rel = (unsigned)(c0 - base), hi_rel = (unsigned)(c1 - base);
 
-        // lanes per A entry: about the expected length of a B-row segment inside this tile
-        int gs = 32;
-        {
-            const i64 nA = pe - ps;
-            const i64 avg = tab.ub[row] / (nA * ntiles > 0 ? nA * ntiles : 1);
-            while (gs > 1 && (gs >> 1) >= avg) gs >>= 1;
-        }
-        const int g = tid / gs, gl = tid % gs, ngroups = DENSE_THREADS / gs;
-        for (i64 p = ps + g; p < pe; p += ngroups) {
+        const int nunits_row = (cnt + CAP - 1) / CAP;
+        const int gs = pick_group_size(tab.ub[row] / nunits_row, pe - ps);
+        const int g = tid / gs, gl = tid % gs, ng = DC_THREADS / gs;
+        for (i64 p = ps + g; p < pe; p += ng) {
             const int k = __ldg(A.crd + p);
             if ((unsigned)k >= (unsigned)B.nrows) continue;
-            i64 qs = __ldg(B.pos + k);
-            const i64 qe = __ldg(B.pos + k + 1);
-            if (ntiles > 1) qs = lower_bound_crd(B.crd, qs, qe, (int)c0);
-            T a = 0;
-            if (NUMERIC) a = __ldg(Aval + p);
-            for (i64 q = qs + gl; q < qe; q += gs) {
-                const unsigned rel = (unsigned)((i64)__ldg(B.crd + q) - c0);
-                if (rel >= width) break;
-                if (NUMERIC) atomicAdd(&acc[rel], a * __ldg(Bval + q));
-                atomicOr(&bm[rel >> 5], 1u << (rel & 31));
+            i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+            if (!whole) {
+                qs = lower_bound_crd(B.crd, qs, qe, c0);
+                qe = lower_bound_crd(B.crd, qs, qe, c1);
+            }
+            const T a = __ldg(Aval + p);
+            i64 q = qs + gl;
+            for (; q + gs < qe; q += 2 * gs) {          // two products in flight per lane
+                const unsigned rel0 = (unsigned)(__ldg(B.crd + q) - base);
+                const unsigned rel1 = (unsigned)(__ldg(B.crd + q + gs) - base);
+                const T v0 = a * __ldg(Bval + q);
+                const T v1 = a * __ldg(Bval + q + gs);
+                if (rel0 >= lo_rel && rel0 < hi_rel) {
+                    const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                    if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], v0);
+                }
+                if (rel1 >= lo_rel && rel1 < hi_rel) {
+                    const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
+                    if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], v1);
+                }
+            }
+            if (q < qe) {
+                const unsigned rel0 = (unsigned)(__ldg(B.crd + q) - base);
+                if (rel0 >= lo_rel && rel0 < hi_rel) {
+                    const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                    if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * __ldg(Bval + q));
+                }
             }
         }
         __syncthreads();
 
-        // ---- copy out in coordinate order
-        const int nwords = (int)((width + 31) >> 5);
-        int running = 0;
-        const i64 out0 = NUMERIC ? rowptr[row] + s_tile_off : 0;
-        for (int w0 = 0; w0 < nwords; w0 += DENSE_THREADS) {
-            const int w = w0 + tid;
-            unsigned bits = (w < nwords) ? bm[w] : 0u;
-            int chunk_total;
-            const int off = block_excl_scan<DENSE_THREADS>(__popc(bits), ws, chunk_total);
-            if (bits) {
-                bm[w] = 0;
-                if (NUMERIC) {
-                    i64 out = out0 + running + off;
-                    while (bits) {
-                        const int b = __ffs(bits) - 1;
-                        bits &= bits - 1;
-                        const int rel = (w << 5) + b;
-                        Ccrd[out] = (int)(c0 + rel);
-                        Cval[out] = acc[rel];
-                        acc[rel] = 0;
-                        ++out;
-                    }
+        // copy out
+        const i64 o0 = out0 + r0;
+        for (int x = tid; x < nout; x += DC_THREADS) { Cval[o0 + x] = acc[x]; acc[x] = 0; }
+        const int w_first = s_w0, w_last = s_w1;
+        for (int w = w_first + tid; w <= w_last; w += DC_THREADS) {
+            unsigned word = bm[w];
+            const int wp = pre[w];
+            const unsigned full = word;
+            while (word) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+                const unsigned rel = ((unsigned)w << 5) + (unsigned)b;
+                if (rel >= lo_rel && rel < hi_rel) {
+                    const int slot = wp + __popc(full & ((1u << b) - 1u));
+                    if ((unsigned)slot < (unsigned)nout) Ccrd[o0 + slot] = base + (int)rel;
                 }
             }
-            running += chunk_total;
-        }
-        if (!NUMERIC && tid == 0) {
-            tab.unit_cnt[u] = running;
-            atomicAdd(&tab.cnt[row], running);
         }
     }
 }
 
-template <typename T>
-static cudaError_t launch_t(const LaunchCtx& c, bool numeric, int n_units_host, const Csr& A, const Csr& B,
-                            const i64* rowptr, int* Ccrd, void* Cval) {
-    const int W = c.prm.tile_cols;
-    const size_t smem = (numeric ? sizeof(T) * (size_t)W : 0) + (size_t)W / 8 + 16;
-    const int slot = CLS_DENSE + (numeric ? 8 : 0);
-    cudaError_t e;
+// ---------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------
+static int persistent_grid(const LaunchCtx& c, int per_sm, i64 work) {
+    i64 grid = (i64)c.sm_count * (per_sm > 0 ? per_sm : 1);
+    if (work >= 0 && work < grid) grid = work > 0 ? work : 1;
+    return (int)grid;
+}
+
+cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B) {
     int per_sm = 0;
-    if (numeric) {
-        auto k = dense_unit_kernel<T, true>;
-        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DENSE_THREADS, smem)) != cudaSuccess) return e;
-        i64 grid = (i64)c.sm_count * (per_sm > 0 ? per_sm : 1);
-        if (n_units_host >= 0 && n_units_host < grid) grid = n_units_host > 0 ? n_units_host : 1;
-        k<<<(int)grid, DENSE_THREADS, smem, c.stream>>>(c.ctl, slot, W, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
-    } else {
-        auto k = dense_unit_kernel<T, false>;
-        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DENSE_THREADS, smem)) != cudaSuccess) return e;
-        i64 grid = (i64)c.sm_count * (per_sm > 0 ? per_sm : 1);
-        if (n_units_host >= 0 && n_units_host < grid) grid = n_units_host > 0 ? n_units_host : 1;
-        k<<<(int)grid, DENSE_THREADS, smem, c.stream>>>(c.ctl, slot, W, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
-    }
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_sym_warp_kernel, DW_THREADS, 0);
+    if (e != cudaSuccess) return e;
+    dense_sym_warp_kernel<<<persistent_grid(c, per_sm, -1), DW_THREADS, 0, c.stream>>>(c.ctl, A, B, c.tab);
     ++c.launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_dense(const LaunchCtx& c, bool numeric, int n_units_host, const Csr& A, const Csr& B,
-                         const i64* rowptr, int* Ccrd, void* Cval) {
-    return c.is_f64 ? launch_t<double>(c, numeric, n_units_host, A, B, rowptr, Ccrd, Cval)
-                    : launch_t<float>(c, numeric, n_units_host, A, B, rowptr, Ccrd, Cval);
+cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B) {
+    const size_t smem = (size_t)c.dense_smem_words * 4;
+    cudaError_t e;
+    int per_sm = 0;
+    if ((e = cudaFuncSetAttribute(dense_sym_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_sym_cta_kernel, DC_THREADS, smem)) != cudaSuccess) return e;
+    dense_sym_cta_kernel<<<persistent_grid(c, per_sm, -1), DC_THREADS, smem, c.stream>>>(c.ctl, c.dense_smem_words, A, B, c.tab);
+    ++c.launches;
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
+    int per_sm = 0;
+    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * DENSE_WARP_ACC + 6 * (size_t)DENSE_WARP_BM_WORDS);
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(dense_num_warp_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_num_warp_kernel<T>, DW_THREADS, smem)) != cudaSuccess) return e;
+    const i64 work = n_host >= 0 ? ((i64)n_host + DW_WARPS - 1) / DW_WARPS : -1;
+    dense_num_warp_kernel<T><<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
+    ++c.launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B,
+                                  const i64* rowptr, int* Ccrd, void* Cval) {
+    return c.is_f64 ? num_warp_t<double>(c, n_host, A, B, rowptr, Ccrd, Cval)
+                    : num_warp_t<float>(c, n_host, A, B, rowptr, Ccrd, Cval);
+}
+
+template <typename T>
+static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, const Csr& A, const Csr& B,
+                             const i64* rowptr, int* Ccrd, void* Cval) {
+    const int CAP = c.prm.unit_outputs;
+    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)words * 2 + 16;
+    cudaError_t e;
+    int per_sm = 0;
+    auto k = dense_num_cta_kernel<T>;
+    if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DC_THREADS, smem)) != cudaSuccess) return e;
+    k<<<persistent_grid(c, per_sm, n_units_host), DC_THREADS, smem, c.stream>>>(c.ctl, words, CAP, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
+    ++c.launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, const Csr& A, const Csr& B,
+                                 const i64* rowptr, int* Ccrd, void* Cval) {
+    int words = max_span_words > 0 ? max_span_words : c.dense_smem_words;
+    words = (words + 7) & ~7;
+    return c.is_f64 ? num_cta_t<double>(c, n_units_host, words, A, B, rowptr, Ccrd, Cval)
+                    : num_cta_t<float>(c, n_units_host, words, A, B, rowptr, Ccrd, Cval);
 }
 
 }  // namespace spws

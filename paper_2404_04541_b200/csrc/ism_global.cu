@@ -21,7 +21,7 @@ constexpr int GL_CAPMAX = 2048;
 
 template <typename T, bool NUMERIC>
 __global__ void __launch_bounds__(GL_THREADS) ism_global_kernel(const int* __restrict__ perm, DevCtl* __restrict__ ctl, int counter_slot,
-                                                                int cap, char* arena, size_t arena_bytes,
+                                                                int cap, char* rest, size_t rest_bytes,
                                                                 Csr A, Csr B, int* __restrict__ cnt,
                                                                 const i64* __restrict__ rowptr, int* __restrict__ Ccrd, T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -46,6 +46,10 @@ __global__ void __launch_bounds__(GL_THREADS) ism_global_kernel(const int* __res
     const T* __restrict__ Bval = (const T*)B.val;
     const int tid = threadIdx.x;
 
+    // the arena follows the bitmap arena in the rest of the scratch buffer
+    const size_t bm_bytes = ((size_t)ctl->bm_words_used * 4 + 255) & ~(size_t)255;
+    char* arena = rest + bm_bytes;
+    const size_t arena_bytes = rest_bytes > bm_bytes ? rest_bytes - bm_bytes : 0;
     // one slot per CTA: two all-array buffers of slot_elems components
     i64 slot_elems = min(ctl->max_ub_global, (i64)B.ncols);
     slot_elems = (slot_elems + 63) & ~63ll;
@@ -249,12 +253,12 @@ static cudaError_t launch_t(const LaunchCtx& c, bool numeric, int n_host, const 
     if (numeric) {
         auto k = ism_global_kernel<T, true>;
         if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        k<<<(int)grid, GL_THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, slot, c.global_cap, c.global_arena, c.global_arena_bytes,
+        k<<<(int)grid, GL_THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, slot, c.global_cap, c.rest, c.rest_bytes,
                                                     A, B, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     } else {
         auto k = ism_global_kernel<T, false>;
         if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        k<<<(int)grid, GL_THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, slot, c.global_cap, c.global_arena, c.global_arena_bytes,
+        k<<<(int)grid, GL_THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, slot, c.global_cap, c.rest, c.rest_bytes,
                                                     A, B, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     }
     ++c.launches;

@@ -40,14 +40,20 @@ cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 
 // [jmin, jmax] of the candidate columns (first / last coordinate of the picked B rows, which
 // are sorted), and the workspace class of the row.
 // ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int dense_class(i64 ub, i64 span_words) {
+    if (span_words <= DENSE_WARP_BM_WORDS && ub <= DENSE_WARP_MAX_UB) return CLS_DENSE_WARP;
+    return ub >= DENSE_HUB_UB ? CLS_DENSE_HUB : CLS_DENSE_CTA;
+}
+
 __device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const ClassParams& prm, DevCtl* ctl) {
     if (ub == 0) return CLS_EMPTY;
     const i64 span = (i64)jmax - jmin + 1;
-    const i64 ntiles = (span + prm.tile_cols - 1) / prm.tile_cols;
+    const i64 span_words = (span + 31) >> 5;
+    const bool dense_ok = span_words <= prm.max_span_words;
     const bool reg_ok = ub <= prm.reg_cap && span <= (1ll << 26);
     if (prm.policy == 0) {                       // dense forced
-        if (ntiles > prm.max_tiles) { raise_status(ctl, DEV_WORKSPACE_TOO_LARGE); return CLS_EMPTY; }
-        return CLS_DENSE;
+        if (!dense_ok) { raise_status(ctl, DEV_WORKSPACE_TOO_LARGE); return CLS_EMPTY; }
+        return dense_class(ub, span_words);
     }
     if (prm.policy == 1) {                       // sparse ISM forced
         if (reg_ok) return CLS_ISM_REG;
@@ -55,14 +61,13 @@ __device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const Cl
         if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
         return CLS_ISM_GLOBAL;
     }
-    // auto: few products -> sort them; a narrow span relative to the work -> dense tile;
-    // mid-size rows -> shared-memory ISM; long rows -> column-tiled dense; otherwise global ISM.
+    // auto: few products -> sort them in registers; a bitmap that is small next to the work ->
+    // dense; mid-size rows -> shared-memory ISM; long rows -> dense; otherwise global ISM.
     if (reg_ok) return CLS_ISM_REG;
-    const i64 span_words = (span + 31) >> 5;
-    if (ntiles == 1 && (float)span_words <= prm.span_words_per_product * (float)ub) return CLS_DENSE;
+    if (dense_ok && (float)span_words <= prm.span_words_per_product * (float)ub) return dense_class(ub, span_words);
     if (ub <= prm.smem_small_cap) return CLS_ISM_SMEM_S;
     if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
-    if (ntiles <= prm.max_tiles) return CLS_DENSE;
+    if (dense_ok) return dense_class(ub, span_words);
     return CLS_ISM_GLOBAL;
 }
 
@@ -71,8 +76,9 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
     __shared__ int s_hist[NCLASS];
     __shared__ i64 s_cprod[NCLASS];
     __shared__ i64 s_products, s_max_ub, s_max_ub_global;
+    __shared__ int s_max_span_words;
     if (threadIdx.x < NCLASS) { s_hist[threadIdx.x] = 0; s_cprod[threadIdx.x] = 0; }
-    if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; }
+    if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; s_max_span_words = 0; }
     __syncthreads();
     const int gl = threadIdx.x % G;
     const unsigned lane = threadIdx.x & 31;
@@ -118,6 +124,8 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             my_products += u;
             my_max = max(my_max, u);
             if (cls == CLS_ISM_GLOBAL) my_max_global = max(my_max_global, u);
+            if (cls == CLS_DENSE_HUB || cls == CLS_DENSE_CTA || cls == CLS_DENSE_WARP)
+                atomicMax(&s_max_span_words, (hi - lo) / 32 + 1);
         }
     }
     if (gl == 0 && my_products) atomicAdd((u64*)&s_products, (u64)my_products);
@@ -132,6 +140,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         if (s_products) atomicAdd((u64*)&ctl->products, (u64)s_products);
         if (s_max_ub) atomicMax(&ctl->max_ub, s_max_ub);
         if (s_max_ub_global) atomicMax(&ctl->max_ub_global, s_max_ub_global);
+        if (s_max_span_words) atomicMax(&ctl->max_span_words, s_max_span_words);
     }
 }
 
@@ -153,7 +162,8 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
 
 // ---------------------------------------------------------------------------------------
 // Binning: rows grouped by class into perm (class c occupies [off[c], off[c+1])); dense rows
-// also reserve their (row, tile) units.  Order inside a class follows block arrival.
+// also reserve the slot of their occupancy bitmap in the arena.  Order inside a class follows
+// block arrival.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
     __shared__ int s_hist[NCLASS], s_base[NCLASS], s_off[NCLASS];
@@ -184,15 +194,14 @@ __global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, Cla
             const i64 row = r0 + x * blockDim.x + threadIdx.x;
             if (cls[x] < 0) continue;
             tab.perm[s_off[cls[x]] + s_base[cls[x]] + rank[x]] = (int)row;
-            if (cls[x] == CLS_DENSE) {
-                const int ntiles = (tab.jmax[row] - tab.jmin[row]) / prm.tile_cols + 1;
-                const int u0 = atomicAdd(&ctl->n_units, ntiles);
-                if (u0 + ntiles > prm.unit_cap) {
+            if (cls[x] == CLS_DENSE_WARP || cls[x] == CLS_DENSE_HUB || cls[x] == CLS_DENSE_CTA) {
+                const u64 words = (u64)((tab.jmax[row] - tab.jmin[row]) / 32 + 1);
+                const u64 at = atomicAdd(&ctl->bm_words_used, words);
+                if (at + words > prm.bm_arena_words) {
                     raise_status(ctl, DEV_SCRATCH_TOO_SMALL);
-                    tab.row_unit0[row] = -1;
+                    tab.bm_off[row] = -1;
                 } else {
-                    tab.row_unit0[row] = u0;
-                    for (int t = 0; t < ntiles; ++t) tab.unit_row[u0 + t] = (int)row;
+                    tab.bm_off[row] = (i64)at;
                 }
             }
         }
@@ -205,6 +214,47 @@ cudaError_t launch_bin_rows(const LaunchCtx& c, int m) {
     i64 want = ((i64)m + 1023) / 1024;
     i64 cap = (i64)c.sm_count * 8;
     bin_rows_kernel<<<(int)(want < cap ? want : cap), 256, 0, c.stream>>>(m, c.tab, c.prm, c.ctl);
+    ++c.launches;
+    return cudaGetLastError();
+}
+
+// Numeric routing of the dense rows, once their output counts are known: a row the warp kernel
+// counted and whose outputs fit a warp's accumulator stays with a warp; every other row is cut
+// into CTA units of `unit_outputs` consecutive outputs (rank ranges).
+__global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
+    int off, n4, n5, n6, o5, o6;
+    class_range(ctl, CLS_DENSE_WARP, off, n4);
+    class_range(ctl, CLS_DENSE_HUB, o5, n5);
+    class_range(ctl, CLS_DENSE_CTA, o6, n6);
+    const int n = n4 + n5 + n6;                       // the three classes are adjacent in perm
+    for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += (i64)gridDim.x * blockDim.x) {
+        const int row = tab.perm[off + r];
+        const int cnt = tab.cnt[row];
+        if (tab.cls[row] == CLS_DENSE_WARP && cnt <= DENSE_WARP_ACC) {
+            tab.warp_rows[atomicAdd(&ctl->n_warp_rows, 1)] = row;
+            tab.row_unit0[row] = -1;
+            atomicAdd((u64*)&ctl->dense_warp_products, (u64)tab.ub[row]);
+            atomicAdd((u64*)&ctl->dense_warp_nnz, (u64)cnt);
+        } else {
+            const int nu = (cnt + prm.unit_outputs - 1) / prm.unit_outputs;
+            const int u0 = atomicAdd(&ctl->n_units, nu);
+            if (u0 + nu > prm.unit_cap) {
+                raise_status(ctl, DEV_SCRATCH_TOO_SMALL);
+                tab.row_unit0[row] = -1;
+            } else {
+                tab.row_unit0[row] = u0;
+                for (int t = 0; t < nu; ++t) tab.unit_row[u0 + t] = row;
+            }
+        }
+    }
+}
+
+cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr) {
+    (void)rowptr;
+    if (m == 0) return cudaSuccess;
+    i64 want = ((i64)m + 255) / 256;
+    i64 cap = (i64)c.sm_count * 8;
+    dense_rebin_kernel<<<(int)(want < cap ? want : cap), 256, 0, c.stream>>>(m, c.tab, c.prm, c.ctl);
     ++c.launches;
     return cudaGetLastError();
 }

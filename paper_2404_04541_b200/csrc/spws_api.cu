@@ -30,6 +30,7 @@ struct spws_plan_s {
     // what the last symbolic pass saw (numeric must be called with the same shapes and scratch)
     int64_t m = 0;
     void* scratch = nullptr;
+    int max_span_words = 0;     // widest dense bitmap of the last symbolic pass
     // optional per-kernel timing: ev[g] is recorded after group g; ev_start[] before each pass
     bool profiling = false;
     cudaEvent_t ev[SPWS_T_COUNT] = {};
@@ -112,9 +113,10 @@ bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
 // ---- scratch layout ------------------------------------------------------------------------
 struct Layout {
-    size_t ctl, ub, rowptr_raw, cnt, jmin, jmax, cls, perm, row_unit0, unit_row, unit_cnt, block_sums,
-        flags, fpos, sflags, spos, arena, fixed_end;
+    size_t ctl, ub, rowptr_raw, cnt, jmin, jmax, cls, perm, bm_off, warp_rows, row_unit0, unit_row, block_sums,
+        flags, fpos, sflags, spos, rest, fixed_end;
     int unit_cap;
+    int dense_smem_words;
 };
 
 Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) {
@@ -129,15 +131,20 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) 
     L.jmax = take(4 * (size_t)m);
     L.cls = take((size_t)m);
     L.perm = take(4 * (size_t)m);
+    L.bm_off = take(8 * (size_t)m);
+    L.warp_rows = take(4 * (size_t)m);
     L.row_unit0 = take(4 * (size_t)m);
-    int64_t tiles_per_row = (ncols + p->opt.dense_tile_cols - 1) / p->opt.dense_tile_cols;
-    if (tiles_per_row > p->opt.max_dense_tiles) tiles_per_row = p->opt.max_dense_tiles;
-    if (tiles_per_row < 1) tiles_per_row = 1;
-    int64_t ucap = m * tiles_per_row;
+    // a dense row has at most min(ncols, dense_max_span) outputs
+    const int64_t span_cap = ncols < p->opt.dense_max_span ? ncols : p->opt.dense_max_span;
+    int64_t units_per_row = (span_cap + p->opt.dense_unit_outputs - 1) / p->opt.dense_unit_outputs;
+    if (units_per_row < 1) units_per_row = 1;
+    int64_t ucap = m * units_per_row;
     if (ucap > 0x7fff0000ll) ucap = 0x7fff0000ll;
     L.unit_cap = (int)ucap;
     L.unit_row = take(4 * (size_t)ucap);
-    L.unit_cnt = take(4 * (size_t)ucap);
+    int64_t words = (span_cap + 31) / 32 + 1;
+    if (words > DENSE_MAX_SPAN_WORDS) words = DENSE_MAX_SPAN_WORDS;
+    L.dense_smem_words = (int)((words + 7) & ~7ll);
     const size_t longest = (size_t)(m > n_i ? m : n_i);
     L.block_sums = take(8 * (longest / 2048 + 2));
     if (p->kind == 1) {
@@ -147,15 +154,24 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) 
         L.spos = take(8 * ((size_t)n_i + 1));
     }
     L.fixed_end = o;
-    L.arena = o;
+    L.rest = o;
     return L;
 }
 
-// reserve for the global-memory ISM: room for a few slots of min(ncols, 2^22) components
-size_t global_reserve(const spws_plan_s* p, int64_t ncols) {
-    const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
-    const size_t comp = 4 + (p->is_f64 ? 8 : 4);
-    return align256(2 * (size_t)((elems + 63) & ~63ll) * comp) * 8;
+// what follows the fixed tables: one bitmap per row in the worst case (dense routes), and room
+// for a few slots of min(ncols, 2^22) components for the global-memory ISM
+size_t rest_reserve(const spws_plan_s* p, int64_t m, int64_t ncols) {
+    size_t bytes = 0;
+    if (p->policy != SPWS_SPARSE_ISM) {
+        const int64_t span_cap = ncols < p->opt.dense_max_span ? ncols : p->opt.dense_max_span;
+        bytes += align256((size_t)m * (size_t)((span_cap + 31) / 32 + 1) * 4);
+    }
+    if (p->policy != SPWS_DENSE) {
+        const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
+        const size_t comp = 4 + (p->is_f64 ? 8 : 4);
+        bytes += align256(2 * (size_t)((elems + 63) & ~63ll) * comp) * 8;
+    }
+    return bytes;
 }
 
 struct Shapes {
@@ -217,22 +233,26 @@ LaunchCtx make_ctx(const spws_plan_s* p, char* scratch, size_t scratch_bytes, co
     c.prm.reg_cap = p->opt.ism_warp_cap;
     c.prm.smem_cap = p->opt.ism_cta_cap;
     c.prm.smem_small_cap = p->opt.ism_cta_cap >= 1024 ? 256 : (p->opt.ism_cta_cap >= 256 ? 64 : p->opt.ism_cta_cap);
-    c.prm.tile_cols = p->opt.dense_tile_cols;
-    c.prm.max_tiles = p->opt.max_dense_tiles;
+    c.prm.unit_outputs = p->opt.dense_unit_outputs;
+    c.prm.max_span_words = (p->opt.dense_max_span + 31) / 32;
     c.prm.span_words_per_product = p->opt.dense_span_words_per_product;
     c.prm.unit_cap = L.unit_cap;
+    c.rest = scratch + L.rest;
+    c.rest_bytes = scratch_bytes > L.rest ? scratch_bytes - L.rest : 0;
+    c.prm.bm_arena_words = p->policy == SPWS_SPARSE_ISM ? 0 : c.rest_bytes / 4;
+    c.dense_smem_words = L.dense_smem_words;
     c.tab.ub = reinterpret_cast<i64*>(scratch + L.ub);
     c.tab.cnt = reinterpret_cast<int*>(scratch + L.cnt);
     c.tab.jmin = reinterpret_cast<int*>(scratch + L.jmin);
     c.tab.jmax = reinterpret_cast<int*>(scratch + L.jmax);
     c.tab.cls = reinterpret_cast<unsigned char*>(scratch + L.cls);
     c.tab.perm = reinterpret_cast<int*>(scratch + L.perm);
+    c.tab.bm_off = reinterpret_cast<i64*>(scratch + L.bm_off);
+    c.tab.bm_arena = reinterpret_cast<unsigned*>(scratch + L.rest);
+    c.tab.warp_rows = reinterpret_cast<int*>(scratch + L.warp_rows);
     c.tab.row_unit0 = reinterpret_cast<int*>(scratch + L.row_unit0);
     c.tab.unit_row = reinterpret_cast<int*>(scratch + L.unit_row);
-    c.tab.unit_cnt = reinterpret_cast<int*>(scratch + L.unit_cnt);
     c.is_f64 = p->is_f64;
-    c.global_arena = scratch + L.arena;
-    c.global_arena_bytes = scratch_bytes > L.arena ? scratch_bytes - L.arena : 0;
     c.global_cap = p->opt.fallback_cap;
     return c;
 }
@@ -317,15 +337,15 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
     const bool f64 = value_type == SPWS_F64;
     if (o.ism_warp_cap == 0) o.ism_warp_cap = 32;
     if (o.ism_cta_cap == 0) o.ism_cta_cap = 4096;
-    if (o.dense_tile_cols == 0) o.dense_tile_cols = f64 ? 8192 : 16384;
-    if (o.max_dense_tiles == 0) o.max_dense_tiles = 64;
+    if (o.dense_unit_outputs == 0) o.dense_unit_outputs = 4096;
+    if (o.dense_max_span == 0) o.dense_max_span = 1 << 20;
     if (o.fallback_cap == 0) o.fallback_cap = 2048;
     if (o.dense_span_words_per_product == 0.0f) o.dense_span_words_per_product = 4.0f;
     if (o.validate != 0 && o.validate != 1) return SPWS_INVALID_ARGUMENT;
     if (o.ism_warp_cap < 1 || o.ism_warp_cap > 32) return SPWS_INVALID_ARGUMENT;
     if (!is_pow2(o.ism_cta_cap) || o.ism_cta_cap < 64 || o.ism_cta_cap > 4096) return SPWS_INVALID_ARGUMENT;
-    if (!is_pow2(o.dense_tile_cols) || o.dense_tile_cols < 256 || o.dense_tile_cols > 16384) return SPWS_INVALID_ARGUMENT;
-    if (o.max_dense_tiles < 1 || o.max_dense_tiles > 4096) return SPWS_INVALID_ARGUMENT;
+    if (!is_pow2(o.dense_unit_outputs) || o.dense_unit_outputs < 64 || o.dense_unit_outputs > 8192) return SPWS_INVALID_ARGUMENT;
+    if (o.dense_max_span < 32 || o.dense_max_span > (1 << 20)) return SPWS_INVALID_ARGUMENT;
     if (!is_pow2(o.fallback_cap) || o.fallback_cap < 2 || o.fallback_cap > 2048) return SPWS_INVALID_ARGUMENT;
     if (!(o.dense_span_words_per_product > 0.0f)) return SPWS_INVALID_ARGUMENT;
     spws_plan_s* p = new (std::nothrow) spws_plan_s;
@@ -390,7 +410,7 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
     spws_status_t st = check_operands(plan, A, B, S, false);   // pointers may still be unset when sizing
     if (st != SPWS_OK) return st;
     const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
-    *bytes = L.fixed_end + global_reserve(plan, S.ncols);
+    *bytes = L.fixed_end + rest_reserve(plan, S.m, S.ncols);
     return SPWS_OK;
 }
 
@@ -434,8 +454,10 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
             mark(plan, SPWS_T_SYM_ISM_SMEM);
         }
         if (plan->policy != SPWS_SPARSE_ISM) {
-            CUDA_TRY(launch_dense(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
-            mark(plan, SPWS_T_SYM_DENSE);
+            CUDA_TRY(launch_dense_sym_warp(c, S.A, S.B));
+            mark(plan, SPWS_T_SYM_DENSE_WARP);
+            CUDA_TRY(launch_dense_sym_cta(c, S.A, S.B));
+            mark(plan, SPWS_T_SYM_DENSE_CTA);
         }
         if (plan->policy != SPWS_DENSE) {
             CUDA_TRY(launch_ism_global(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
@@ -450,6 +472,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
                                     reinterpret_cast<int*>(sc + L.sflags), reinterpret_cast<i64*>(sc + L.spos),
                                     reinterpret_cast<i64*>(sc + L.block_sums), LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
     }
+    if (plan->policy != SPWS_SPARSE_ISM) CUDA_TRY(launch_dense_rebin(c, (int)S.m, rowptr));
     CUDA_TRY(launch_class_nnz(c, (int)S.m));
     mark(plan, SPWS_T_SYM_SCAN);
     CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
@@ -468,6 +491,11 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
         plan->stats.nnz_per_class[k] = hc.class_nnz[k];
     }
     plan->stats.dense_units = hc.n_units;
+    plan->stats.dense_warp_rows = hc.n_warp_rows;
+    plan->stats.dense_warp_products = hc.dense_warp_products;
+    plan->stats.dense_warp_nnz = hc.dense_warp_nnz;
+    plan->stats.bitmap_bytes = (int64_t)hc.bm_words_used * 4;
+    plan->max_span_words = hc.max_span_words;
     plan->stats.launches_symbolic = c.launches;
     if (plan->kind == 0) {
         C->n[0] = C->dims[0];
@@ -518,9 +546,13 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM, (int)s.rows_per_class[CLS_ISM_SMEM], S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_ISM_SMEM);
     }
+    if (s.dense_warp_rows > 0) {
+        CUDA_TRY(launch_dense_num_warp(c, (int)s.dense_warp_rows, S.A, S.B, rowptr, crd, C->val));
+        mark(plan, SPWS_T_NUM_DENSE_WARP);
+    }
     if (s.dense_units > 0) {
-        CUDA_TRY(launch_dense(c, true, (int)s.dense_units, S.A, S.B, rowptr, crd, C->val));
-        mark(plan, SPWS_T_NUM_DENSE);
+        CUDA_TRY(launch_dense_num_cta(c, (int)s.dense_units, plan->max_span_words, S.A, S.B, rowptr, crd, C->val));
+        mark(plan, SPWS_T_NUM_DENSE_CTA);
     }
     if (s.rows_per_class[CLS_ISM_GLOBAL] > 0) {
         CUDA_TRY(launch_ism_global(c, true, (int)s.rows_per_class[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));

@@ -14,7 +14,8 @@ pytestmark = pytest.mark.gpu
 
 POLICIES = ("dense", "ism", "auto")
 # thresholds that force every route on small inputs
-SMALL_ROUTES = dict(ism_warp_cap=8, ism_cta_cap=64, dense_tile_cols=256, max_dense_tiles=4096, fallback_cap=16)
+SMALL_ROUTES = dict(ism_warp_cap=8, ism_cta_cap=64, dense_unit_outputs=64, fallback_cap=16)
+GLOBAL, DENSE = 7, slice(4, 7)          # indices into stats["rows_per_class"]
 
 
 @pytest.fixture(scope="module")
@@ -74,9 +75,9 @@ def test_random_small_all_routes(ctx, oracle_mod, policy, m, k, n, dens, seed):
     check_spgemm(ctx, oracle_mod, A, B, policy)                      # default thresholds
     stats = check_spgemm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
     if policy == "ism" and m >= 37:
-        assert stats["rows_per_class"][5] > 0                        # the global-memory ISM ran
-    if policy == "dense" and n >= 700:
-        assert stats["dense_units"] > stats["rows_per_class"][4]      # some row used several tiles
+        assert stats["rows_per_class"][GLOBAL] > 0                   # the global-memory ISM ran
+    if policy == "dense" and n >= 700:                               # some row was cut into several units
+        assert stats["dense_units"] > sum(stats["rows_per_class"][DENSE]) - stats["dense_warp_rows"]
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float64])
@@ -113,7 +114,7 @@ def test_capacity_boundaries(ctx, oracle_mod, policy):
     stats = check_spgemm(ctx, oracle_mod, A, B, policy)
     assert stats["max_row_products"] == 20000
     if policy == "ism":
-        assert stats["rows_per_class"][5] == 5                       # rows above the shared-memory capacity
+        assert stats["rows_per_class"][GLOBAL] == 5                  # rows above the shared-memory capacity
     A, B = _rows_with_products(targets[:17], 3000, 12)
     check_spgemm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
 
@@ -151,9 +152,26 @@ def test_ism_routes_reproduce_sequential_sum(ctx, oracle_mod):
     ref = oracle_mod.spgemm(A, A)
     for opts in ({}, dict(ism_warp_cap=8, ism_cta_cap=1024), dict(ism_warp_cap=16, ism_cta_cap=256)):
         pos, crd, val, stats = run_spgemm(ctx, A, A, "ism", **opts)
-        assert stats["rows_per_class"][5] == 0
+        assert stats["rows_per_class"][GLOBAL] == 0
         assert np.array_equal(pos, ref.pos) and np.array_equal(crd, ref.crd)
         assert (val != ref.val).sum() == 0
+
+
+def test_warp_dense_route_reproduces_sequential_sum(ctx, oracle_mod):
+    """With its lanes across one B row at a time, the warp-per-row dense workspace sums every
+    output in loop order.  That holds for rows whose B rows are long enough for a full-warp
+    group (here: the interior grid points, 27 x 27 products); rows with short B rows keep
+    several A entries in flight and are held to the tolerance."""
+    A = stencil27_csr(10, 3)
+    ref = oracle_mod.spgemm(A, A)
+    pos, crd, val, stats = run_spgemm(ctx, A, A, "dense")
+    assert stats["dense_warp_rows"] == A.nrows
+    assert np.array_equal(pos, ref.pos) and np.array_equal(crd, ref.crd)
+    interior = np.repeat(ref.products == 729, np.diff(ref.pos))
+    assert interior.sum() == 6 ** 3 * 125
+    assert np.array_equal(val[interior], ref.val[interior])
+    ok, _ = values_close(val, ref.val_ref, ref.abs, 1e-12)
+    assert ok.all()
 
 
 # ------------------------------------------------------------------ benchmark configurations
