@@ -238,28 +238,51 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 // ---------------------------------------------------------------------------------------
 // numeric, CTA units (row, rank range)
 // ---------------------------------------------------------------------------------------
+constexpr int DN_THREADS = 512;
+constexpr int DN_WARPS = DN_THREADS / 32;
+
 __device__ __forceinline__ int nth_set_bit(unsigned word, int nth) {   // position of the nth (0-based) set bit
     for (int x = 0; x < nth; ++x) word &= word - 1;
     return __ffs(word) - 1;
 }
 
+// First q in [lo, hi) with crd[q] >= c, found by the gs lanes of a group together: each step
+// probes gs positions at once, so a row of n entries takes about log(n)/log(gs+1) dependent
+// loads instead of log2(n).  All lanes of the group must call it with the same lo, hi, c.
+__device__ __forceinline__ i64 group_lower_bound(const int* __restrict__ crd, i64 lo, i64 hi, i64 c, int gl, int gs,
+                                                 unsigned gmask, unsigned gshift) {
+    while (lo < hi) {
+        const i64 len = hi - lo;
+        const i64 step = (len + gs) / (gs + 1);
+        const i64 mine = min(lo + (i64)(gl + 1) * step - 1, hi - 1);
+        const bool less = (i64)__ldg(crd + mine) < c;
+        const int t = __popc((__ballot_sync(gmask, less) & gmask) >> gshift);   // the first t probes are < c
+        const i64 new_lo = t > 0 ? min(lo + (i64)t * step - 1, hi - 1) + 1 : lo;
+        const i64 new_hi = t < gs ? min(lo + (i64)(t + 1) * step - 1, hi - 1) : hi;
+        lo = new_lo;
+        hi = new_hi;
+    }
+    return lo;
+}
+
 template <typename T>
-__global__ void __launch_bounds__(DC_THREADS) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, Csr A, Csr B,
+__global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, Csr A, Csr B,
                                                                    RowTables tab, const i64* __restrict__ rowptr,
                                                                    int* __restrict__ Ccrd, T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
     unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
-    short* pre = reinterpret_cast<short*>(bm + smem_words);                          // smem_words: rank of word start - r0
+    int* chunk = reinterpret_cast<int*>(bm + smem_words);                            // smem_words / 32: rank of each 32-word chunk
+    short* pre = reinterpret_cast<short*>(chunk + smem_words / 32);                  // smem_words: rank of word start - r0
     __shared__ int s_next, s_w0, s_w1;
     __shared__ i64 s_c0, s_c1;
     __shared__ int ws[33];
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
-    for (int x = tid; x < CAP; x += DC_THREADS) acc[x] = 0;
+    for (int x = tid; x < CAP; x += DN_THREADS) acc[x] = 0;
 
     for (;;) {
         __syncthreads();
@@ -279,58 +302,73 @@ __global__ void __launch_bounds__(DC_THREADS) dense_num_cta_kernel(DevCtl* __res
         const bool whole = (r0 == 0 && r1 == cnt);
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         if (tid == 0) { s_w0 = 0; s_w1 = nw - 1; s_c0 = base; s_c1 = (i64)last + 1; }
-        __syncthreads();
 
-        // bitmap + word prefix; the words holding ranks r0 and r1 give the unit's column range
+        // bitmap words + rank of every word's first bit, in three steps: per 32-word chunk by
+        // warp shuffles, chunk totals by one block scan, then the sum
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        int carry = 0;
-        for (int w0 = 0; w0 < nw; w0 += DC_THREADS) {
-            const int w = w0 + tid;
+        const int nchunks = (nw + 31) >> 5;
+        for (int c = warp; c < nchunks; c += DN_WARPS) {
+            const int w = (c << 5) + lane;
             const unsigned word = (w < nw) ? src[w] : 0u;
-            const int c = __popc(word);
-            int chunk_total;
-            const int start = carry + block_excl_scan<DC_THREADS>(c, ws, chunk_total);   // rank of the word's first bit
-            if (w < nw) {
-                bm[w] = word;
-                const int rel = start - r0;
-                pre[w] = (short)max(-32768, min(32767, rel));
-                if (start <= r0 && r0 < start + c) { s_w0 = w; s_c0 = (i64)base + (w << 5) + nth_set_bit(word, r0 - start); }
-                if (r1 < cnt && start <= r1 && r1 < start + c) { s_w1 = w; s_c1 = (i64)base + (w << 5) + nth_set_bit(word, r1 - start); }
-            }
-            carry += chunk_total;
+            const int pc = __popc(word);
+            const int incl = warp_incl_scan(pc);
+            if (w < nw) { bm[w] = word; pre[w] = (short)(incl - pc); }
+            if (lane == 31) chunk[c] = incl;
         }
         __syncthreads();
-        const i64 c0 = s_c0, c1 = s_c1;               // the unit owns columns [c0, c1)
+        {
+            const int cpt = (nchunks + DN_THREADS - 1) / DN_THREADS;
+            const int c_lo = min(nchunks, tid * cpt), c_hi = min(nchunks, c_lo + cpt);
+            int local = 0;
+            for (int c = c_lo; c < c_hi; ++c) local += chunk[c];
+            int total;
+            int run = block_excl_scan<DN_THREADS>(local, ws, total);
+            for (int c = c_lo; c < c_hi; ++c) { const int t = chunk[c]; chunk[c] = run; run += t; }
+        }
+        __syncthreads();
+        for (int w = tid; w < nw; w += DN_THREADS) {
+            const unsigned word = bm[w];
+            const int c = __popc(word);
+            const int start = chunk[w >> 5] + pre[w];
+            pre[w] = (short)max(-32768, min(32767, start - r0));
+            // the words holding ranks r0 and r1 give the unit's column range [c0, c1)
+            if (start <= r0 && r0 < start + c) { s_w0 = w; s_c0 = (i64)base + (w << 5) + nth_set_bit(word, r0 - start); }
+            if (r1 < cnt && start <= r1 && r1 < start + c) { s_w1 = w; s_c1 = (i64)base + (w << 5) + nth_set_bit(word, r1 - start); }
+        }
+        __syncthreads();
+        const i64 c0 = s_c0, c1 = s_c1;
         const unsigned lo_rel = (unsigned)(c0 - base), hi_rel = (unsigned)(c1 - base);
 
         const int nunits_row = (cnt + CAP - 1) / CAP;
         const int gs = pick_group_size(tab.ub[row] / nunits_row, pe - ps);
-        const int g = tid / gs, gl = tid % gs, ng = DC_THREADS / gs;
+        const int g = tid / gs, gl = tid % gs, ng = DN_THREADS / gs;
+        const unsigned gshift = (unsigned)(lane - gl);
+        const unsigned gmask = (gs == 32) ? 0xffffffffu : (((1u << gs) - 1u) << gshift);
         for (i64 p = ps + g; p < pe; p += ng) {
             const int k = __ldg(A.crd + p);
             if ((unsigned)k >= (unsigned)B.nrows) continue;
-            i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
-            if (!whole) {
-                qs = lower_bound_crd(B.crd, qs, qe, c0);
-                qe = lower_bound_crd(B.crd, qs, qe, c1);
-            }
+            i64 qs = __ldg(B.pos + k);
+            const i64 qe = __ldg(B.pos + k + 1);
+            if (!whole) qs = group_lower_bound(B.crd, qs, qe, c0, gl, gs, gmask, gshift);
             const T a = __ldg(Aval + p);
             i64 q = qs + gl;
             for (; q + gs < qe; q += 2 * gs) {          // two products in flight per lane
                 const unsigned rel0 = (unsigned)(__ldg(B.crd + q) - base);
                 const unsigned rel1 = (unsigned)(__ldg(B.crd + q + gs) - base);
+                if (rel0 >= hi_rel) break;              // sorted row: nothing further belongs to this unit
                 const T v0 = a * __ldg(Bval + q);
-                const T v1 = a * __ldg(Bval + q + gs);
-                if (rel0 >= lo_rel && rel0 < hi_rel) {
+                if (rel0 >= lo_rel) {
                     const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
                     if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], v0);
                 }
-                if (rel1 >= lo_rel && rel1 < hi_rel) {
+                if (rel1 >= hi_rel) break;
+                const T v1 = a * __ldg(Bval + q + gs);
+                if (rel1 >= lo_rel) {
                     const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
                     if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], v1);
                 }
             }
-            if (q < qe) {
+            if (q < qe && q + gs >= qe) {
                 const unsigned rel0 = (unsigned)(__ldg(B.crd + q) - base);
                 if (rel0 >= lo_rel && rel0 < hi_rel) {
                     const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
@@ -342,9 +380,9 @@ __global__ void __launch_bounds__(DC_THREADS) dense_num_cta_kernel(DevCtl* __res
 
         // copy out
         const i64 o0 = out0 + r0;
-        for (int x = tid; x < nout; x += DC_THREADS) { Cval[o0 + x] = acc[x]; acc[x] = 0; }
+        for (int x = tid; x < nout; x += DN_THREADS) { Cval[o0 + x] = acc[x]; acc[x] = 0; }
         const int w_first = s_w0, w_last = s_w1;
-        for (int w = w_first + tid; w <= w_last; w += DC_THREADS) {
+        for (int w = w_first + tid; w <= w_last; w += DN_THREADS) {
             unsigned word = bm[w];
             const int wp = pre[w];
             const unsigned full = word;
@@ -413,13 +451,13 @@ template <typename T>
 static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, const Csr& A, const Csr& B,
                              const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
-    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)words * 2 + 16;
+    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32) * 4 + (size_t)words * 2 + 16;
     cudaError_t e;
     int per_sm = 0;
     auto k = dense_num_cta_kernel<T>;
     if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DC_THREADS, smem)) != cudaSuccess) return e;
-    k<<<persistent_grid(c, per_sm, n_units_host), DC_THREADS, smem, c.stream>>>(c.ctl, words, CAP, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DN_THREADS, smem)) != cudaSuccess) return e;
+    k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
     ++c.launches;
     return cudaGetLastError();
 }
@@ -427,7 +465,7 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, co
 cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, const Csr& A, const Csr& B,
                                  const i64* rowptr, int* Ccrd, void* Cval) {
     int words = max_span_words > 0 ? max_span_words : c.dense_smem_words;
-    words = (words + 7) & ~7;
+    words = (words + 31) & ~31;
     return c.is_f64 ? num_cta_t<double>(c, n_units_host, words, A, B, rowptr, Ccrd, Cval)
                     : num_cta_t<float>(c, n_units_host, words, A, B, rowptr, Ccrd, Cval);
 }

@@ -167,6 +167,8 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
     __shared__ int s_hist[NCLASS], s_base[NCLASS], s_off[NCLASS];
+    __shared__ int ws[33];
+    __shared__ u64 s_bm_base;
     const int rows_per_block = blockDim.x * 4;
     if (threadIdx.x == 0) {
         int o = 0;
@@ -189,15 +191,29 @@ __global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, Cla
         if (threadIdx.x < NCLASS && s_hist[threadIdx.x])
             s_base[threadIdx.x] = atomicAdd(&ctl->class_cursor[threadIdx.x], s_hist[threadIdx.x]);
         __syncthreads();
+        // bitmap words of this thread's dense rows; one arena reservation per block
+        int words[4], my_words = 0;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const i64 row = r0 + x * blockDim.x + threadIdx.x;
+            words[x] = 0;
+            if (cls[x] == CLS_DENSE_WARP || cls[x] == CLS_DENSE_HUB || cls[x] == CLS_DENSE_CTA)
+                words[x] = (tab.jmax[row] - tab.jmin[row]) / 32 + 1;
+            my_words += words[x];
+        }
+        int block_words;
+        int my_off = block_excl_scan<256>(my_words, ws, block_words);
+        if (threadIdx.x == 0 && block_words) s_bm_base = atomicAdd(&ctl->bm_words_used, (u64)block_words);
+        __syncthreads();
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
             const i64 row = r0 + x * blockDim.x + threadIdx.x;
             if (cls[x] < 0) continue;
             tab.perm[s_off[cls[x]] + s_base[cls[x]] + rank[x]] = (int)row;
-            if (cls[x] == CLS_DENSE_WARP || cls[x] == CLS_DENSE_HUB || cls[x] == CLS_DENSE_CTA) {
-                const u64 words = (u64)((tab.jmax[row] - tab.jmin[row]) / 32 + 1);
-                const u64 at = atomicAdd(&ctl->bm_words_used, words);
-                if (at + words > prm.bm_arena_words) {
+            if (words[x]) {
+                const u64 at = s_bm_base + (u64)my_off;
+                my_off += words[x];
+                if (at + (u64)words[x] > prm.bm_arena_words) {
                     raise_status(ctl, DEV_SCRATCH_TOO_SMALL);
                     tab.bm_off[row] = -1;
                 } else {
@@ -222,30 +238,55 @@ cudaError_t launch_bin_rows(const LaunchCtx& c, int m) {
 // counted and whose outputs fit a warp's accumulator stays with a warp; every other row is cut
 // into CTA units of `unit_outputs` consecutive outputs (rank ranges).
 __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
+    __shared__ int ws[33];
+    __shared__ int s_wbase, s_ubase;
+    __shared__ i64 s_wp, s_wn;
     int off, n4, n5, n6, o5, o6;
     class_range(ctl, CLS_DENSE_WARP, off, n4);
     class_range(ctl, CLS_DENSE_HUB, o5, n5);
     class_range(ctl, CLS_DENSE_CTA, o6, n6);
     const int n = n4 + n5 + n6;                       // the three classes are adjacent in perm
-    for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += (i64)gridDim.x * blockDim.x) {
-        const int row = tab.perm[off + r];
-        const int cnt = tab.cnt[row];
-        if (tab.cls[row] == CLS_DENSE_WARP && cnt <= DENSE_WARP_ACC) {
-            tab.warp_rows[atomicAdd(&ctl->n_warp_rows, 1)] = row;
-            tab.row_unit0[row] = -1;
-            atomicAdd((u64*)&ctl->dense_warp_products, (u64)tab.ub[row]);
-            atomicAdd((u64*)&ctl->dense_warp_nnz, (u64)cnt);
-        } else {
-            const int nu = (cnt + prm.unit_outputs - 1) / prm.unit_outputs;
-            const int u0 = atomicAdd(&ctl->n_units, nu);
-            if (u0 + nu > prm.unit_cap) {
-                raise_status(ctl, DEV_SCRATCH_TOO_SMALL);
+    for (i64 b0 = (i64)blockIdx.x * blockDim.x; b0 < n; b0 += (i64)gridDim.x * blockDim.x) {
+        const i64 r = b0 + threadIdx.x;
+        int row = -1, cnt = 0, to_warp = 0, nu = 0;
+        if (threadIdx.x == 0) { s_wp = 0; s_wn = 0; }
+        if (r < n) {
+            row = tab.perm[off + r];
+            cnt = tab.cnt[row];
+            to_warp = tab.cls[row] == CLS_DENSE_WARP && cnt <= DENSE_WARP_ACC;
+            nu = to_warp ? 0 : (cnt + prm.unit_outputs - 1) / prm.unit_outputs;
+        }
+        int wtot, utot;
+        const int wpos = block_excl_scan<256>(to_warp, ws, wtot);
+        const int upos = block_excl_scan<256>(nu, ws, utot);
+        if (threadIdx.x == 0) {
+            s_wbase = wtot ? atomicAdd(&ctl->n_warp_rows, wtot) : 0;
+            s_ubase = utot ? atomicAdd(&ctl->n_units, utot) : 0;
+        }
+        __syncthreads();
+        if (row >= 0) {
+            if (to_warp) {
+                tab.warp_rows[s_wbase + wpos] = row;
                 tab.row_unit0[row] = -1;
+                atomicAdd((u64*)&s_wp, (u64)tab.ub[row]);
+                atomicAdd((u64*)&s_wn, (u64)cnt);
             } else {
-                tab.row_unit0[row] = u0;
-                for (int t = 0; t < nu; ++t) tab.unit_row[u0 + t] = row;
+                const int u0 = s_ubase + upos;
+                if (u0 + nu > prm.unit_cap) {
+                    raise_status(ctl, DEV_SCRATCH_TOO_SMALL);
+                    tab.row_unit0[row] = -1;
+                } else {
+                    tab.row_unit0[row] = u0;
+                    for (int t = 0; t < nu; ++t) tab.unit_row[u0 + t] = row;
+                }
             }
         }
+        __syncthreads();
+        if (threadIdx.x == 0 && s_wp) {
+            atomicAdd((u64*)&ctl->dense_warp_products, (u64)s_wp);
+            atomicAdd((u64*)&ctl->dense_warp_nnz, (u64)s_wn);
+        }
+        __syncthreads();
     }
 }
 
