@@ -26,13 +26,20 @@ namespace spws {
 
 constexpr int DW_THREADS = 256;            // warp-per-row kernels: 8 warps per CTA
 constexpr int DW_WARPS = DW_THREADS / 32;
-constexpr int DC_THREADS = 256;            // CTA kernels
+constexpr int DC_THREADS = 256;            // symbolic CTA kernel
+constexpr int DC_WARPS = DC_THREADS / 32;
+constexpr int DN_THREADS = 512;            // numeric CTA kernel
+constexpr int DN_WARPS = DN_THREADS / 32;
 
-__device__ __forceinline__ int pick_group_size(i64 ub, i64 entries) {
-    // lanes per A entry: the smallest power of two >= the mean B-row segment length
-    const i64 avg = ub / (entries > 0 ? entries : 1);
+// A dense row's slot in the arena: nw bitmap words, then for every chunk of 32 words the rank of
+// the chunk's first bit (an exclusive prefix of the chunk popcounts).
+__device__ __forceinline__ int chunks_of(int nw) { return (nw + 31) >> 5; }
+
+// lanes per A entry: the smallest power of two >= the mean B-row segment length
+__device__ __forceinline__ int pick_group_size(i64 ub, i64 entries, int parts) {
+    const float avg = (float)ub / fmaxf(1.0f, (float)entries * (float)parts);
     int gs = 32;
-    while (gs > 1 && (gs >> 1) >= avg) gs >>= 1;
+    while (gs > 1 && (float)(gs >> 1) >= avg) gs >>= 1;
     return gs;
 }
 
@@ -58,27 +65,32 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         for (int w = lane; w < nw; w += 32) bm[w] = 0;
         __syncwarp();
-        const int gs = pick_group_size(tab.ub[row], pe - ps);
+        const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
         const int g = lane / gs, gl = lane % gs, ng = 32 / gs;
         for (i64 p = ps + g; p < pe; p += ng) {
             const int k = __ldg(A.crd + p);
             if ((unsigned)k >= (unsigned)B.nrows) continue;
-            const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
-            for (i64 q = qs + gl; q < qe; q += gs) {
-                const unsigned rel = (unsigned)(__ldg(B.crd + q) - base);
+            const i64 qs = __ldg(B.pos + k);
+            const int len = (int)(__ldg(B.pos + k + 1) - qs);
+            const int* __restrict__ ck = B.crd + qs;
+            for (int t = gl; t < len; t += gs) {
+                const unsigned rel = (unsigned)(__ldg(ck + t) - base);
                 if (rel < span) atomicOr(&bm[rel >> 5], 1u << (rel & 31));
             }
         }
         __syncwarp();
         unsigned* out = tab.bm_arena + tab.bm_off[row];
-        int c = 0;
-        for (int w = lane; w < nw; w += 32) {
-            const unsigned word = bm[w];
-            c += __popc(word);
-            out[w] = word;
+        int carry = 0;
+        for (int w0 = 0; w0 < nw; w0 += 32) {
+            const int w = w0 + lane;
+            const unsigned word = (w < nw) ? bm[w] : 0u;
+            if (w < nw) out[w] = word;
+            int c = __popc(word);
+            for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
+            if (lane == 0) out[nw + (w0 >> 5)] = (unsigned)carry;
+            carry += c;
         }
-        for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
-        if (lane == 0) tab.cnt[row] = c;
+        if (lane == 0) tab.cnt[row] = carry;
         __syncwarp();
     }
 }
@@ -88,7 +100,8 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, Csr A, Csr B, RowTables tab) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned* bm = reinterpret_cast<unsigned*>(smem_raw);
+    unsigned* bm = reinterpret_cast<unsigned*>(smem_raw);                 // smem_words
+    int* chunk = reinterpret_cast<int*>(bm + smem_words);                  // smem_words / 32
     __shared__ int s_next;
     __shared__ int ws[33];
     if (ctl->status != 0) return;
@@ -96,7 +109,7 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
     class_range(ctl, CLS_DENSE_HUB, off, n_hub);
     class_range(ctl, CLS_DENSE_CTA, o6, n_cta);
     const int n = n_hub + n_cta;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (;;) {
         __syncthreads();
         if (tid == 0) s_next = atomicAdd(&ctl->work_counter[CLS_DENSE_CTA], 1);
@@ -110,34 +123,50 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         for (int w = tid; w < nw; w += DC_THREADS) bm[w] = 0;
         __syncthreads();
-        const int gs = pick_group_size(tab.ub[row], pe - ps);
+        const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
         const int g = tid / gs, gl = tid % gs, ng = DC_THREADS / gs;
         for (i64 p = ps + g; p < pe; p += ng) {
             const int k = __ldg(A.crd + p);
             if ((unsigned)k >= (unsigned)B.nrows) continue;
-            const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
-            i64 q = qs + gl;
-            for (; q + gs < qe; q += 2 * gs) {          // two loads in flight per lane
-                const unsigned r0 = (unsigned)(__ldg(B.crd + q) - base);
-                const unsigned r1 = (unsigned)(__ldg(B.crd + q + gs) - base);
+            const i64 qs = __ldg(B.pos + k);
+            const int len = (int)(__ldg(B.pos + k + 1) - qs);
+            const int* __restrict__ ck = B.crd + qs;
+            int t = gl;
+            for (; t + 3 * gs < len; t += 4 * gs) {     // four loads in flight per lane
+                const unsigned r0 = (unsigned)(__ldg(ck + t) - base);
+                const unsigned r1 = (unsigned)(__ldg(ck + t + gs) - base);
+                const unsigned r2 = (unsigned)(__ldg(ck + t + 2 * gs) - base);
+                const unsigned r3 = (unsigned)(__ldg(ck + t + 3 * gs) - base);
                 if (r0 < span) atomicOr(&bm[r0 >> 5], 1u << (r0 & 31));
                 if (r1 < span) atomicOr(&bm[r1 >> 5], 1u << (r1 & 31));
+                if (r2 < span) atomicOr(&bm[r2 >> 5], 1u << (r2 & 31));
+                if (r3 < span) atomicOr(&bm[r3 >> 5], 1u << (r3 & 31));
             }
-            if (q < qe) {
-                const unsigned r0 = (unsigned)(__ldg(B.crd + q) - base);
+            for (; t < len; t += gs) {
+                const unsigned r0 = (unsigned)(__ldg(ck + t) - base);
                 if (r0 < span) atomicOr(&bm[r0 >> 5], 1u << (r0 & 31));
             }
         }
         __syncthreads();
+        // save the bitmap, then the rank at every chunk start
         unsigned* out = tab.bm_arena + tab.bm_off[row];
-        int c = 0;
-        for (int w = tid; w < nw; w += DC_THREADS) {
-            const unsigned word = bm[w];
-            c += __popc(word);
-            out[w] = word;
+        const int nch = chunks_of(nw);
+        for (int c = warp; c < nch; c += DC_WARPS) {
+            const int w = (c << 5) + lane;
+            const unsigned word = (w < nw) ? bm[w] : 0u;
+            if (w < nw) out[w] = word;
+            int pc = __popc(word);
+            for (int d = 16; d > 0; d >>= 1) pc += __shfl_xor_sync(0xffffffffu, pc, d);
+            if (lane == 0) chunk[c] = pc;
         }
+        __syncthreads();
+        const int cpt = (nch + DC_THREADS - 1) / DC_THREADS;
+        const int c_lo = min(nch, tid * cpt), c_hi = min(nch, c_lo + cpt);
+        int local = 0;
+        for (int c = c_lo; c < c_hi; ++c) local += chunk[c];
         int total;
-        block_excl_scan<DC_THREADS>(c, ws, total);
+        int run = block_excl_scan<DC_THREADS>(local, ws, total);
+        for (int c = c_lo; c < c_hi; ++c) { out[nw + c] = (unsigned)run; run += chunk[c]; }
         if (tid == 0) tab.cnt[row] = total;
     }
 }
@@ -171,33 +200,32 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const i64 out0 = rowptr[row];
         const int cnt = (int)(rowptr[row + 1] - out0);
-        // reload the bitmap and prefix-sum its words (rank of each word's first bit)
+        // reload the bitmap; rank of each word's first bit = chunk rank + prefix inside the chunk
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        int carry = 0;
         for (int w0 = 0; w0 < nw; w0 += 32) {
             const int w = w0 + lane;
             const unsigned word = (w < nw) ? src[w] : 0u;
             const int c = __popc(word);
             const int incl = warp_incl_scan(c);
-            if (w < nw) { bm[w] = word; pre[w] = (unsigned short)(carry + incl - c); }
-            carry += __shfl_sync(0xffffffffu, incl, 31);
+            if (w < nw) { bm[w] = word; pre[w] = (unsigned short)((int)src[nw + (w0 >> 5)] + incl - c); }
         }
         for (int x = lane; x < cnt; x += 32) acc[x] = 0;
         __syncwarp();
-        const int gs = pick_group_size(tab.ub[row], pe - ps);
+        const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
         if (gs == 32) {
             // one A entry at a time, lanes across its B row: distinct columns, no atomics,
             // every output summed in loop order
             for (i64 p = ps; p < pe; ++p) {
                 const int k = __ldg(A.crd + p);
                 if ((unsigned)k >= (unsigned)B.nrows) continue;
-                const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                const i64 qs = __ldg(B.pos + k);
+                const int len = (int)(__ldg(B.pos + k + 1) - qs);
                 const T a = __ldg(Aval + p);
-                for (i64 q = qs + lane; q < qe; q += 32) {
-                    const unsigned rel = (unsigned)(__ldg(B.crd + q) - base);
+                for (int t = lane; t < len; t += 32) {
+                    const unsigned rel = (unsigned)(__ldg(B.crd + qs + t) - base);
                     if (rel < span) {
                         const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a, __ldg(Bval + q)));
+                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a, __ldg(Bval + qs + t)));
                     }
                 }
                 __syncwarp();
@@ -208,13 +236,14 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
             for (i64 p = ps + g; p < pe; p += ng) {
                 const int k = __ldg(A.crd + p);
                 if ((unsigned)k >= (unsigned)B.nrows) continue;
-                const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                const i64 qs = __ldg(B.pos + k);
+                const int len = (int)(__ldg(B.pos + k + 1) - qs);
                 const T a = __ldg(Aval + p);
-                for (i64 q = qs + gl; q < qe; q += gs) {
-                    const unsigned rel = (unsigned)(__ldg(B.crd + q) - base);
+                for (int t = gl; t < len; t += gs) {
+                    const unsigned rel = (unsigned)(__ldg(B.crd + qs + t) - base);
                     if (rel < span) {
                         const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                        if (slot < DENSE_WARP_ACC) atomicAdd(&acc[slot], mul_rn(a, __ldg(Bval + q)));
+                        if (slot < DENSE_WARP_ACC) atomicAdd(&acc[slot], mul_rn(a, __ldg(Bval + qs + t)));
                     }
                 }
             }
@@ -238,27 +267,25 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 // ---------------------------------------------------------------------------------------
 // numeric, CTA units (row, rank range)
 // ---------------------------------------------------------------------------------------
-constexpr int DN_THREADS = 512;
-constexpr int DN_WARPS = DN_THREADS / 32;
-
 __device__ __forceinline__ int nth_set_bit(unsigned word, int nth) {   // position of the nth (0-based) set bit
     for (int x = 0; x < nth; ++x) word &= word - 1;
     return __ffs(word) - 1;
 }
 
-// First q in [lo, hi) with crd[q] >= c, found by the gs lanes of a group together: each step
-// probes gs positions at once, so a row of n entries takes about log(n)/log(gs+1) dependent
-// loads instead of log2(n).  All lanes of the group must call it with the same lo, hi, c.
-__device__ __forceinline__ i64 group_lower_bound(const int* __restrict__ crd, i64 lo, i64 hi, i64 c, int gl, int gs,
+// First t in [0, len) with ck[t] >= c, found by the gs lanes of a group together: each step
+// probes gs positions at once, so a row of n entries takes about log(n)/log(gs) dependent loads
+// instead of log2(n).  All lanes of the group must call it with the same arguments.
+__device__ __forceinline__ int group_lower_bound(const int* __restrict__ ck, int len, int c, int gl, int gs, int lg,
                                                  unsigned gmask, unsigned gshift) {
+    int lo = 0, hi = len;
     while (lo < hi) {
-        const i64 len = hi - lo;
-        const i64 step = (len + gs) / (gs + 1);
-        const i64 mine = min(lo + (i64)(gl + 1) * step - 1, hi - 1);
-        const bool less = (i64)__ldg(crd + mine) < c;
+        const int n = hi - lo;
+        const int step = (gs == 1) ? ((n + 1) >> 1) : ((n + gs - 1) >> lg);
+        const int mine = min(lo + (gl + 1) * step - 1, hi - 1);
+        const bool less = __ldg(ck + mine) < c;
         const int t = __popc((__ballot_sync(gmask, less) & gmask) >> gshift);   // the first t probes are < c
-        const i64 new_lo = t > 0 ? min(lo + (i64)t * step - 1, hi - 1) + 1 : lo;
-        const i64 new_hi = t < gs ? min(lo + (i64)(t + 1) * step - 1, hi - 1) : hi;
+        const int new_lo = t > 0 ? min(lo + t * step - 1, hi - 1) + 1 : lo;
+        const int new_hi = t < gs ? min(lo + (t + 1) * step - 1, hi - 1) : hi;
         lo = new_lo;
         hi = new_hi;
     }
@@ -272,11 +299,8 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
     unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
-    int* chunk = reinterpret_cast<int*>(bm + smem_words);                            // smem_words / 32: rank of each 32-word chunk
-    short* pre = reinterpret_cast<short*>(chunk + smem_words / 32);                  // smem_words: rank of word start - r0
-    __shared__ int s_next, s_w0, s_w1;
-    __shared__ i64 s_c0, s_c1;
-    __shared__ int ws[33];
+    short* pre = reinterpret_cast<short*>(bm + smem_words);                          // smem_words: rank of word start - r0
+    __shared__ int s_next, s_ca, s_cb, s_w0, s_w1, s_c0, s_c1, s_entry;
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -294,6 +318,7 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
         const int uidx = u - tab.row_unit0[row];
         const int base = tab.jmin[row], last = tab.jmax[row];
         const int nw = min((last - base) / 32 + 1, smem_words);
+        const int nch = chunks_of(nw);
         const i64 out0 = rowptr[row];
         const int cnt = (int)(rowptr[row + 1] - out0);
         const int r0 = uidx * CAP;
@@ -301,80 +326,82 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
         const int r1 = r0 + nout;
         const bool whole = (r0 == 0 && r1 == cnt);
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
-        if (tid == 0) { s_w0 = 0; s_w1 = nw - 1; s_c0 = base; s_c1 = (i64)last + 1; }
-
-        // bitmap words + rank of every word's first bit, in three steps: per 32-word chunk by
-        // warp shuffles, chunk totals by one block scan, then the sum
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        const int nchunks = (nw + 31) >> 5;
-        for (int c = warp; c < nchunks; c += DN_WARPS) {
+        const int* cpre = reinterpret_cast<const int*>(src + nw);      // rank at every chunk start
+        if (tid == 0) { s_ca = 0; s_cb = nch - 1; s_w0 = 0; s_w1 = nw - 1; s_c0 = 0; s_c1 = last - base + 1; s_entry = 0; }
+        __syncthreads();
+        // the chunks that hold ranks r0 and r1 bound the part of the bitmap this unit needs
+        if (!whole) {
+            for (int c = tid; c < nch; c += DN_THREADS) {
+                const int lo = cpre[c], hi = (c + 1 < nch) ? cpre[c + 1] : cnt;
+                if (lo <= r0 && r0 < hi) s_ca = c;
+                if (r1 < cnt && lo <= r1 && r1 < hi) s_cb = c;
+            }
+            __syncthreads();
+        }
+        const int ca = s_ca, cb = s_cb;
+        for (int c = ca + warp; c <= cb; c += DN_WARPS) {
             const int w = (c << 5) + lane;
             const unsigned word = (w < nw) ? src[w] : 0u;
             const int pc = __popc(word);
-            const int incl = warp_incl_scan(pc);
-            if (w < nw) { bm[w] = word; pre[w] = (short)(incl - pc); }
-            if (lane == 31) chunk[c] = incl;
+            const int start = cpre[c] + warp_incl_scan(pc) - pc;       // rank of this word's first bit
+            if (w < nw) {
+                bm[w] = word;
+                pre[w] = (short)max(-32768, min(32767, start - r0));
+                if (start <= r0 && r0 < start + pc) { s_w0 = w; s_c0 = (w << 5) + nth_set_bit(word, r0 - start); }
+                if (r1 < cnt && start <= r1 && r1 < start + pc) { s_w1 = w; s_c1 = (w << 5) + nth_set_bit(word, r1 - start); }
+            }
         }
         __syncthreads();
-        {
-            const int cpt = (nchunks + DN_THREADS - 1) / DN_THREADS;
-            const int c_lo = min(nchunks, tid * cpt), c_hi = min(nchunks, c_lo + cpt);
-            int local = 0;
-            for (int c = c_lo; c < c_hi; ++c) local += chunk[c];
-            int total;
-            int run = block_excl_scan<DN_THREADS>(local, ws, total);
-            for (int c = c_lo; c < c_hi; ++c) { const int t = chunk[c]; chunk[c] = run; run += t; }
-        }
-        __syncthreads();
-        for (int w = tid; w < nw; w += DN_THREADS) {
-            const unsigned word = bm[w];
-            const int c = __popc(word);
-            const int start = chunk[w >> 5] + pre[w];
-            pre[w] = (short)max(-32768, min(32767, start - r0));
-            // the words holding ranks r0 and r1 give the unit's column range [c0, c1)
-            if (start <= r0 && r0 < start + c) { s_w0 = w; s_c0 = (i64)base + (w << 5) + nth_set_bit(word, r0 - start); }
-            if (r1 < cnt && start <= r1 && r1 < start + c) { s_w1 = w; s_c1 = (i64)base + (w << 5) + nth_set_bit(word, r1 - start); }
-        }
-        __syncthreads();
-        const i64 c0 = s_c0, c1 = s_c1;
-        const unsigned lo_rel = (unsigned)(c0 - base), hi_rel = (unsigned)(c1 - base);
+        // the unit owns the columns base + [lo_rel, hi_rel)
+        const unsigned lo_rel = (unsigned)s_c0, hi_rel = (unsigned)s_c1;
+        const int c_lo_abs = base + (int)lo_rel;
 
-        const int nunits_row = (cnt + CAP - 1) / CAP;
-        const int gs = pick_group_size(tab.ub[row] / nunits_row, pe - ps);
-        const int g = tid / gs, gl = tid % gs, ng = DN_THREADS / gs;
+        const int gs = pick_group_size(tab.ub[row], pe - ps, (cnt + CAP - 1) / CAP);
+        const int lg = __ffs(gs) - 1;
+        const int gl = tid & (gs - 1), ng = DN_THREADS >> lg;
         const unsigned gshift = (unsigned)(lane - gl);
         const unsigned gmask = (gs == 32) ? 0xffffffffu : (((1u << gs) - 1u) << gshift);
-        for (i64 p = ps + g; p < pe; p += ng) {
+        const bool dynamic = gs >= 8;                   // long segments: groups pull entries as they finish
+        i64 p = ps + (tid >> lg);
+        for (;;) {
+            if (dynamic) {
+                int e = 0;
+                if (gl == 0) e = atomicAdd(&s_entry, 1);
+                e = __shfl_sync(gmask, e, (int)gshift);
+                p = ps + e;
+            }
+            if (p >= pe) break;
             const int k = __ldg(A.crd + p);
-            if ((unsigned)k >= (unsigned)B.nrows) continue;
-            i64 qs = __ldg(B.pos + k);
-            const i64 qe = __ldg(B.pos + k + 1);
-            if (!whole) qs = group_lower_bound(B.crd, qs, qe, c0, gl, gs, gmask, gshift);
-            const T a = __ldg(Aval + p);
-            i64 q = qs + gl;
-            for (; q + gs < qe; q += 2 * gs) {          // two products in flight per lane
-                const unsigned rel0 = (unsigned)(__ldg(B.crd + q) - base);
-                const unsigned rel1 = (unsigned)(__ldg(B.crd + q + gs) - base);
-                if (rel0 >= hi_rel) break;              // sorted row: nothing further belongs to this unit
-                const T v0 = a * __ldg(Bval + q);
-                if (rel0 >= lo_rel) {
-                    const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                    if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], v0);
-                }
-                if (rel1 >= hi_rel) break;
-                const T v1 = a * __ldg(Bval + q + gs);
-                if (rel1 >= lo_rel) {
-                    const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
-                    if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], v1);
+            if ((unsigned)k < (unsigned)B.nrows) {
+                const i64 qs = __ldg(B.pos + k);
+                const int len = (int)(__ldg(B.pos + k + 1) - qs);
+                const int* __restrict__ ck = B.crd + qs;
+                const T* __restrict__ vk = Bval + qs;
+                const T a = __ldg(Aval + p);
+                int t = gl;
+                if (!whole) t += group_lower_bound(ck, len, c_lo_abs, gl, gs, lg, gmask, gshift);
+                while (t < len) {                       // two products in flight per lane
+                    const int t2 = t + gs;
+                    const bool two = t2 < len;
+                    const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
+                    const unsigned rel1 = two ? (unsigned)(__ldg(ck + t2) - base) : 0xffffffffu;
+                    const T v0 = __ldg(vk + t);
+                    const T v1 = two ? __ldg(vk + t2) : (T)0;
+                    if (rel0 >= hi_rel) break;          // sorted row: nothing further belongs to this unit
+                    {
+                        const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                        if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v0);
+                    }
+                    if (rel1 >= hi_rel) break;
+                    {
+                        const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
+                        if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v1);
+                    }
+                    t = t2 + gs;
                 }
             }
-            if (q < qe && q + gs >= qe) {
-                const unsigned rel0 = (unsigned)(__ldg(B.crd + q) - base);
-                if (rel0 >= lo_rel && rel0 < hi_rel) {
-                    const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                    if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * __ldg(Bval + q));
-                }
-            }
+            if (!dynamic) p += ng;
         }
         __syncthreads();
 
@@ -418,7 +445,7 @@ cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B
 }
 
 cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B) {
-    const size_t smem = (size_t)c.dense_smem_words * 4;
+    const size_t smem = (size_t)c.dense_smem_words * 4 + (size_t)(c.dense_smem_words / 32 + 1) * 4;
     cudaError_t e;
     int per_sm = 0;
     if ((e = cudaFuncSetAttribute(dense_sym_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
@@ -451,7 +478,7 @@ template <typename T>
 static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, const Csr& A, const Csr& B,
                              const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
-    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32) * 4 + (size_t)words * 2 + 16;
+    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)words * 2 + 16;
     cudaError_t e;
     int per_sm = 0;
     auto k = dense_num_cta_kernel<T>;

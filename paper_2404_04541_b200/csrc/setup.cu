@@ -198,7 +198,10 @@ __global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, Cla
             const i64 row = r0 + x * blockDim.x + threadIdx.x;
             words[x] = 0;
             if (cls[x] == CLS_DENSE_WARP || cls[x] == CLS_DENSE_HUB || cls[x] == CLS_DENSE_CTA)
-                words[x] = (tab.jmax[row] - tab.jmin[row]) / 32 + 1;
+            {   // the row's slot: bitmap words, then the rank at the start of every 32-word chunk
+                const int nw = (tab.jmax[row] - tab.jmin[row]) / 32 + 1;
+                words[x] = nw + (nw + 31) / 32;
+            }
             my_words += words[x];
         }
         int block_words;

@@ -164,7 +164,8 @@ size_t rest_reserve(const spws_plan_s* p, int64_t m, int64_t ncols) {
     size_t bytes = 0;
     if (p->policy != SPWS_SPARSE_ISM) {
         const int64_t span_cap = ncols < p->opt.dense_max_span ? ncols : p->opt.dense_max_span;
-        bytes += align256((size_t)m * (size_t)((span_cap + 31) / 32 + 1) * 4);
+        const size_t nw = (size_t)((span_cap + 31) / 32 + 1);
+        bytes += align256((size_t)m * (nw + (nw + 31) / 32) * 4);
     }
     if (p->policy != SPWS_DENSE) {
         const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
