@@ -215,20 +215,57 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         if (gs == 32) {
             // one A entry at a time, lanes across its B row: distinct columns, no atomics,
             // every output summed in loop order
-            for (i64 p = ps; p < pe; ++p) {
-                const int k = __ldg(A.crd + p);
-                if ((unsigned)k >= (unsigned)B.nrows) continue;
-                const i64 qs = __ldg(B.pos + k);
-                const int len = (int)(__ldg(B.pos + k + 1) - qs);
-                const T a = __ldg(Aval + p);
-                for (int t = lane; t < len; t += 32) {
-                    const unsigned rel = (unsigned)(__ldg(B.crd + qs + t) - base);
-                    if (rel < span) {
-                        const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a, __ldg(Bval + qs + t)));
+            // (the entries' descriptors are fetched 32 at a time, one per lane, and the first 32
+            // elements of two B rows are loaded before either is consumed, to keep loads in flight)
+            for (i64 p0 = ps; p0 < pe; p0 += 32) {
+                i64 my_qs = 0;
+                int my_len = 0;
+                T my_a = 0;
+                if (p0 + lane < pe) {
+                    const int k = __ldg(A.crd + p0 + lane);
+                    if ((unsigned)k < (unsigned)B.nrows) {
+                        my_qs = __ldg(B.pos + k);
+                        my_len = (int)(__ldg(B.pos + k + 1) - my_qs);
                     }
+                    my_a = __ldg(Aval + p0 + lane);
                 }
-                __syncwarp();
+                const int nE = (int)min((i64)32, pe - p0);
+                for (int e = 0; e < nE; e += 2) {
+                    const i64 qs0 = __shfl_sync(0xffffffffu, my_qs, e), qs1 = __shfl_sync(0xffffffffu, my_qs, (e + 1) & 31);
+                    const int len0 = __shfl_sync(0xffffffffu, my_len, e);
+                    const int len1 = (e + 1 < nE) ? __shfl_sync(0xffffffffu, my_len, (e + 1) & 31) : 0;
+                    const T a0 = __shfl_sync(0xffffffffu, my_a, e), a1 = __shfl_sync(0xffffffffu, my_a, (e + 1) & 31);
+                    unsigned rel0 = 0xffffffffu, rel1 = 0xffffffffu;
+                    T v0 = 0, v1 = 0;
+                    if (lane < len0) { rel0 = (unsigned)(__ldg(B.crd + qs0 + lane) - base); v0 = __ldg(Bval + qs0 + lane); }
+                    if (lane < len1) { rel1 = (unsigned)(__ldg(B.crd + qs1 + lane) - base); v1 = __ldg(Bval + qs1 + lane); }
+                    // entry e
+                    if (rel0 < span) {
+                        const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a0, v0));
+                    }
+                    for (int t = lane + 32; t < len0; t += 32) {
+                        const unsigned rel = (unsigned)(__ldg(B.crd + qs0 + t) - base);
+                        if (rel < span) {
+                            const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
+                            if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a0, __ldg(Bval + qs0 + t)));
+                        }
+                    }
+                    __syncwarp();
+                    // entry e + 1
+                    if (rel1 < span) {
+                        const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
+                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a1, v1));
+                    }
+                    for (int t = lane + 32; t < len1; t += 32) {
+                        const unsigned rel = (unsigned)(__ldg(B.crd + qs1 + t) - base);
+                        if (rel < span) {
+                            const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
+                            if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a1, __ldg(Bval + qs1 + t)));
+                        }
+                    }
+                    __syncwarp();
+                }
             }
         } else {
             // short B rows: several A entries in flight, so slots can collide -> atomics
@@ -272,25 +309,18 @@ __device__ __forceinline__ int nth_set_bit(unsigned word, int nth) {   // positi
     return __ffs(word) - 1;
 }
 
-// First t in [0, len) with ck[t] >= c, found by the gs lanes of a group together: each step
-// probes gs positions at once, so a row of n entries takes about log(n)/log(gs) dependent loads
-// instead of log2(n).  All lanes of the group must call it with the same arguments.
-__device__ __forceinline__ int group_lower_bound(const int* __restrict__ ck, int len, int c, int gl, int gs, int lg,
-                                                 unsigned gmask, unsigned gshift) {
-    int lo = 0, hi = len;
+// Plain lower bound by one lane (all lanes of a warp search different rows at once).
+__device__ __forceinline__ int lane_lower_bound(const int* __restrict__ ck, int lo, int hi, int c) {
     while (lo < hi) {
-        const int n = hi - lo;
-        const int step = (gs == 1) ? ((n + 1) >> 1) : ((n + gs - 1) >> lg);
-        const int mine = min(lo + (gl + 1) * step - 1, hi - 1);
-        const bool less = __ldg(ck + mine) < c;
-        const int t = __popc((__ballot_sync(gmask, less) & gmask) >> gshift);   // the first t probes are < c
-        const int new_lo = t > 0 ? min(lo + t * step - 1, hi - 1) + 1 : lo;
-        const int new_hi = t < gs ? min(lo + (t + 1) * step - 1, hi - 1) : hi;
-        lo = new_lo;
-        hi = new_hi;
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(ck + mid) < c) lo = mid + 1; else hi = mid;
     }
     return lo;
 }
+
+constexpr int DN_ENTRIES = 1024;     // A entries examined per round
+constexpr int DN_LONG = 2048;        // segments at least this long are walked by the whole CTA
+constexpr int DN_LONG_CAP = 32;
 
 template <typename T>
 __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, Csr A, Csr B,
@@ -298,9 +328,13 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
                                                                    int* __restrict__ Ccrd, T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
-    unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
+    T* item_a = acc + CAP;                                                           // DN_ENTRIES
+    i64* item_q = reinterpret_cast<i64*>(item_a + DN_ENTRIES);                       // DN_ENTRIES
+    int* item_len = reinterpret_cast<int*>(item_q + DN_ENTRIES);                     // DN_ENTRIES
+    unsigned* bm = reinterpret_cast<unsigned*>(item_len + DN_ENTRIES);               // smem_words
     short* pre = reinterpret_cast<short*>(bm + smem_words);                          // smem_words: rank of word start - r0
-    __shared__ int s_next, s_ca, s_cb, s_w0, s_w1, s_c0, s_c1, s_entry;
+    __shared__ int s_next, s_ca, s_cb, s_w0, s_w1, s_c0, s_c1, s_items, s_fetch, s_nlong, s_sumlen;
+    __shared__ int s_long[DN_LONG_CAP];
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -328,7 +362,7 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
         const int* cpre = reinterpret_cast<const int*>(src + nw);      // rank at every chunk start
-        if (tid == 0) { s_ca = 0; s_cb = nch - 1; s_w0 = 0; s_w1 = nw - 1; s_c0 = 0; s_c1 = last - base + 1; s_entry = 0; }
+        if (tid == 0) { s_ca = 0; s_cb = nch - 1; s_w0 = 0; s_w1 = nw - 1; s_c0 = 0; s_c1 = last - base + 1; }
         __syncthreads();
         // the chunks that hold ranks r0 and r1 bound the part of the bitmap this unit needs
         if (!whole) {
@@ -355,55 +389,104 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
         __syncthreads();
         // the unit owns the columns base + [lo_rel, hi_rel)
         const unsigned lo_rel = (unsigned)s_c0, hi_rel = (unsigned)s_c1;
-        const int c_lo_abs = base + (int)lo_rel;
+        const int c_lo_abs = base + (int)lo_rel, c_hi_abs = base + (int)hi_rel;
+        const unsigned span_bits = (unsigned)nw * 32u;
 
-        const int gs = pick_group_size(tab.ub[row], pe - ps, (cnt + CAP - 1) / CAP);
-        const int lg = __ffs(gs) - 1;
-        const int gl = tid & (gs - 1), ng = DN_THREADS >> lg;
-        const unsigned gshift = (unsigned)(lane - gl);
-        const unsigned gmask = (gs == 32) ? 0xffffffffu : (((1u << gs) - 1u) << gshift);
-        const bool dynamic = gs >= 8;                   // long segments: groups pull entries as they finish
-        i64 p = ps + (tid >> lg);
-        for (;;) {
-            if (dynamic) {
-                int e = 0;
-                if (gl == 0) e = atomicAdd(&s_entry, 1);
-                e = __shfl_sync(gmask, e, (int)gshift);
-                p = ps + e;
-            }
-            if (p >= pe) break;
-            const int k = __ldg(A.crd + p);
-            if ((unsigned)k < (unsigned)B.nrows) {
+        for (i64 e0 = ps; e0 < pe; e0 += DN_ENTRIES) {
+            // ---- round, step 1: one lane per A entry finds the entry's B-row segment inside the
+            // unit's column range; non-empty segments are appended to the item list
+            if (tid == 0) { s_items = 0; s_fetch = 0; s_nlong = 0; s_sumlen = 0; }
+            __syncthreads();
+            const i64 e1 = min(pe, e0 + DN_ENTRIES);
+            for (i64 p = e0 + tid; p < e1; p += DN_THREADS) {
+                const int k = __ldg(A.crd + p);
+                if ((unsigned)k >= (unsigned)B.nrows) continue;
                 const i64 qs = __ldg(B.pos + k);
                 const int len = (int)(__ldg(B.pos + k + 1) - qs);
-                const int* __restrict__ ck = B.crd + qs;
-                const T* __restrict__ vk = Bval + qs;
-                const T a = __ldg(Aval + p);
-                int t = gl;
-                if (!whole) t += group_lower_bound(ck, len, c_lo_abs, gl, gs, lg, gmask, gshift);
-                while (t < len) {                       // two products in flight per lane
-                    const int t2 = t + gs;
-                    const bool two = t2 < len;
-                    const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                    const unsigned rel1 = two ? (unsigned)(__ldg(ck + t2) - base) : 0xffffffffu;
-                    const T v0 = __ldg(vk + t);
-                    const T v1 = two ? __ldg(vk + t2) : (T)0;
-                    if (rel0 >= hi_rel) break;          // sorted row: nothing further belongs to this unit
-                    {
-                        const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                        if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v0);
+                int s0 = 0, s1 = len;
+                if (!whole && len > 0) {
+                    const int* __restrict__ ck = B.crd + qs;
+                    s0 = lane_lower_bound(ck, 0, len, c_lo_abs);
+                    s1 = lane_lower_bound(ck, s0, len, c_hi_abs);
+                }
+                if (s1 > s0) {
+                    const int i = atomicAdd(&s_items, 1);
+                    item_q[i] = qs + s0;
+                    item_len[i] = s1 - s0;
+                    item_a[i] = __ldg(Aval + p);
+                    atomicAdd(&s_sumlen, s1 - s0);
+                    if (s1 - s0 >= DN_LONG) {
+                        const int l = atomicAdd(&s_nlong, 1);
+                        if (l < DN_LONG_CAP) { s_long[l] = i; item_len[i] = -(s1 - s0); }   // negative: taken by the CTA-wide pass
                     }
-                    if (rel1 >= hi_rel) break;
-                    {
-                        const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
-                        if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v1);
-                    }
-                    t = t2 + gs;
                 }
             }
-            if (!dynamic) p += ng;
+            __syncthreads();
+            // ---- step 2: lane groups pull items; group size ~ mean segment length
+            const int n_items = s_items;
+            int gs = 32;
+            {
+                const float avg = (float)s_sumlen / fmaxf(1.0f, (float)n_items);
+                while (gs > 1 && (float)(gs >> 1) >= avg) gs >>= 1;
+            }
+            const int lg = __ffs(gs) - 1;
+            const int gl = tid & (gs - 1);
+            const unsigned gshift = (unsigned)(lane - gl);
+            const unsigned gmask = (gs == 32) ? 0xffffffffu : (((1u << gs) - 1u) << gshift);
+            const int batch = gs >= 8 ? 1 : (8 >> lg);          // items a group takes per fetch
+            for (;;) {
+                int i0 = 0;
+                if (gl == 0) i0 = atomicAdd(&s_fetch, batch);
+                i0 = __shfl_sync(gmask, i0, (int)gshift);
+                if (i0 >= n_items) break;
+                const int i1 = min(n_items, i0 + batch);
+                for (int i = i0; i < i1; ++i) {
+                    const int len = item_len[i];
+                    if (len < 0) continue;
+                    const int* __restrict__ ck = B.crd + item_q[i];
+                    const T* __restrict__ vk = Bval + item_q[i];
+                    const T a = item_a[i];
+                    int t = gl;
+                    for (; t + gs < len; t += 2 * gs) {         // two products in flight per lane
+                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
+                        const unsigned rel1 = (unsigned)(__ldg(ck + t + gs) - base);
+                        const T v0 = __ldg(vk + t), v1 = __ldg(vk + t + gs);
+                        if (rel0 < span_bits) {
+                            const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                            if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v0);
+                        }
+                        if (rel1 < span_bits) {
+                            const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
+                            if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v1);
+                        }
+                    }
+                    if (t < len) {
+                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
+                        if (rel0 < span_bits) {
+                            const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                            if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * __ldg(vk + t));
+                        }
+                    }
+                }
+            }
+            // ---- step 3: very long segments, all threads of the CTA together
+            const int n_long = min(s_nlong, DN_LONG_CAP);
+            for (int l = 0; l < n_long; ++l) {
+                const int i = s_long[l];
+                const int len = -item_len[i];
+                const int* __restrict__ ck = B.crd + item_q[i];
+                const T* __restrict__ vk = Bval + item_q[i];
+                const T a = item_a[i];
+                for (int t = tid; t < len; t += DN_THREADS) {
+                    const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
+                    if (rel0 < span_bits) {
+                        const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
+                        if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * __ldg(vk + t));
+                    }
+                }
+            }
+            __syncthreads();
         }
-        __syncthreads();
 
         // copy out
         const i64 o0 = out0 + r0;
@@ -478,7 +561,7 @@ template <typename T>
 static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, const Csr& A, const Csr& B,
                              const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
-    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)words * 2 + 16;
+    const size_t smem = sizeof(T) * (size_t)CAP + (sizeof(T) + 12) * (size_t)DN_ENTRIES + (size_t)words * 4 + (size_t)words * 2 + 16;
     cudaError_t e;
     int per_sm = 0;
     auto k = dense_num_cta_kernel<T>;
