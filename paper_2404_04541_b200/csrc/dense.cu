@@ -28,7 +28,7 @@ constexpr int DW_THREADS = 256;            // warp-per-row kernels: 8 warps per 
 constexpr int DW_WARPS = DW_THREADS / 32;
 constexpr int DC_THREADS = 256;            // symbolic CTA kernel
 constexpr int DC_WARPS = DC_THREADS / 32;
-constexpr int DN_THREADS = 512;            // numeric CTA kernel
+constexpr int DN_THREADS = 1024;           // numeric CTA kernel
 constexpr int DN_WARPS = DN_THREADS / 32;
 
 // A dense row's slot in the arena: nw bitmap words, then for every chunk of 32 words the rank of
@@ -488,24 +488,35 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
             __syncthreads();
         }
 
-        // copy out
+        // copy out: values are already in output order.  The coordinates are expanded from the
+        // bitmap into shared memory (the accumulator's storage, once the values have left) so
+        // that the global stores are contiguous.
         const i64 o0 = out0 + r0;
-        for (int x = tid; x < nout; x += DN_THREADS) { Cval[o0 + x] = acc[x]; acc[x] = 0; }
+        for (int x = tid; x < nout; x += DN_THREADS) Cval[o0 + x] = acc[x];
+        __syncthreads();
+        int* stage = reinterpret_cast<int*>(acc);
         const int w_first = s_w0, w_last = s_w1;
         for (int w = w_first + tid; w <= w_last; w += DN_THREADS) {
             unsigned word = bm[w];
-            const int wp = pre[w];
-            const unsigned full = word;
+            int slot = pre[w];
+            if (w == w_first) {                         // drop the bits below the unit's first column
+                const unsigned below = (1u << (lo_rel & 31)) - 1u;
+                slot += __popc(word & below);
+                word &= ~below;
+            }
+            if (w == w_last && (hi_rel >> 5) == (unsigned)w) word &= (1u << (hi_rel & 31)) - 1u;
+            const int col0 = base + (w << 5);
             while (word) {
                 const int b = __ffs(word) - 1;
                 word &= word - 1;
-                const unsigned rel = ((unsigned)w << 5) + (unsigned)b;
-                if (rel >= lo_rel && rel < hi_rel) {
-                    const int slot = wp + __popc(full & ((1u << b) - 1u));
-                    if ((unsigned)slot < (unsigned)nout) Ccrd[o0 + slot] = base + (int)rel;
-                }
+                if ((unsigned)slot < (unsigned)nout) stage[slot] = col0 + b;
+                ++slot;
             }
         }
+        __syncthreads();
+        for (int x = tid; x < nout; x += DN_THREADS) Ccrd[o0 + x] = stage[x];
+        __syncthreads();
+        for (int x = tid; x < nout; x += DN_THREADS) acc[x] = 0;
     }
 }
 
