@@ -91,9 +91,10 @@ typedef struct {
     int32_t ism_warp_cap;     /* rows with <= this many products use the register ISM (<= 32)    */
     int32_t ism_cta_cap;      /* accumulation-array capacity of the shared-memory ISM, power of
                                  two in [64, 4096]; default 4096                                  */
-    int32_t dense_unit_outputs;/* outputs one CTA unit of the dense workspace accumulates (a long
-                                 row is cut into units of this many consecutive outputs), power
-                                 of two in [64, 8192]; default 4096                               */
+    int32_t dense_unit_outputs;/* outputs of a row the CTA dense workspace accumulates in shared
+                                 memory (outputs beyond them accumulate in the row's own value
+                                 segment in global memory), power of two in [64, 8192];
+                                 default 4096                                                      */
     int32_t dense_max_span;   /* widest column span (jmax - jmin + 1) a dense workspace may cover,
                                  in [32, 2^20]; default 2^20.  Wider rows go to ISM (AUTO) or
                                  fail with SPWS_WORKSPACE_TOO_LARGE (DENSE)                       */
@@ -111,7 +112,8 @@ typedef struct {
     int64_t max_row_products;
     int64_t rows_per_class[8];/* empty, ISM-register, ISM-shared(small), ISM-shared, dense-warp,
                                  dense-CTA(hub), dense-CTA, ISM-global                            */
-    int64_t dense_units;      /* CTA work units (row, output range) of the dense numeric pass     */
+    int64_t dense_units;      /* CTA work units (row, share of its A entries) of the dense numeric
+                                 pass                                                               */
     int32_t device_status;    /* last status word read back from the device                      */
     int32_t reserved;
     int64_t products_per_class[8];

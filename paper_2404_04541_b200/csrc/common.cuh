@@ -91,6 +91,17 @@ struct RowTables {
     int* unit_row;      // numeric: row of a CTA unit
 };
 
+// Products one dense CTA unit should take: 2^17, or more when the whole job is so large that the
+// unit table (rows + 2^19 entries) would not hold that many units.
+__host__ __device__ inline i64 dense_unit_products(i64 total_products) {
+    const i64 need = (total_products + (1ll << 19) - 1) >> 19;
+    return need > (1ll << 17) ? need : (1ll << 17);
+}
+__host__ __device__ inline int dense_units_of_row(i64 ub, i64 unit_products) {
+    const i64 n = (ub + unit_products - 1) / unit_products;
+    return (int)(n < 1 ? 1 : n);
+}
+
 __device__ __forceinline__ void raise_status(DevCtl* ctl, int s) { atomicCAS(&ctl->status, 0, s); }
 
 // Rows of class `cls` are perm[off, off + n).
@@ -179,8 +190,8 @@ cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B
 cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B);
 cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B,
                                   const i64* rowptr, int* Ccrd, void* Cval);
-cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, const Csr& A, const Csr& B,
-                                 const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, i64 total_products,
+                                 const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
                               const i64* rowptr, int* Ccrd, void* Cval);
 

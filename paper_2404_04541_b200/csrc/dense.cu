@@ -28,7 +28,7 @@ constexpr int DW_THREADS = 256;            // warp-per-row kernels: 8 warps per 
 constexpr int DW_WARPS = DW_THREADS / 32;
 constexpr int DC_THREADS = 256;            // symbolic CTA kernel
 constexpr int DC_WARPS = DC_THREADS / 32;
-constexpr int DN_THREADS = 1024;           // numeric CTA kernel
+constexpr int DN_THREADS = 512;            // numeric CTA kernel
 constexpr int DN_WARPS = DN_THREADS / 32;
 
 // A dense row's slot in the arena: nw bitmap words, then for every chunk of 32 words the rank of
@@ -302,39 +302,43 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 }
 
 // ---------------------------------------------------------------------------------------
-// numeric, CTA units (row, rank range)
+// numeric, CTA units.  A unit is a row, or an equal share of the A entries of a row with very
+// many products.  Every unit streams its B rows once, whole.  Outputs with rank < CAP accumulate
+// in shared memory; outputs beyond accumulate straight into the row's value segment in global
+// memory (zeroed beforehand), which keeps any row to a single pass whatever its output count.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ int nth_set_bit(unsigned word, int nth) {   // position of the nth (0-based) set bit
-    for (int x = 0; x < nth; ++x) word &= word - 1;
-    return __ffs(word) - 1;
-}
-
-// Plain lower bound by one lane (all lanes of a warp search different rows at once).
-__device__ __forceinline__ int lane_lower_bound(const int* __restrict__ ck, int lo, int hi, int c) {
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (__ldg(ck + mid) < c) lo = mid + 1; else hi = mid;
-    }
-    return lo;
-}
-
-constexpr int DN_ENTRIES = 1024;     // A entries examined per round
-constexpr int DN_LONG = 2048;        // segments at least this long are walked by the whole CTA
+constexpr int DN_LONG = 4096;        // B rows at least this long are walked by the whole CTA
 constexpr int DN_LONG_CAP = 32;
 
+// zero the part of the value segment that units add into
 template <typename T>
-__global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, Csr A, Csr B,
-                                                                   RowTables tab, const i64* __restrict__ rowptr,
+__global__ void __launch_bounds__(256) dense_zero_kernel(DevCtl* __restrict__ ctl, int CAP, i64 unit_products, RowTables tab,
+                                                         const i64* __restrict__ rowptr, T* __restrict__ Cval) {
+    if (ctl->status != 0) return;
+    const int n_units = ctl->n_units;
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+        const int row = tab.unit_row[u];
+        if (u != tab.row_unit0[row]) continue;
+        const i64 out0 = rowptr[row];
+        const int cnt = (int)(rowptr[row + 1] - out0);
+        const int first = dense_units_of_row(tab.ub[row], unit_products) > 1 ? 0 : CAP;
+        for (int x = first + threadIdx.x; x < cnt; x += 256) Cval[out0 + x] = 0;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, i64 unit_products,
+                                                                   Csr A, Csr B, RowTables tab, const i64* __restrict__ rowptr,
                                                                    int* __restrict__ Ccrd, T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
-    T* item_a = acc + CAP;                                                           // DN_ENTRIES
-    i64* item_q = reinterpret_cast<i64*>(item_a + DN_ENTRIES);                       // DN_ENTRIES
-    int* item_len = reinterpret_cast<int*>(item_q + DN_ENTRIES);                     // DN_ENTRIES
-    unsigned* bm = reinterpret_cast<unsigned*>(item_len + DN_ENTRIES);               // smem_words
-    short* pre = reinterpret_cast<short*>(bm + smem_words);                          // smem_words: rank of word start - r0
-    __shared__ int s_next, s_ca, s_cb, s_w0, s_w1, s_c0, s_c1, s_items, s_fetch, s_nlong, s_sumlen;
-    __shared__ int s_long[DN_LONG_CAP];
+    unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
+    int* crank = reinterpret_cast<int*>(bm + smem_words);                            // smem_words / 32 + 1: rank at chunk start
+    unsigned short* pre = reinterpret_cast<unsigned short*>(crank + smem_words / 32 + 1);   // rank of word start inside its chunk
+    __shared__ int s_next, s_entry, s_nlong;
+    __shared__ i64 s_long_q[DN_LONG_CAP];
+    __shared__ int s_long_len[DN_LONG_CAP];
+    __shared__ T s_long_a[DN_LONG_CAP];
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -344,179 +348,167 @@ __global__ void __launch_bounds__(DN_THREADS) dense_num_cta_kernel(DevCtl* __res
 
     for (;;) {
         __syncthreads();
-        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_CTA], 1);
+        if (tid == 0) { s_next = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_CTA], 1); s_entry = 0; s_nlong = 0; }
         __syncthreads();
         const int u = s_next;
         if (u >= n_units) break;
         const int row = tab.unit_row[u];
         const int uidx = u - tab.row_unit0[row];
+        const int nun = dense_units_of_row(tab.ub[row], unit_products);
         const int base = tab.jmin[row], last = tab.jmax[row];
         const int nw = min((last - base) / 32 + 1, smem_words);
         const int nch = chunks_of(nw);
+        const unsigned span_bits = (unsigned)nw * 32u;
         const i64 out0 = rowptr[row];
         const int cnt = (int)(rowptr[row + 1] - out0);
-        const int r0 = uidx * CAP;
-        const int nout = min(CAP, cnt - r0);
-        const int r1 = r0 + nout;
-        const bool whole = (r0 == 0 && r1 == cnt);
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        const i64 e_lo = ps + (pe - ps) * uidx / nun, e_hi = ps + (pe - ps) * (uidx + 1) / nun;
+        T* const gacc = Cval + out0;
+
+        // the row's bitmap, the rank at every chunk start and the rank of every word inside its chunk
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        const int* cpre = reinterpret_cast<const int*>(src + nw);      // rank at every chunk start
-        if (tid == 0) { s_ca = 0; s_cb = nch - 1; s_w0 = 0; s_w1 = nw - 1; s_c0 = 0; s_c1 = last - base + 1; }
-        __syncthreads();
-        // the chunks that hold ranks r0 and r1 bound the part of the bitmap this unit needs
-        if (!whole) {
-            for (int c = tid; c < nch; c += DN_THREADS) {
-                const int lo = cpre[c], hi = (c + 1 < nch) ? cpre[c + 1] : cnt;
-                if (lo <= r0 && r0 < hi) s_ca = c;
-                if (r1 < cnt && lo <= r1 && r1 < hi) s_cb = c;
-            }
-            __syncthreads();
-        }
-        const int ca = s_ca, cb = s_cb;
-        for (int c = ca + warp; c <= cb; c += DN_WARPS) {
+        for (int c = warp; c < nch; c += DN_WARPS) {
             const int w = (c << 5) + lane;
             const unsigned word = (w < nw) ? src[w] : 0u;
             const int pc = __popc(word);
-            const int start = cpre[c] + warp_incl_scan(pc) - pc;       // rank of this word's first bit
-            if (w < nw) {
-                bm[w] = word;
-                pre[w] = (short)max(-32768, min(32767, start - r0));
-                if (start <= r0 && r0 < start + pc) { s_w0 = w; s_c0 = (w << 5) + nth_set_bit(word, r0 - start); }
-                if (r1 < cnt && start <= r1 && r1 < start + pc) { s_w1 = w; s_c1 = (w << 5) + nth_set_bit(word, r1 - start); }
-            }
+            const int incl = warp_incl_scan(pc);
+            if (w < nw) { bm[w] = word; pre[w] = (unsigned short)(incl - pc); }
+            if (lane == 0) crank[c] = (int)src[nw + c];
         }
         __syncthreads();
-        // the unit owns the columns base + [lo_rel, hi_rel)
-        const unsigned lo_rel = (unsigned)s_c0, hi_rel = (unsigned)s_c1;
-        const int c_lo_abs = base + (int)lo_rel, c_hi_abs = base + (int)hi_rel;
-        const unsigned span_bits = (unsigned)nw * 32u;
 
-        for (i64 e0 = ps; e0 < pe; e0 += DN_ENTRIES) {
-            // ---- round, step 1: one lane per A entry finds the entry's B-row segment inside the
-            // unit's column range; non-empty segments are appended to the item list
-            if (tid == 0) { s_items = 0; s_fetch = 0; s_nlong = 0; s_sumlen = 0; }
-            __syncthreads();
-            const i64 e1 = min(pe, e0 + DN_ENTRIES);
-            for (i64 p = e0 + tid; p < e1; p += DN_THREADS) {
+#define SPWS_DENSE_ADD(REL, VAL)                                                                          \
+        if ((REL) < span_bits) {                                                                          \
+            const unsigned w_ = (REL) >> 5;                                                               \
+            const int r_ = crank[w_ >> 5] + pre[w_] + __popc(bm[w_] & ((1u << ((REL) & 31)) - 1u));        \
+            if (r_ < CAP) atomicAdd(&acc[r_], (VAL));                                                     \
+            else if (r_ < cnt) atomicAdd(gacc + r_, (VAL));                                               \
+        }
+
+        const float avg_len = (float)tab.ub[row] / fmaxf(1.0f, (float)(pe - ps));
+        if (avg_len >= 8.0f) {
+            // warps pull batches of 32 A entries: one lane per entry fetches its descriptor, then
+            // the warp walks the 32 B rows one after the other with its lanes across the row
+            for (;;) {
+                int b0 = 0;
+                if (lane == 0) b0 = atomicAdd(&s_entry, 32);
+                b0 = __shfl_sync(0xffffffffu, b0, 0);
+                const i64 p0 = e_lo + b0;
+                if (p0 >= e_hi) break;
+                i64 my_qs = 0;
+                int my_len = 0;
+                T my_a = 0;
+                if (p0 + lane < e_hi) {
+                    const int k = __ldg(A.crd + p0 + lane);
+                    if ((unsigned)k < (unsigned)B.nrows) {
+                        my_qs = __ldg(B.pos + k);
+                        my_len = (int)(__ldg(B.pos + k + 1) - my_qs);
+                    }
+                    my_a = __ldg(Aval + p0 + lane);
+                }
+                const int nE = (int)min((i64)32, e_hi - p0);
+                for (int e = 0; e < nE; ++e) {
+                    const i64 qs = __shfl_sync(0xffffffffu, my_qs, e);
+                    const int len = __shfl_sync(0xffffffffu, my_len, e);
+                    const T a = __shfl_sync(0xffffffffu, my_a, e);
+                    if (len >= DN_LONG) {               // defer: the whole CTA takes it after the loop
+                        int l = 0;
+                        if (lane == 0) l = atomicAdd(&s_nlong, 1);
+                        l = __shfl_sync(0xffffffffu, l, 0);
+                        if (l < DN_LONG_CAP) {
+                            if (lane == 0) { s_long_q[l] = qs; s_long_len[l] = len; s_long_a[l] = a; }
+                            continue;
+                        }
+                    }
+                    const int* __restrict__ ck = B.crd + qs;
+                    const T* __restrict__ vk = Bval + qs;
+                    int t = lane;
+                    for (; t + 96 < len; t += 128) {    // four products in flight per lane
+                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base), rel1 = (unsigned)(__ldg(ck + t + 32) - base);
+                        const unsigned rel2 = (unsigned)(__ldg(ck + t + 64) - base), rel3 = (unsigned)(__ldg(ck + t + 96) - base);
+                        const T v0 = a * __ldg(vk + t), v1 = a * __ldg(vk + t + 32);
+                        const T v2 = a * __ldg(vk + t + 64), v3 = a * __ldg(vk + t + 96);
+                        SPWS_DENSE_ADD(rel0, v0)
+                        SPWS_DENSE_ADD(rel1, v1)
+                        SPWS_DENSE_ADD(rel2, v2)
+                        SPWS_DENSE_ADD(rel3, v3)
+                    }
+                    for (; t < len; t += 32) {
+                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
+                        const T v0 = a * __ldg(vk + t);
+                        SPWS_DENSE_ADD(rel0, v0)
+                    }
+                }
+            }
+        } else {
+            // short B rows: one lane per A entry
+            for (i64 p = e_lo + tid; p < e_hi; p += DN_THREADS) {
                 const int k = __ldg(A.crd + p);
                 if ((unsigned)k >= (unsigned)B.nrows) continue;
                 const i64 qs = __ldg(B.pos + k);
                 const int len = (int)(__ldg(B.pos + k + 1) - qs);
-                int s0 = 0, s1 = len;
-                if (!whole && len > 0) {
-                    const int* __restrict__ ck = B.crd + qs;
-                    s0 = lane_lower_bound(ck, 0, len, c_lo_abs);
-                    s1 = lane_lower_bound(ck, s0, len, c_hi_abs);
-                }
-                if (s1 > s0) {
-                    const int i = atomicAdd(&s_items, 1);
-                    item_q[i] = qs + s0;
-                    item_len[i] = s1 - s0;
-                    item_a[i] = __ldg(Aval + p);
-                    atomicAdd(&s_sumlen, s1 - s0);
-                    if (s1 - s0 >= DN_LONG) {
-                        const int l = atomicAdd(&s_nlong, 1);
-                        if (l < DN_LONG_CAP) { s_long[l] = i; item_len[i] = -(s1 - s0); }   // negative: taken by the CTA-wide pass
-                    }
+                const T a = __ldg(Aval + p);
+                for (int t = 0; t < len; ++t) {
+                    const unsigned rel0 = (unsigned)(__ldg(B.crd + qs + t) - base);
+                    const T v0 = a * __ldg(Bval + qs + t);
+                    SPWS_DENSE_ADD(rel0, v0)
                 }
             }
-            __syncthreads();
-            // ---- step 2: lane groups pull items; group size ~ mean segment length
-            const int n_items = s_items;
-            int gs = 32;
-            {
-                const float avg = (float)s_sumlen / fmaxf(1.0f, (float)n_items);
-                while (gs > 1 && (float)(gs >> 1) >= avg) gs >>= 1;
-            }
-            const int lg = __ffs(gs) - 1;
-            const int gl = tid & (gs - 1);
-            const unsigned gshift = (unsigned)(lane - gl);
-            const unsigned gmask = (gs == 32) ? 0xffffffffu : (((1u << gs) - 1u) << gshift);
-            const int batch = gs >= 8 ? 1 : (8 >> lg);          // items a group takes per fetch
-            for (;;) {
-                int i0 = 0;
-                if (gl == 0) i0 = atomicAdd(&s_fetch, batch);
-                i0 = __shfl_sync(gmask, i0, (int)gshift);
-                if (i0 >= n_items) break;
-                const int i1 = min(n_items, i0 + batch);
-                for (int i = i0; i < i1; ++i) {
-                    const int len = item_len[i];
-                    if (len < 0) continue;
-                    const int* __restrict__ ck = B.crd + item_q[i];
-                    const T* __restrict__ vk = Bval + item_q[i];
-                    const T a = item_a[i];
-                    int t = gl;
-                    for (; t + gs < len; t += 2 * gs) {         // two products in flight per lane
-                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                        const unsigned rel1 = (unsigned)(__ldg(ck + t + gs) - base);
-                        const T v0 = __ldg(vk + t), v1 = __ldg(vk + t + gs);
-                        if (rel0 < span_bits) {
-                            const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                            if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v0);
-                        }
-                        if (rel1 < span_bits) {
-                            const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
-                            if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * v1);
-                        }
-                    }
-                    if (t < len) {
-                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                        if (rel0 < span_bits) {
-                            const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                            if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * __ldg(vk + t));
-                        }
-                    }
-                }
-            }
-            // ---- step 3: very long segments, all threads of the CTA together
+        }
+        __syncthreads();
+        {   // very long B rows, all threads of the CTA together
             const int n_long = min(s_nlong, DN_LONG_CAP);
             for (int l = 0; l < n_long; ++l) {
-                const int i = s_long[l];
-                const int len = -item_len[i];
-                const int* __restrict__ ck = B.crd + item_q[i];
-                const T* __restrict__ vk = Bval + item_q[i];
-                const T a = item_a[i];
+                const int len = s_long_len[l];
+                const int* __restrict__ ck = B.crd + s_long_q[l];
+                const T* __restrict__ vk = Bval + s_long_q[l];
+                const T a = s_long_a[l];
                 for (int t = tid; t < len; t += DN_THREADS) {
                     const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                    if (rel0 < span_bits) {
-                        const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                        if ((unsigned)slot < (unsigned)CAP) atomicAdd(&acc[slot], a * __ldg(vk + t));
-                    }
+                    const T v0 = a * __ldg(vk + t);
+                    SPWS_DENSE_ADD(rel0, v0)
                 }
             }
-            __syncthreads();
+            if (n_long) __syncthreads();
         }
+#undef SPWS_DENSE_ADD
 
-        // copy out: values are already in output order.  The coordinates are expanded from the
-        // bitmap into shared memory (the accumulator's storage, once the values have left) so
-        // that the global stores are contiguous.
-        const i64 o0 = out0 + r0;
-        for (int x = tid; x < nout; x += DN_THREADS) Cval[o0 + x] = acc[x];
-        __syncthreads();
-        int* stage = reinterpret_cast<int*>(acc);
-        const int w_first = s_w0, w_last = s_w1;
-        for (int w = w_first + tid; w <= w_last; w += DN_THREADS) {
-            unsigned word = bm[w];
-            int slot = pre[w];
-            if (w == w_first) {                         // drop the bits below the unit's first column
-                const unsigned below = (1u << (lo_rel & 31)) - 1u;
-                slot += __popc(word & below);
-                word &= ~below;
-            }
-            if (w == w_last && (hi_rel >> 5) == (unsigned)w) word &= (1u << (hi_rel & 31)) - 1u;
-            const int col0 = base + (w << 5);
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                if ((unsigned)slot < (unsigned)nout) stage[slot] = col0 + b;
-                ++slot;
+        // copy out the shared-memory part of the values
+        const int n_smem = min(cnt, CAP);
+        if (nun == 1) {
+            for (int x = tid; x < n_smem; x += DN_THREADS) gacc[x] = acc[x];
+        } else {
+            for (int x = tid; x < n_smem; x += DN_THREADS) {
+                const T v = acc[x];
+                if (v != (T)0) atomicAdd(gacc + x, v);
             }
         }
         __syncthreads();
-        for (int x = tid; x < nout; x += DN_THREADS) Ccrd[o0 + x] = stage[x];
-        __syncthreads();
-        for (int x = tid; x < nout; x += DN_THREADS) acc[x] = 0;
+        // the row's first unit writes the coordinates: bits are expanded into shared memory (the
+        // accumulator's storage) in passes of STAGE outputs so that the global stores are contiguous
+        if (uidx == 0) {
+            int* stage = reinterpret_cast<int*>(acc);
+            const int STAGE = (int)(CAP * sizeof(T) / sizeof(int));
+            for (int lo = 0; lo < cnt; lo += STAGE) {
+                const int hi = min(cnt, lo + STAGE);
+                for (int w = tid; w < nw; w += DN_THREADS) {
+                    unsigned word = bm[w];
+                    int slot = crank[w >> 5] + pre[w] - lo;
+                    if (slot >= hi - lo || slot + __popc(word) <= 0) continue;
+                    const int col0 = base + (w << 5);
+                    while (word) {
+                        const int b = __ffs(word) - 1;
+                        word &= word - 1;
+                        if ((unsigned)slot < (unsigned)(hi - lo)) stage[slot] = col0 + b;
+                        ++slot;
+                    }
+                }
+                __syncthreads();
+                for (int x = tid; x < hi - lo; x += DN_THREADS) Ccrd[out0 + lo + x] = stage[x];
+                __syncthreads();
+            }
+        }
+        for (int x = tid; x < CAP; x += DN_THREADS) acc[x] = 0;
     }
 }
 
@@ -569,26 +561,29 @@ cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, 
 }
 
 template <typename T>
-static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, const Csr& A, const Csr& B,
+static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, i64 total_products, const Csr& A, const Csr& B,
                              const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
-    const size_t smem = sizeof(T) * (size_t)CAP + (sizeof(T) + 12) * (size_t)DN_ENTRIES + (size_t)words * 4 + (size_t)words * 2 + 16;
+    const i64 unit_products = dense_unit_products(total_products);
+    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32 + 1) * 4 + (size_t)words * 2 + 16;
     cudaError_t e;
     int per_sm = 0;
     auto k = dense_num_cta_kernel<T>;
     if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DN_THREADS, smem)) != cudaSuccess) return e;
-    k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
-    ++c.launches;
+    dense_zero_kernel<T><<<persistent_grid(c, 8, n_units_host), 256, 0, c.stream>>>(c.ctl, CAP, unit_products, c.tab, rowptr, (T*)Cval);
+    k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab, rowptr,
+                                                                             Ccrd, (T*)Cval);
+    c.launches += 2;
     return cudaGetLastError();
 }
 
-cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, const Csr& A, const Csr& B,
-                                 const i64* rowptr, int* Ccrd, void* Cval) {
+cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, i64 total_products,
+                                 const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
     int words = max_span_words > 0 ? max_span_words : c.dense_smem_words;
     words = (words + 31) & ~31;
-    return c.is_f64 ? num_cta_t<double>(c, n_units_host, words, A, B, rowptr, Ccrd, Cval)
-                    : num_cta_t<float>(c, n_units_host, words, A, B, rowptr, Ccrd, Cval);
+    return c.is_f64 ? num_cta_t<double>(c, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval)
+                    : num_cta_t<float>(c, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval);
 }
 
 }  // namespace spws

@@ -238,8 +238,9 @@ cudaError_t launch_bin_rows(const LaunchCtx& c, int m) {
 }
 
 // Numeric routing of the dense rows, once their output counts are known: a row the warp kernel
-// counted and whose outputs fit a warp's accumulator stays with a warp; every other row is cut
-// into CTA units of `unit_outputs` consecutive outputs (rank ranges).
+// counted and whose outputs fit a warp's accumulator stays with a warp; every other row becomes
+// one CTA unit, or several when it has many products: unit c of n takes the c-th n-th of the
+// row's A entries (all units of a row add into the same outputs).
 __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
     __shared__ int ws[33];
     __shared__ int s_wbase, s_ubase;
@@ -249,6 +250,7 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
     class_range(ctl, CLS_DENSE_HUB, o5, n5);
     class_range(ctl, CLS_DENSE_CTA, o6, n6);
     const int n = n4 + n5 + n6;                       // the three classes are adjacent in perm
+    const i64 unit_products = dense_unit_products(ctl->products);
     for (i64 b0 = (i64)blockIdx.x * blockDim.x; b0 < n; b0 += (i64)gridDim.x * blockDim.x) {
         const i64 r = b0 + threadIdx.x;
         int row = -1, cnt = 0, to_warp = 0, nu = 0;
@@ -257,7 +259,7 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
             row = tab.perm[off + r];
             cnt = tab.cnt[row];
             to_warp = tab.cls[row] == CLS_DENSE_WARP && cnt <= DENSE_WARP_ACC;
-            nu = to_warp ? 0 : (cnt + prm.unit_outputs - 1) / prm.unit_outputs;
+            nu = to_warp ? 0 : dense_units_of_row(tab.ub[row], unit_products);
         }
         int wtot, utot;
         const int wpos = block_excl_scan<256>(to_warp, ws, wtot);

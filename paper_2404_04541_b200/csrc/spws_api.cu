@@ -134,11 +134,9 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) 
     L.bm_off = take(8 * (size_t)m);
     L.warp_rows = take(4 * (size_t)m);
     L.row_unit0 = take(4 * (size_t)m);
-    // a dense row has at most min(ncols, dense_max_span) outputs
+    // one unit per dense row plus at most 2^19 more for rows split by product count
     const int64_t span_cap = ncols < p->opt.dense_max_span ? ncols : p->opt.dense_max_span;
-    int64_t units_per_row = (span_cap + p->opt.dense_unit_outputs - 1) / p->opt.dense_unit_outputs;
-    if (units_per_row < 1) units_per_row = 1;
-    int64_t ucap = m * units_per_row;
+    int64_t ucap = m + (1ll << 19) + 1024;
     if (ucap > 0x7fff0000ll) ucap = 0x7fff0000ll;
     L.unit_cap = (int)ucap;
     L.unit_row = take(4 * (size_t)ucap);
@@ -552,7 +550,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         mark(plan, SPWS_T_NUM_DENSE_WARP);
     }
     if (s.dense_units > 0) {
-        CUDA_TRY(launch_dense_num_cta(c, (int)s.dense_units, plan->max_span_words, S.A, S.B, rowptr, crd, C->val));
+        CUDA_TRY(launch_dense_num_cta(c, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_DENSE_CTA);
     }
     if (s.rows_per_class[CLS_ISM_GLOBAL] > 0) {

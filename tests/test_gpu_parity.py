@@ -76,8 +76,8 @@ def test_random_small_all_routes(ctx, oracle_mod, policy, m, k, n, dens, seed):
     stats = check_spgemm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
     if policy == "ism" and m >= 37:
         assert stats["rows_per_class"][GLOBAL] > 0                   # the global-memory ISM ran
-    if policy == "dense" and n >= 700:                               # some row was cut into several units
-        assert stats["dense_units"] > sum(stats["rows_per_class"][DENSE]) - stats["dense_warp_rows"]
+    if policy == "dense" and n >= 700:                               # rows beyond a warp's capacity went to CTA units
+        assert stats["dense_units"] == sum(stats["rows_per_class"][DENSE]) - stats["dense_warp_rows"] > 0
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float64])
@@ -141,6 +141,23 @@ def test_edge_cases(ctx, oracle_mod, policy):
                       np.concatenate([np.sort(rng.choice(5000, 5, replace=False)) for _ in live]),
                       rng.uniform(-1, 1, 5 * live.size))
     check_spgemm(ctx, oracle_mod, A2, B3, policy)
+
+
+@pytest.mark.parametrize("policy", ["dense", "auto"])
+def test_heavy_row_is_split_over_several_units(ctx, oracle_mod, policy):
+    """A row with ~400 k products is shared by several CTAs (each takes a slice of its A entries
+    and adds into the same outputs); with a 64-output shared-memory accumulator most outputs
+    accumulate in global memory."""
+    rng = np.random.default_rng(5)
+    cols = np.sort(rng.choice(4000, 2000, replace=False))
+    A = CSR.from_coo(40, 4000, np.concatenate([np.full(2000, 7), np.arange(40)]),
+                     np.concatenate([cols, rng.integers(0, 4000, 40)]), rng.uniform(-1, 1, 2040))
+    A = CSR.from_dense(A.to_dense())                                 # merges accidental duplicates
+    B = uniform_rows_csr(4000, 30000, 200, 6)
+    for opts in ({}, dict(dense_unit_outputs=64)):
+        stats = check_spgemm(ctx, oracle_mod, A, B, policy, **opts)
+        assert stats["max_row_products"] >= 400000
+        assert stats["dense_units"] >= sum(stats["rows_per_class"][DENSE]) - stats["dense_warp_rows"] + 3
 
 
 def test_ism_routes_reproduce_sequential_sum(ctx, oracle_mod):
