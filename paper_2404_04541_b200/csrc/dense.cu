@@ -307,8 +307,8 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 // in shared memory; outputs beyond accumulate straight into the row's value segment in global
 // memory (zeroed beforehand), which keeps any row to a single pass whatever its output count.
 // ---------------------------------------------------------------------------------------
-constexpr int DN_LONG = 4096;        // B rows at least this long are walked by the whole CTA
-constexpr int DN_LONG_CAP = 32;
+constexpr int DN_ENTRIES = 1024;     // A entries whose descriptors are staged per round
+constexpr int DN_TILE = 256;         // products a warp takes per fetch
 
 // zero the part of the value segment that units add into
 template <typename T>
@@ -335,10 +335,13 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
     unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
     int* crank = reinterpret_cast<int*>(bm + smem_words);                            // smem_words / 32 + 1: rank at chunk start
     unsigned short* pre = reinterpret_cast<unsigned short*>(crank + smem_words / 32 + 1);   // rank of word start inside its chunk
-    __shared__ int s_next, s_entry, s_nlong;
-    __shared__ i64 s_long_q[DN_LONG_CAP];
-    __shared__ int s_long_len[DN_LONG_CAP];
-    __shared__ T s_long_a[DN_LONG_CAP];
+    // staged descriptors of up to DN_ENTRIES A entries: B-row start, A value, running product count
+    i64* d_qs = reinterpret_cast<i64*>(smem_raw + ((sizeof(T) * (size_t)CAP + 4 * (size_t)smem_words + 4 * (size_t)(smem_words / 32 + 1) +
+                                                     2 * (size_t)smem_words + 15) & ~(size_t)15));
+    T* d_a = reinterpret_cast<T*>(d_qs + DN_ENTRIES);
+    int* d_pre = reinterpret_cast<int*>(d_a + DN_ENTRIES);                           // DN_ENTRIES + 1
+    __shared__ int s_next, s_tile;
+    __shared__ int ws[33];
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -348,7 +351,7 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
 
     for (;;) {
         __syncthreads();
-        if (tid == 0) { s_next = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_CTA], 1); s_entry = 0; s_nlong = 0; }
+        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_CTA], 1);
         __syncthreads();
         const int u = s_next;
         if (u >= n_units) break;
@@ -387,58 +390,76 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
 
         const float avg_len = (float)tab.ub[row] / fmaxf(1.0f, (float)(pe - ps));
         if (avg_len >= 8.0f) {
-            // warps pull batches of 32 A entries: one lane per entry fetches its descriptor, then
-            // the warp walks the 32 B rows one after the other with its lanes across the row
-            for (;;) {
-                int b0 = 0;
-                if (lane == 0) b0 = atomicAdd(&s_entry, 32);
-                b0 = __shfl_sync(0xffffffffu, b0, 0);
-                const i64 p0 = e_lo + b0;
-                if (p0 >= e_hi) break;
-                i64 my_qs = 0;
-                int my_len = 0;
-                T my_a = 0;
-                if (p0 + lane < e_hi) {
-                    const int k = __ldg(A.crd + p0 + lane);
-                    if ((unsigned)k < (unsigned)B.nrows) {
-                        my_qs = __ldg(B.pos + k);
-                        my_len = (int)(__ldg(B.pos + k + 1) - my_qs);
-                    }
-                    my_a = __ldg(Aval + p0 + lane);
-                }
-                const int nE = (int)min((i64)32, e_hi - p0);
-                for (int e = 0; e < nE; ++e) {
-                    const i64 qs = __shfl_sync(0xffffffffu, my_qs, e);
-                    const int len = __shfl_sync(0xffffffffu, my_len, e);
-                    const T a = __shfl_sync(0xffffffffu, my_a, e);
-                    if (len >= DN_LONG) {               // defer: the whole CTA takes it after the loop
-                        int l = 0;
-                        if (lane == 0) l = atomicAdd(&s_nlong, 1);
-                        l = __shfl_sync(0xffffffffu, l, 0);
-                        if (l < DN_LONG_CAP) {
-                            if (lane == 0) { s_long_q[l] = qs; s_long_len[l] = len; s_long_a[l] = a; }
-                            continue;
+            // Rounds of up to DN_ENTRIES A entries.  Step 1: every thread fetches the descriptors
+            // of two entries; a block scan turns the B-row lengths into a running product count.
+            // Step 2: warps pull tiles of DN_TILE consecutive products of that stream, so the
+            // work is shared evenly however long the individual B rows are.
+            for (i64 e0 = e_lo; e0 < e_hi; e0 += DN_ENTRIES) {
+                const int nE = (int)min((i64)DN_ENTRIES, e_hi - e0);
+                int len2[2] = {0, 0};
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    const int i = 2 * tid + x;
+                    if (i < nE) {
+                        const int k = __ldg(A.crd + e0 + i);
+                        i64 qs = 0;
+                        if ((unsigned)k < (unsigned)B.nrows) {
+                            qs = __ldg(B.pos + k);
+                            len2[x] = (int)(__ldg(B.pos + k + 1) - qs);
                         }
-                    }
-                    const int* __restrict__ ck = B.crd + qs;
-                    const T* __restrict__ vk = Bval + qs;
-                    int t = lane;
-                    for (; t + 96 < len; t += 128) {    // four products in flight per lane
-                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base), rel1 = (unsigned)(__ldg(ck + t + 32) - base);
-                        const unsigned rel2 = (unsigned)(__ldg(ck + t + 64) - base), rel3 = (unsigned)(__ldg(ck + t + 96) - base);
-                        const T v0 = a * __ldg(vk + t), v1 = a * __ldg(vk + t + 32);
-                        const T v2 = a * __ldg(vk + t + 64), v3 = a * __ldg(vk + t + 96);
-                        SPWS_DENSE_ADD(rel0, v0)
-                        SPWS_DENSE_ADD(rel1, v1)
-                        SPWS_DENSE_ADD(rel2, v2)
-                        SPWS_DENSE_ADD(rel3, v3)
-                    }
-                    for (; t < len; t += 32) {
-                        const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                        const T v0 = a * __ldg(vk + t);
-                        SPWS_DENSE_ADD(rel0, v0)
+                        d_qs[i] = qs;
+                        d_a[i] = __ldg(Aval + e0 + i);
                     }
                 }
+                int total;
+                const int excl = block_excl_scan<DN_THREADS>(len2[0] + len2[1], ws, total);
+                if (2 * tid < nE) d_pre[2 * tid] = excl;
+                if (2 * tid + 1 < nE) d_pre[2 * tid + 1] = excl + len2[0];
+                if (tid == 0) { d_pre[nE] = total; s_tile = 0; }
+                __syncthreads();
+                for (;;) {
+                    int t0 = 0;
+                    if (lane == 0) t0 = atomicAdd(&s_tile, DN_TILE);
+                    t0 = __shfl_sync(0xffffffffu, t0, 0);
+                    if (t0 >= total) break;
+                    const int t1 = min(total, t0 + DN_TILE);
+                    int e = 0;
+                    {   // entry that holds product t0: the last one whose running count is <= t0
+                        int lo = 0, hi = nE;
+                        while (hi - lo > 1) {
+                            const int mid = (lo + hi) >> 1;
+                            if (d_pre[mid] <= t0) lo = mid; else hi = mid;
+                        }
+                        e = lo;
+                    }
+                    while (t0 < t1) {
+                        const int e_end = d_pre[e + 1];
+                        if (e_end <= t0) { ++e; continue; }
+                        const int seg_end = min(t1, e_end);
+                        const int off = t0 - d_pre[e], n = seg_end - t0;
+                        const int* __restrict__ ck = B.crd + d_qs[e] + off;
+                        const T* __restrict__ vk = Bval + d_qs[e] + off;
+                        const T a = d_a[e];
+                        int t = lane;
+                        for (; t + 96 < n; t += 128) {    // four products in flight per lane
+                            const unsigned rel0 = (unsigned)(__ldg(ck + t) - base), rel1 = (unsigned)(__ldg(ck + t + 32) - base);
+                            const unsigned rel2 = (unsigned)(__ldg(ck + t + 64) - base), rel3 = (unsigned)(__ldg(ck + t + 96) - base);
+                            const T v0 = a * __ldg(vk + t), v1 = a * __ldg(vk + t + 32);
+                            const T v2 = a * __ldg(vk + t + 64), v3 = a * __ldg(vk + t + 96);
+                            SPWS_DENSE_ADD(rel0, v0)
+                            SPWS_DENSE_ADD(rel1, v1)
+                            SPWS_DENSE_ADD(rel2, v2)
+                            SPWS_DENSE_ADD(rel3, v3)
+                        }
+                        for (; t < n; t += 32) {
+                            const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
+                            const T v0 = a * __ldg(vk + t);
+                            SPWS_DENSE_ADD(rel0, v0)
+                        }
+                        t0 = seg_end;
+                    }
+                }
+                __syncthreads();
             }
         } else {
             // short B rows: one lane per A entry
@@ -454,22 +475,7 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
                     SPWS_DENSE_ADD(rel0, v0)
                 }
             }
-        }
-        __syncthreads();
-        {   // very long B rows, all threads of the CTA together
-            const int n_long = min(s_nlong, DN_LONG_CAP);
-            for (int l = 0; l < n_long; ++l) {
-                const int len = s_long_len[l];
-                const int* __restrict__ ck = B.crd + s_long_q[l];
-                const T* __restrict__ vk = Bval + s_long_q[l];
-                const T a = s_long_a[l];
-                for (int t = tid; t < len; t += DN_THREADS) {
-                    const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                    const T v0 = a * __ldg(vk + t);
-                    SPWS_DENSE_ADD(rel0, v0)
-                }
-            }
-            if (n_long) __syncthreads();
+            __syncthreads();
         }
 #undef SPWS_DENSE_ADD
 
@@ -565,7 +571,8 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, i6
                              const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
     const i64 unit_products = dense_unit_products(total_products);
-    const size_t smem = sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32 + 1) * 4 + (size_t)words * 2 + 16;
+    const size_t smem = ((sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32 + 1) * 4 + (size_t)words * 2 + 15) & ~(size_t)15) +
+                        (size_t)DN_ENTRIES * (8 + sizeof(T)) + (size_t)(DN_ENTRIES + 1) * 4 + 16;
     cudaError_t e;
     int per_sm = 0;
     auto k = dense_num_cta_kernel<T>;
