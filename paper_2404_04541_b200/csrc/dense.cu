@@ -479,42 +479,71 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
         }
 #undef SPWS_DENSE_ADD
 
-        // copy out the shared-memory part of the values
+        // copy out the shared-memory part of the values (the coordinates are written by
+        // dense_emit_crd_kernel)
         const int n_smem = min(cnt, CAP);
         if (nun == 1) {
-            for (int x = tid; x < n_smem; x += DN_THREADS) gacc[x] = acc[x];
+            for (int x = tid; x < n_smem; x += DN_THREADS) { gacc[x] = acc[x]; acc[x] = 0; }
         } else {
             for (int x = tid; x < n_smem; x += DN_THREADS) {
                 const T v = acc[x];
+                acc[x] = 0;
                 if (v != (T)0) atomicAdd(gacc + x, v);
             }
         }
-        __syncthreads();
-        // the row's first unit writes the coordinates: bits are expanded into shared memory (the
-        // accumulator's storage) in passes of STAGE outputs so that the global stores are contiguous
-        if (uidx == 0) {
-            int* stage = reinterpret_cast<int*>(acc);
-            const int STAGE = (int)(CAP * sizeof(T) / sizeof(int));
-            for (int lo = 0; lo < cnt; lo += STAGE) {
-                const int hi = min(cnt, lo + STAGE);
-                for (int w = tid; w < nw; w += DN_THREADS) {
-                    unsigned word = bm[w];
-                    int slot = crank[w >> 5] + pre[w] - lo;
-                    if (slot >= hi - lo || slot + __popc(word) <= 0) continue;
-                    const int col0 = base + (w << 5);
-                    while (word) {
-                        const int b = __ffs(word) - 1;
-                        word &= word - 1;
-                        if ((unsigned)slot < (unsigned)(hi - lo)) stage[slot] = col0 + b;
-                        ++slot;
-                    }
+    }
+}
+
+// Coordinates of the CTA-unit rows: a warp expands one 32-word chunk of the saved bitmap at a
+// time (its outputs are the contiguous range that starts at the chunk's saved rank) into a small
+// shared-memory stage and stores it with contiguous writes.
+constexpr int DE_THREADS = 256;
+constexpr int DE_WARPS = DE_THREADS / 32;
+
+__global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __restrict__ ctl, RowTables tab,
+                                                                    const i64* __restrict__ rowptr, int* __restrict__ Ccrd) {
+    __shared__ int s_stage[DE_WARPS][1024];
+    if (ctl->status != 0) return;
+    const int n_units = ctl->n_units;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int* stage = s_stage[warp];
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+        const int row = tab.unit_row[u];
+        if (u != tab.row_unit0[row]) continue;
+        const int base = tab.jmin[row];
+        const int nw = (tab.jmax[row] - base) / 32 + 1;
+        const int nch = chunks_of(nw);
+        const unsigned* src = tab.bm_arena + tab.bm_off[row];
+        const i64 out0 = rowptr[row];
+        for (int c0 = warp * 4; c0 < nch; c0 += DE_WARPS * 4) {      // four chunks' loads in flight
+            unsigned words[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int w = ((c0 + x) << 5) + lane;
+                words[x] = (w < nw) ? src[w] : 0u;
+            }
+            const int my_rank = (lane < 4 && c0 + lane < nch) ? (int)src[nw + c0 + lane] : 0;
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                unsigned word = words[x];
+                const int pc = __popc(word);
+                const int incl = warp_incl_scan(pc);
+                const int n = __shfl_sync(0xffffffffu, incl, 31);
+                const int rank0 = __shfl_sync(0xffffffffu, my_rank, x);
+                if (n == 0) continue;
+                int slot = incl - pc;
+                const int col0 = base + (((c0 + x) << 5) + lane << 5);
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+                    stage[slot++] = col0 + b;
                 }
-                __syncthreads();
-                for (int x = tid; x < hi - lo; x += DN_THREADS) Ccrd[out0 + lo + x] = stage[x];
-                __syncthreads();
+                __syncwarp();
+                const i64 o = out0 + rank0;
+                for (int y = lane; y < n; y += 32) Ccrd[o + y] = stage[y];
+                __syncwarp();
             }
         }
-        for (int x = tid; x < CAP; x += DN_THREADS) acc[x] = 0;
     }
 }
 
@@ -581,7 +610,8 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, i6
     dense_zero_kernel<T><<<persistent_grid(c, 8, n_units_host), 256, 0, c.stream>>>(c.ctl, CAP, unit_products, c.tab, rowptr, (T*)Cval);
     k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab, rowptr,
                                                                              Ccrd, (T*)Cval);
-    c.launches += 2;
+    dense_emit_crd_kernel<<<persistent_grid(c, 8, n_units_host), DE_THREADS, 0, c.stream>>>(c.ctl, c.tab, rowptr, Ccrd);
+    c.launches += 3;
     return cudaGetLastError();
 }
 
