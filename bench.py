@@ -174,6 +174,7 @@ def main():
     ap.add_argument("--policy", default="auto")
     ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--opt", action="append", default=[], help="plan option as name=value (repeatable)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -204,7 +205,11 @@ def main():
     ctx = api.Context(dev)
     dA = api.DeviceCSR.from_host(A, device=dev)
     dB = dA if B is A else api.DeviceCSR.from_host(B, device=dev)
-    plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, cfg["dtype"], args.policy)
+    options = {}
+    for kv in args.opt:
+        name, value = kv.split("=", 1)
+        options[name] = float(value) if "." in value else int(value)
+    plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, cfg["dtype"], args.policy, **options)
     plan.set_profiling(True)
 
     # a first pass sizes C; its buffers are reused by every step (allocation is outside the timed region)
@@ -286,7 +291,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64" if V == 8 else "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "policy": args.policy,
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "policy": args.policy, "options": options,
                        "seed": args.seed, "rows": int(A.nrows), "nnzA": int(A.nnz), "products": int(products),
                        "nnzC": int(nnzC), "l2": "512 MiB buffer written between timed steps",
                        "timed": "spws_symbolic + spws_numeric; C buffers preallocated"},

@@ -389,7 +389,8 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
         }
 
         const float avg_len = (float)tab.ub[row] / fmaxf(1.0f, (float)(pe - ps));
-        if (avg_len >= 8.0f) {
+        const bool long_rows = avg_len >= 64.0f;
+        {
             // Rounds of up to DN_ENTRIES A entries.  Step 1: every thread fetches the descriptors
             // of two entries; a block scan turns the B-row lengths into a running product count.
             // Step 2: warps pull tiles of DN_TILE consecutive products of that stream, so the
@@ -432,6 +433,32 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
                         }
                         e = lo;
                     }
+                    if (!long_rows) {
+                        // short B rows: every lane walks its own products (t0 + lane, + 32, ...) and
+                        // advances its own entry index, so lanes stay busy across row boundaries
+                        int my_e = e;
+                        for (int t = t0 + lane; t < t1; t += 64) {      // two products in flight per lane
+                            while (d_pre[my_e + 1] <= t) ++my_e;
+                            const i64 q0 = d_qs[my_e] + (t - d_pre[my_e]);
+                            const T a0 = d_a[my_e];
+                            const int t2 = t + 32;
+                            const bool two = t2 < t1;
+                            i64 q1 = q0;
+                            T a1 = 0;
+                            if (two) {
+                                while (d_pre[my_e + 1] <= t2) ++my_e;
+                                q1 = d_qs[my_e] + (t2 - d_pre[my_e]);
+                                a1 = d_a[my_e];
+                            }
+                            const unsigned rel0 = (unsigned)(__ldg(B.crd + q0) - base);
+                            const unsigned rel1 = two ? (unsigned)(__ldg(B.crd + q1) - base) : 0xffffffffu;
+                            const T v0 = a0 * __ldg(Bval + q0);
+                            const T v1 = a1 * __ldg(Bval + q1);
+                            SPWS_DENSE_ADD(rel0, v0)
+                            SPWS_DENSE_ADD(rel1, v1)
+                        }
+                        continue;
+                    }
                     while (t0 < t1) {
                         const int e_end = d_pre[e + 1];
                         if (e_end <= t0) { ++e; continue; }
@@ -461,21 +488,6 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
                 }
                 __syncthreads();
             }
-        } else {
-            // short B rows: one lane per A entry
-            for (i64 p = e_lo + tid; p < e_hi; p += DN_THREADS) {
-                const int k = __ldg(A.crd + p);
-                if ((unsigned)k >= (unsigned)B.nrows) continue;
-                const i64 qs = __ldg(B.pos + k);
-                const int len = (int)(__ldg(B.pos + k + 1) - qs);
-                const T a = __ldg(Aval + p);
-                for (int t = 0; t < len; ++t) {
-                    const unsigned rel0 = (unsigned)(__ldg(B.crd + qs + t) - base);
-                    const T v0 = a * __ldg(Bval + qs + t);
-                    SPWS_DENSE_ADD(rel0, v0)
-                }
-            }
-            __syncthreads();
         }
 #undef SPWS_DENSE_ADD
 
@@ -516,21 +528,27 @@ __global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __re
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
         const i64 out0 = rowptr[row];
         for (int c0 = warp * 4; c0 < nch; c0 += DE_WARPS * 4) {      // four chunks' loads in flight
+            // ranks at the starts of chunks c0 .. c0+4 (lanes 0..4); equal neighbours = empty chunk
+            const int cnt_row = (int)(rowptr[row + 1] - out0);
+            int my_rank = cnt_row;
+            if (lane < 5 && c0 + lane < nch) my_rank = (int)src[nw + c0 + lane];
+            const int next_rank = __shfl_down_sync(0xffffffffu, my_rank, 1);
+            const int my_n = next_rank - my_rank;            // outputs of chunk c0 + lane (lanes 0..3)
             unsigned words[4];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int w = ((c0 + x) << 5) + lane;
-                words[x] = (w < nw) ? src[w] : 0u;
+                const int nx = __shfl_sync(0xffffffffu, my_n, x);
+                words[x] = (w < nw && nx > 0) ? src[w] : 0u;
             }
-            const int my_rank = (lane < 4 && c0 + lane < nch) ? (int)src[nw + c0 + lane] : 0;
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
+                const int n = __shfl_sync(0xffffffffu, my_n, x);
+                const int rank0 = __shfl_sync(0xffffffffu, my_rank, x);
+                if (n <= 0 || c0 + x >= nch) continue;
                 unsigned word = words[x];
                 const int pc = __popc(word);
                 const int incl = warp_incl_scan(pc);
-                const int n = __shfl_sync(0xffffffffu, incl, 31);
-                const int rank0 = __shfl_sync(0xffffffffu, my_rank, x);
-                if (n == 0) continue;
                 int slot = incl - pc;
                 const int col0 = base + (((c0 + x) << 5) + lane << 5);
                 while (word) {
