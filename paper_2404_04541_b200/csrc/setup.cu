@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(256) bin_rows_kernel(int m, RowTables tab, Cla
             if (cls[x] == CLS_DENSE_WARP || cls[x] == CLS_DENSE_HUB || cls[x] == CLS_DENSE_CTA)
             {   // the row's slot: bitmap words, then the rank at the start of every 32-word chunk
                 const int nw = (tab.jmax[row] - tab.jmin[row]) / 32 + 1;
-                words[x] = nw + (nw + 31) / 32;
+                words[x] = (nw + (nw + 31) / 32 + 3) & ~3;      // 16-byte aligned slots
             }
             my_words += words[x];
         }

@@ -163,7 +163,7 @@ size_t rest_reserve(const spws_plan_s* p, int64_t m, int64_t ncols) {
     if (p->policy != SPWS_SPARSE_ISM) {
         const int64_t span_cap = ncols < p->opt.dense_max_span ? ncols : p->opt.dense_max_span;
         const size_t nw = (size_t)((span_cap + 31) / 32 + 1);
-        bytes += align256((size_t)m * (nw + (nw + 31) / 32) * 4);
+        bytes += align256((size_t)m * ((nw + (nw + 31) / 32 + 3) & ~(size_t)3) * 4);
     }
     if (p->policy != SPWS_DENSE) {
         const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
