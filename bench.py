@@ -35,6 +35,15 @@ WORKLOAD_TEXT = {
     "wide26": "wide-output SpGEMM, A 65536 x 2^26, B 2^26 x 2^26, 4 nnz/row, fp32",
 }
 NOMINAL_HBM_GBS = 8000.0
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per product of the two kernels that
+# dominate the default and the stencil workloads, from the ncu captures summarised under
+# profiles/ (taken on a smaller case of the same recipe where noted; traffic grows in proportion
+# to the products).  Valid only for the kernel source the capture was taken on.
+PROFILED_TRAFFIC = {
+    "num_dense_cta": {"bytes_per_product": 7442280000 / 1079487607, "source": "profiles/dense_num_cta_kernel_rmat17.md"},
+    "num_dense_warp": {"bytes_per_product": 1201252352 / 181321496, "source": "profiles/dense_num_warp_kernel_stencil64.md"},
+}
+PROFILED_SOURCE_SHA = "421aaa839f7799fa"   # sha256 prefix of csrc/dense.cu at capture time
 
 
 def algorithmic_bytes(m, nnzA, products, nnzC, V):
@@ -273,19 +282,30 @@ def main():
                    "ism_global": (pc[7], nc[7])}
     kname = top.split("_", 1)[1]
     if top == "num_dense_warp":
-        gp, gn = dw_p, dw_n
-    elif top == "num_dense_cta":
-        gp, gn = dense_p - dw_p, dense_n - dw_n
+        kbytes = dw_p * (4 + V) + dw_n * (4 + V)
+    elif top == "num_dense_cta":                    # gathers index + value per product, writes the values
+        kbytes = (dense_p - dw_p) * (4 + V) + (dense_n - dw_n) * V
+    elif top == "num_dense_emit":                   # writes the coordinates
+        kbytes = (dense_n - dw_n) * 4
+    elif top == "num_dense_zero":
+        kbytes = 0
     elif top == "sym_dense_warp":
-        gp, gn = pc[4], nc[4]
+        kbytes = pc[4] * 4
     elif top == "sym_dense_cta":
-        gp, gn = pc[5] + pc[6], nc[5] + nc[6]
+        kbytes = (pc[5] + pc[6]) * 4
     else:
         gp, gn = group_units.get(kname, (0, 0))
-    kbytes = gp * (4 + V) + gn * (4 + V) if top.startswith("num_") else gp * 4
+        kbytes = gp * (4 + V) + gn * (4 + V) if top.startswith("num_") else gp * 4
+    kunits = {"num_dense_cta": dense_p - dw_p, "num_dense_warp": dw_p}.get(top, 0)
+    traffic = None
+    if top in PROFILED_TRAFFIC and kunits:
+        import hashlib
+        src = os.path.join(ROOT, "paper_2404_04541_b200", "csrc", "dense.cu")
+        if hashlib.sha256(open(src, "rb").read()).hexdigest().startswith(PROFILED_SOURCE_SHA):
+            traffic = PROFILED_TRAFFIC[top]["bytes_per_product"] * kunits
     achieved = kbytes / (avg[top] * 1e-3) / 1e9 if avg[top] > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                 "kernel_ms": avg[top], "algorithmic_bytes": kbytes}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -142,9 +142,11 @@ enum {
     SPWS_T_NUM_ISM_SMEM_S = 10,
     SPWS_T_NUM_ISM_SMEM = 11,
     SPWS_T_NUM_DENSE_WARP = 12,
-    SPWS_T_NUM_DENSE_CTA = 13,
-    SPWS_T_NUM_ISM_GLOBAL = 14,
-    SPWS_T_COUNT = 15
+    SPWS_T_NUM_DENSE_ZERO = 13, /* clears the value segments the CTA dense kernel adds into        */
+    SPWS_T_NUM_DENSE_CTA = 14,
+    SPWS_T_NUM_DENSE_EMIT = 15, /* coordinates of the CTA dense rows                               */
+    SPWS_T_NUM_ISM_GLOBAL = 16,
+    SPWS_T_COUNT = 17
 };
 
 spws_status_t spws_create(spws_handle_t* handle);

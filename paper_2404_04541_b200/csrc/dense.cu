@@ -614,8 +614,8 @@ cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, 
 }
 
 template <typename T>
-static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, i64 total_products, const Csr& A, const Csr& B,
-                             const i64* rowptr, int* Ccrd, void* Cval) {
+static cudaError_t num_cta_t(const LaunchCtx& c, int phase, int n_units_host, int words, i64 total_products, const Csr& A,
+                             const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
     const i64 unit_products = dense_unit_products(total_products);
     const size_t smem = ((sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32 + 1) * 4 + (size_t)words * 2 + 15) & ~(size_t)15) +
@@ -625,20 +625,23 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int n_units_host, int words, i6
     auto k = dense_num_cta_kernel<T>;
     if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DN_THREADS, smem)) != cudaSuccess) return e;
-    dense_zero_kernel<T><<<persistent_grid(c, 8, n_units_host), 256, 0, c.stream>>>(c.ctl, CAP, unit_products, c.tab, rowptr, (T*)Cval);
-    k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab, rowptr,
-                                                                             Ccrd, (T*)Cval);
-    dense_emit_crd_kernel<<<persistent_grid(c, 8, n_units_host), DE_THREADS, 0, c.stream>>>(c.ctl, c.tab, rowptr, Ccrd);
-    c.launches += 3;
+    if (phase == 0)
+        dense_zero_kernel<T><<<persistent_grid(c, 8, n_units_host), 256, 0, c.stream>>>(c.ctl, CAP, unit_products, c.tab, rowptr, (T*)Cval);
+    else if (phase == 1)
+        k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab,
+                                                                                 rowptr, Ccrd, (T*)Cval);
+    else
+        dense_emit_crd_kernel<<<persistent_grid(c, 8, n_units_host), DE_THREADS, 0, c.stream>>>(c.ctl, c.tab, rowptr, Ccrd);
+    ++c.launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_dense_num_cta(const LaunchCtx& c, int n_units_host, int max_span_words, i64 total_products,
+cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host, int max_span_words, i64 total_products,
                                  const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
     int words = max_span_words > 0 ? max_span_words : c.dense_smem_words;
     words = (words + 31) & ~31;
-    return c.is_f64 ? num_cta_t<double>(c, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval)
-                    : num_cta_t<float>(c, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval);
+    return c.is_f64 ? num_cta_t<double>(c, phase, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval)
+                    : num_cta_t<float>(c, phase, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval);
 }
 
 }  // namespace spws

@@ -550,8 +550,12 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         mark(plan, SPWS_T_NUM_DENSE_WARP);
     }
     if (s.dense_units > 0) {
-        CUDA_TRY(launch_dense_num_cta(c, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
+        CUDA_TRY(launch_dense_num_cta(c, 0, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
+        mark(plan, SPWS_T_NUM_DENSE_ZERO);
+        CUDA_TRY(launch_dense_num_cta(c, 1, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_DENSE_CTA);
+        CUDA_TRY(launch_dense_num_cta(c, 2, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
+        mark(plan, SPWS_T_NUM_DENSE_EMIT);
     }
     if (s.rows_per_class[CLS_ISM_GLOBAL] > 0) {
         CUDA_TRY(launch_ism_global(c, true, (int)s.rows_per_class[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));
