@@ -8,18 +8,23 @@ namespace spws {
 typedef long long i64;
 typedef unsigned long long u64;
 
-constexpr int NCLASS = 8;
+constexpr int NCLASS = 10;
 // Row classes = the workspace a row (or (i,j) fibre) is routed to in the symbolic pass.
 enum RowClass : int {
     CLS_EMPTY = 0,      // no intermediate product
-    CLS_ISM_REG = 1,    // insert-sort-merge in registers, one lane group per row
-    CLS_ISM_SMEM_S = 2, // insert-sort-merge in shared memory, small CTA
-    CLS_ISM_SMEM = 3,   // insert-sort-merge in shared memory, full CTA
-    CLS_DENSE_WARP = 4, // dense workspace (occupancy bitmap), one warp per row
-    CLS_DENSE_HUB = 5,  // dense workspace, one CTA per row, heaviest rows (scheduled first)
-    CLS_DENSE_CTA = 6,  // dense workspace, one CTA per row
-    CLS_ISM_GLOBAL = 7  // accumulation array in shared memory, all array in global memory
+    CLS_ISM_REG8 = 1,   // insert-sort-merge in registers, 8 lanes per row (<= 8 products)
+    CLS_ISM_REG16 = 2,  // ... 16 lanes per row (<= 16 products)
+    CLS_ISM_REG = 3,    // ... one warp per row (<= 32 products)
+    CLS_ISM_SMEM_S = 4, // insert-sort-merge in shared memory, small CTA
+    CLS_ISM_SMEM = 5,   // insert-sort-merge in shared memory, full CTA
+    CLS_DENSE_WARP = 6, // dense workspace (occupancy bitmap), one warp per row
+    CLS_DENSE_HUB = 7,  // dense workspace, one CTA per row, heaviest rows (scheduled first)
+    CLS_DENSE_CTA = 8,  // dense workspace, one CTA per row
+    CLS_ISM_GLOBAL = 9  // accumulation array in shared memory, all array in global memory
 };
+constexpr int NUM_SLOT = 16;   // work_counter[cls] in the symbolic pass, work_counter[NUM_SLOT + cls] in the numeric pass
+// index of a class in the public statistics (the three register classes are reported as one)
+__host__ __device__ inline int public_class(int cls) { return cls == 0 ? 0 : (cls <= 3 ? 1 : cls - 2); }
 
 // Capacities fixed at compile time.
 constexpr int DENSE_WARP_BM_WORDS = 1024;  // bitmap words a warp-per-row workspace may span (32768 columns)
@@ -50,7 +55,7 @@ struct DevCtl {
     int max_span_words;     // widest bitmap among CTA-class dense rows
     int class_count[NCLASS];
     int class_cursor[NCLASS];
-    int work_counter[16];   // dynamic work distribution; cleared before each pass
+    int work_counter[32];   // dynamic work distribution; cleared before each pass
     i64 class_products[NCLASS];
     i64 class_nnz[NCLASS];
     i64 dense_warp_products, dense_warp_nnz;   // share of the dense rows the warp numeric kernel takes
@@ -182,7 +187,7 @@ cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64*
                                const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
                                i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2);
 // class kernels: n_host < 0 means "size the grid for any count"
-cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                            const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_ism_smem(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                             const i64* rowptr, int* Ccrd, void* Cval);

@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
     const T* __restrict__ Bval = (const T*)B.val;
     for (;;) {
         int r = 0;
-        if (lane == 0) r = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_WARP], 1);
+        if (lane == 0) r = atomicAdd(&ctl->work_counter[NUM_SLOT + CLS_DENSE_WARP], 1);
         r = __shfl_sync(0xffffffffu, r, 0);
         if (r >= n) break;
         const int row = tab.warp_rows[r];
@@ -351,7 +351,7 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
 
     for (;;) {
         __syncthreads();
-        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[8 + CLS_DENSE_CTA], 1);
+        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[NUM_SLOT + CLS_DENSE_CTA], 1);
         __syncthreads();
         const int u = s_next;
         if (u >= n_units) break;

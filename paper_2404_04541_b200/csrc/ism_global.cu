@@ -246,7 +246,7 @@ static cudaError_t launch_t(const LaunchCtx& c, bool numeric, int n_host, const 
                             const i64* rowptr, int* Ccrd, void* Cval) {
     const size_t smem = sizeof(u64) * GL_CAPMAX + sizeof(T) * GL_CAPMAX * 2 + sizeof(i64) * GL_THREADS + sizeof(T) * GL_THREADS +
                         sizeof(int) * (3 * GL_CAPMAX + 1 + GL_THREADS + 1 + 33) + 16;
-    const int slot = CLS_ISM_GLOBAL + (numeric ? 8 : 0);
+    const int slot = CLS_ISM_GLOBAL + (numeric ? NUM_SLOT : 0);
     cudaError_t e;
     i64 grid = (i64)c.sm_count * 2;
     if (n_host >= 0 && n_host < grid) grid = n_host > 0 ? n_host : 1;

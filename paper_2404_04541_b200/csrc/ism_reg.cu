@@ -11,12 +11,12 @@
 namespace spws {
 
 template <typename T, int G, bool NUMERIC>
-__global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ perm, const DevCtl* __restrict__ ctl,
+__global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ perm, const DevCtl* __restrict__ ctl, int cls,
                                                       Csr A, Csr B, const int* __restrict__ jmin, int* __restrict__ cnt,
                                                       const i64* __restrict__ rowptr, int* __restrict__ Ccrd, T* __restrict__ Cval) {
     if (ctl->status != 0) return;
     int off, n;
-    class_range(ctl, CLS_ISM_REG, off, n);
+    class_range(ctl, cls, off, n);
     const int* __restrict__ rows = perm + off;
     const unsigned lane = threadIdx.x & 31;
     const int gl = threadIdx.x % G;
@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ pe
 }
 
 template <typename T, int G>
-static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                             const i64* rowptr, int* Ccrd, void* Cval) {
     const int threads = 256;
     i64 groups = (n_host >= 0) ? n_host : A.nrows;
@@ -123,26 +123,25 @@ static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int n_host, const 
     int grid = (int)(want < cap ? want : cap);
     if (grid < 1) grid = 1;
     if (numeric)
-        ism_reg_kernel<T, G, true><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, A, B,
+        ism_reg_kernel<T, G, true><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, cls, A, B,
                                                                  c.tab.jmin, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     else
-        ism_reg_kernel<T, G, false><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, A, B,
+        ism_reg_kernel<T, G, false><<<grid, threads, 0, c.stream>>>(c.tab.perm, c.ctl, cls, A, B,
                                                                   c.tab.jmin, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     ++c.launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
+cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                            const i64* rowptr, int* Ccrd, void* Cval) {
-    const int cap = c.prm.reg_cap;
     if (c.is_f64) {
-        if (cap <= 8) return launch_g<double, 8>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
-        if (cap <= 16) return launch_g<double, 16>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
-        return launch_g<double, 32>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+        if (cls == CLS_ISM_REG8) return launch_g<double, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
+        if (cls == CLS_ISM_REG16) return launch_g<double, 16>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
+        return launch_g<double, 32>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
     }
-    if (cap <= 8) return launch_g<float, 8>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
-    if (cap <= 16) return launch_g<float, 16>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
-    return launch_g<float, 32>(c, numeric, n_host, A, B, rowptr, Ccrd, Cval);
+    if (cls == CLS_ISM_REG8) return launch_g<float, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
+    if (cls == CLS_ISM_REG16) return launch_g<float, 16>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
+    return launch_g<float, 32>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
 }
 
 }  // namespace spws

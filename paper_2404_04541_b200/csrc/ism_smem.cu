@@ -133,7 +133,7 @@ template <typename T, int CAP, int THREADS>
 static cudaError_t launch_cap(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                               const i64* rowptr, int* Ccrd, void* Cval) {
     const size_t smem = smem_bytes<T, CAP, THREADS>(numeric);
-    const int slot = cls + (numeric ? 8 : 0);
+    const int slot = cls + (numeric ? NUM_SLOT : 0);
     cudaError_t e;
     int per_sm = 0;
     if (numeric) {

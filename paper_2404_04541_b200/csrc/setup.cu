@@ -55,15 +55,16 @@ __device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const Cl
         if (!dense_ok) { raise_status(ctl, DEV_WORKSPACE_TOO_LARGE); return CLS_EMPTY; }
         return dense_class(ub, span_words);
     }
+    const int reg_cls = ub <= 8 ? CLS_ISM_REG8 : (ub <= 16 ? CLS_ISM_REG16 : CLS_ISM_REG);
     if (prm.policy == 1) {                       // sparse ISM forced
-        if (reg_ok) return CLS_ISM_REG;
+        if (reg_ok) return reg_cls;
         if (ub <= prm.smem_small_cap) return CLS_ISM_SMEM_S;
         if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
         return CLS_ISM_GLOBAL;
     }
     // auto: few products -> sort them in registers; a bitmap that is small next to the work ->
     // dense; mid-size rows -> shared-memory ISM; long rows -> dense; otherwise global ISM.
-    if (reg_ok) return CLS_ISM_REG;
+    if (reg_ok) return reg_cls;
     if (dense_ok && (float)span_words <= prm.span_words_per_product * (float)ub) return dense_class(ub, span_words);
     if (ub <= prm.smem_small_cap) return CLS_ISM_SMEM_S;
     if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
@@ -305,17 +306,22 @@ cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr) {
     return cudaGetLastError();
 }
 
-// Output entries per class (statistics for the per-kernel byte counts).
+// Output entries per class (statistics for the per-kernel byte counts).  Rows are grouped by
+// class in perm, so each class is one contiguous range: sum it with a grid-stride loop and one
+// atomic per warp.
 __global__ void __launch_bounds__(256) class_nnz_kernel(int m, RowTables tab, DevCtl* ctl) {
-    __shared__ i64 s_nnz[NCLASS];
-    if (threadIdx.x < NCLASS) s_nnz[threadIdx.x] = 0;
-    __syncthreads();
-    for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < m; r += (i64)gridDim.x * blockDim.x) {
-        const int c = tab.cnt[r];
-        if (c) atomicAdd((u64*)&s_nnz[tab.cls[r]], (u64)c);
+    int off = 0;
+    for (int c = 0; c < NCLASS; ++c) {
+        const int n = ctl->class_count[c];
+        if (c != CLS_EMPTY && n > 0) {
+            i64 sum = 0;
+            for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += (i64)gridDim.x * blockDim.x)
+                sum += tab.cnt[tab.perm[off + r]];
+            for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+            if ((threadIdx.x & 31) == 0 && sum) atomicAdd((u64*)&ctl->class_nnz[c], (u64)sum);
+        }
+        off += n;
     }
-    __syncthreads();
-    if (threadIdx.x < NCLASS && s_nnz[threadIdx.x]) atomicAdd((u64*)&ctl->class_nnz[threadIdx.x], (u64)s_nnz[threadIdx.x]);
 }
 
 cudaError_t launch_class_nnz(const LaunchCtx& c, int m) {

@@ -31,6 +31,7 @@ struct spws_plan_s {
     int64_t m = 0;
     void* scratch = nullptr;
     int max_span_words = 0;     // widest dense bitmap of the last symbolic pass
+    int64_t bin_rows[NCLASS] = {};  // rows per internal class of the last symbolic pass
     // optional per-kernel timing: ev[g] is recorded after group g; ev_start[] before each pass
     bool profiling = false;
     cudaEvent_t ev[SPWS_T_COUNT] = {};
@@ -445,7 +446,9 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<i64*>(sc + L.rowptr_raw);
     if (S.m > 0) {
         if (plan->policy != SPWS_DENSE) {
-            CUDA_TRY(launch_ism_reg(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG8, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG16, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG, -1, S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_REG);
             CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_SMEM_S);
@@ -485,9 +488,10 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     plan->stats.nnz = hc.nnz;
     plan->stats.max_row_products = hc.max_ub;
     for (int k = 0; k < NCLASS; ++k) {
-        plan->stats.rows_per_class[k] = hc.class_count[k];
-        plan->stats.products_per_class[k] = hc.class_products[k];
-        plan->stats.nnz_per_class[k] = hc.class_nnz[k];
+        plan->bin_rows[k] = hc.class_count[k];
+        plan->stats.rows_per_class[public_class(k)] += hc.class_count[k];
+        plan->stats.products_per_class[public_class(k)] += hc.class_products[k];
+        plan->stats.nnz_per_class[public_class(k)] += hc.class_nnz[k];
     }
     plan->stats.dense_units = hc.n_units;
     plan->stats.dense_warp_rows = hc.n_warp_rows;
@@ -533,16 +537,18 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     mark_start(plan, 1);
     const spws_stats_t& s = plan->stats;
     int* crd = C->crd[last];
-    if (s.rows_per_class[CLS_ISM_REG] > 0) {
-        CUDA_TRY(launch_ism_reg(c, true, (int)s.rows_per_class[CLS_ISM_REG], S.A, S.B, rowptr, crd, C->val));
-        mark(plan, SPWS_T_NUM_ISM_REG);
-    }
-    if (s.rows_per_class[CLS_ISM_SMEM_S] > 0) {
-        CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM_S, (int)s.rows_per_class[CLS_ISM_SMEM_S], S.A, S.B, rowptr, crd, C->val));
+    const int64_t* bins = plan->bin_rows;
+    for (int cls = CLS_ISM_REG8; cls <= CLS_ISM_REG; ++cls)
+        if (bins[cls] > 0) {
+            CUDA_TRY(launch_ism_reg(c, true, cls, (int)bins[cls], S.A, S.B, rowptr, crd, C->val));
+            mark(plan, SPWS_T_NUM_ISM_REG);
+        }
+    if (bins[CLS_ISM_SMEM_S] > 0) {
+        CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM_S, (int)bins[CLS_ISM_SMEM_S], S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_ISM_SMEM_S);
     }
-    if (s.rows_per_class[CLS_ISM_SMEM] > 0) {
-        CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM, (int)s.rows_per_class[CLS_ISM_SMEM], S.A, S.B, rowptr, crd, C->val));
+    if (bins[CLS_ISM_SMEM] > 0) {
+        CUDA_TRY(launch_ism_smem(c, true, CLS_ISM_SMEM, (int)bins[CLS_ISM_SMEM], S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_ISM_SMEM);
     }
     if (s.dense_warp_rows > 0) {
@@ -557,8 +563,8 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         CUDA_TRY(launch_dense_num_cta(c, 2, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_DENSE_EMIT);
     }
-    if (s.rows_per_class[CLS_ISM_GLOBAL] > 0) {
-        CUDA_TRY(launch_ism_global(c, true, (int)s.rows_per_class[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));
+    if (bins[CLS_ISM_GLOBAL] > 0) {
+        CUDA_TRY(launch_ism_global(c, true, (int)bins[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_ISM_GLOBAL);
     }
     plan->stats.launches_numeric = c.launches;
