@@ -310,7 +310,8 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 constexpr int DN_ENTRIES = 1024;     // A entries whose descriptors are staged per round
 constexpr int DN_TILE = 256;         // products a warp takes per fetch
 
-// zero the part of the value segment that units add into
+// Zero the value segments of the rows that several units add into (a row with a single unit
+// clears its own overflow part inside the accumulate kernel).
 template <typename T>
 __global__ void __launch_bounds__(256) dense_zero_kernel(DevCtl* __restrict__ ctl, int CAP, i64 unit_products, RowTables tab,
                                                          const i64* __restrict__ rowptr, T* __restrict__ Cval) {
@@ -319,10 +320,10 @@ __global__ void __launch_bounds__(256) dense_zero_kernel(DevCtl* __restrict__ ct
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
         const int row = tab.unit_row[u];
         if (u != tab.row_unit0[row]) continue;
+        if (dense_units_of_row(tab.ub[row], unit_products) == 1) continue;
         const i64 out0 = rowptr[row];
         const int cnt = (int)(rowptr[row + 1] - out0);
-        const int first = dense_units_of_row(tab.ub[row], unit_products) > 1 ? 0 : CAP;
-        for (int x = first + threadIdx.x; x < cnt; x += 256) Cval[out0 + x] = 0;
+        for (int x = threadIdx.x; x < cnt; x += 256) Cval[out0 + x] = 0;
     }
 }
 
@@ -367,6 +368,8 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const i64 e_lo = ps + (pe - ps) * uidx / nun, e_hi = ps + (pe - ps) * (uidx + 1) / nun;
         T* const gacc = Cval + out0;
+        if (nun == 1)                                   // outputs beyond the shared-memory part start at zero
+            for (int x = CAP + tid; x < cnt; x += DN_THREADS) gacc[x] = 0;
 
         // the row's bitmap, the rank at every chunk start and the rank of every word inside its chunk
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
