@@ -66,16 +66,52 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
         for (int w = lane; w < nw; w += 32) bm[w] = 0;
         __syncwarp();
         const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
-        const int g = lane / gs, gl = lane % gs, ng = 32 / gs;
-        for (i64 p = ps + g; p < pe; p += ng) {
-            const int k = __ldg(A.crd + p);
-            if ((unsigned)k >= (unsigned)B.nrows) continue;
-            const i64 qs = __ldg(B.pos + k);
-            const int len = (int)(__ldg(B.pos + k + 1) - qs);
-            const int* __restrict__ ck = B.crd + qs;
-            for (int t = gl; t < len; t += gs) {
-                const unsigned rel = (unsigned)(__ldg(ck + t) - base);
-                if (rel < span) atomicOr(&bm[rel >> 5], 1u << (rel & 31));
+        if (gs == 32) {
+            // descriptors of 32 A entries at a time (one per lane), then the first 32 elements of
+            // four B rows are loaded before any is consumed, to keep loads in flight
+            for (i64 p0 = ps; p0 < pe; p0 += 32) {
+                i64 my_qs = 0;
+                int my_len = 0;
+                if (p0 + lane < pe) {
+                    const int k = __ldg(A.crd + p0 + lane);
+                    if ((unsigned)k < (unsigned)B.nrows) {
+                        my_qs = __ldg(B.pos + k);
+                        my_len = (int)(__ldg(B.pos + k + 1) - my_qs);
+                    }
+                }
+                const int nE = (int)min((i64)32, pe - p0);
+                for (int e = 0; e < nE; e += 4) {
+                    i64 qs[4];
+                    int len[4];
+                    unsigned rel[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        qs[x] = __shfl_sync(0xffffffffu, my_qs, (e + x) & 31);
+                        len[x] = (e + x < nE) ? __shfl_sync(0xffffffffu, my_len, (e + x) & 31) : 0;
+                        rel[x] = (lane < len[x]) ? (unsigned)(__ldg(B.crd + qs[x] + lane) - base) : 0xffffffffu;
+                    }
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        if (rel[x] < span) atomicOr(&bm[rel[x] >> 5], 1u << (rel[x] & 31));
+                        for (int t = lane + 32; t < len[x]; t += 32) {
+                            const unsigned r2 = (unsigned)(__ldg(B.crd + qs[x] + t) - base);
+                            if (r2 < span) atomicOr(&bm[r2 >> 5], 1u << (r2 & 31));
+                        }
+                    }
+                }
+            }
+        } else {
+            const int g = lane / gs, gl = lane % gs, ng = 32 / gs;
+            for (i64 p = ps + g; p < pe; p += ng) {
+                const int k = __ldg(A.crd + p);
+                if ((unsigned)k >= (unsigned)B.nrows) continue;
+                const i64 qs = __ldg(B.pos + k);
+                const int len = (int)(__ldg(B.pos + k + 1) - qs);
+                const int* __restrict__ ck = B.crd + qs;
+                for (int t = gl; t < len; t += gs) {
+                    const unsigned rel = (unsigned)(__ldg(ck + t) - base);
+                    if (rel < span) atomicOr(&bm[rel >> 5], 1u << (rel & 31));
+                }
             }
         }
         __syncwarp();

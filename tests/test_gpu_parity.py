@@ -205,6 +205,19 @@ def test_wide_reduced(ctx, oracle_mod, policy):
     check_spgemm(ctx, oracle_mod, c["A"], c["B"], policy)
 
 
+@pytest.mark.parametrize("policy", ["ism", "auto"])
+def test_wide_columns_with_many_products(ctx, oracle_mod, policy):
+    """2^26 columns and rows with hundreds to thousands of products: the shared-memory ISM must
+    sort 64-bit (column, slot) words here (26 column bits + 12 slot bits do not fit 32)."""
+    B = uniform_rows_csr(300, 1 << 26, 24, 21)
+    A = random_csr(80, 300, 0.12, 22, empty_row_frac=0.1)
+    A.val[:] = np.round(A.val * 16) / 16
+    stats = check_spgemm(ctx, oracle_mod, A, B, policy)
+    assert stats["rows_per_class"][2] + stats["rows_per_class"][3] > 0
+    Abig = random_csr(12, 300, 0.6, 23)                               # ~4300 products per row -> beyond 4096
+    check_spgemm(ctx, oracle_mod, Abig, B, policy)
+
+
 def test_dense_policy_refuses_prohibitive_workspace(ctx):
     from paper_2404_04541_b200 import binding
     c = config_inputs("wide26", reduced=True)
