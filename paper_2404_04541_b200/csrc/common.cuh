@@ -193,7 +193,7 @@ cudaError_t launch_ism_smem(const LaunchCtx& c, bool numeric, int cls, int n_hos
                             const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B);
 cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B);
-cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B,
+cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, const Csr& A, const Csr& B,
                                   const i64* rowptr, int* Ccrd, void* Cval);
 // phase 0: clear the value segments units add into; 1: accumulate; 2: write the coordinates
 cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host, int max_span_words, i64 total_products,

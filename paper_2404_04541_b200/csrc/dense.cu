@@ -211,17 +211,18 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
 // numeric, warp per row
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __restrict__ ctl, Csr A, Csr B, RowTables tab,
+__global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __restrict__ ctl, int bmw, Csr A, Csr B, RowTables tab,
                                                                     const i64* __restrict__ rowptr, int* __restrict__ Ccrd,
                                                                     T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (ctl->status != 0) return;
     const int n = ctl->n_warp_rows;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // per warp: DENSE_WARP_ACC values, bmw bitmap words, bmw word ranks (bmw = widest row of this launch)
     T* acc = reinterpret_cast<T*>(smem_raw) + warp * DENSE_WARP_ACC;
-    unsigned* bm = reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) + warp * DENSE_WARP_BM_WORDS;
+    unsigned* bm = reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) + warp * bmw;
     unsigned short* pre = reinterpret_cast<unsigned short*>(reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) +
-                                                            DW_WARPS * DENSE_WARP_BM_WORDS) + warp * DENSE_WARP_BM_WORDS;
+                                                            DW_WARPS * bmw) + warp * bmw;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
     for (;;) {
@@ -231,7 +232,7 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         if (r >= n) break;
         const int row = tab.warp_rows[r];
         const int base = tab.jmin[row];
-        const int nw = (tab.jmax[row] - base) / 32 + 1;
+        const int nw = min((tab.jmax[row] - base) / 32 + 1, bmw);
         const unsigned span = (unsigned)nw * 32u;
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const i64 out0 = rowptr[row];
@@ -634,22 +635,25 @@ cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B)
 }
 
 template <typename T>
-static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
+static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, int bmw, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
     int per_sm = 0;
-    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * DENSE_WARP_ACC + 6 * (size_t)DENSE_WARP_BM_WORDS);
+    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * DENSE_WARP_ACC + 6 * (size_t)bmw);
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(dense_num_warp_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_num_warp_kernel<T>, DW_THREADS, smem)) != cudaSuccess) return e;
     const i64 work = n_host >= 0 ? ((i64)n_host + DW_WARPS - 1) / DW_WARPS : -1;
-    dense_num_warp_kernel<T><<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
+    dense_num_warp_kernel<T><<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, bmw, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
     ++c.launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, const Csr& A, const Csr& B,
+cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, const Csr& A, const Csr& B,
                                   const i64* rowptr, int* Ccrd, void* Cval) {
-    return c.is_f64 ? num_warp_t<double>(c, n_host, A, B, rowptr, Ccrd, Cval)
-                    : num_warp_t<float>(c, n_host, A, B, rowptr, Ccrd, Cval);
+    // bitmap words reserved per warp: the widest dense row of this pass, at most the class limit
+    int bmw = max_span_words > 0 ? ((max_span_words + 31) & ~31) : DENSE_WARP_BM_WORDS;
+    if (bmw > DENSE_WARP_BM_WORDS) bmw = DENSE_WARP_BM_WORDS;
+    return c.is_f64 ? num_warp_t<double>(c, n_host, bmw, A, B, rowptr, Ccrd, Cval)
+                    : num_warp_t<float>(c, n_host, bmw, A, B, rowptr, Ccrd, Cval);
 }
 
 template <typename T>

@@ -552,7 +552,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         mark(plan, SPWS_T_NUM_ISM_SMEM);
     }
     if (s.dense_warp_rows > 0) {
-        CUDA_TRY(launch_dense_num_warp(c, (int)s.dense_warp_rows, S.A, S.B, rowptr, crd, C->val));
+        CUDA_TRY(launch_dense_num_warp(c, (int)s.dense_warp_rows, plan->max_span_words, S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_DENSE_WARP);
     }
     if (s.dense_units > 0) {
