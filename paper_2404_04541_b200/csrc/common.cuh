@@ -52,7 +52,9 @@ struct DevCtl {
     int status;
     int n_units;            // numeric dense CTA units (row, rank range)
     int n_warp_rows;        // numeric dense warp rows
-    int max_span_words;     // widest bitmap among CTA-class dense rows
+    int max_span_words;     // widest bitmap among the dense rows
+    int max_warp_cnt;       // most outputs of a row the warp numeric kernel takes
+    int pad_;
     int class_count[NCLASS];
     int class_cursor[NCLASS];
     int work_counter[32];   // dynamic work distribution; cleared before each pass
@@ -193,7 +195,7 @@ cudaError_t launch_ism_smem(const LaunchCtx& c, bool numeric, int cls, int n_hos
                             const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B);
 cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B);
-cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, const Csr& A, const Csr& B,
+cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, int max_cnt, const Csr& A, const Csr& B,
                                   const i64* rowptr, int* Ccrd, void* Cval);
 // phase 0: clear the value segments units add into; 1: accumulate; 2: write the coordinates
 cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host, int max_span_words, i64 total_products,

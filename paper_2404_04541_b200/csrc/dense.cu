@@ -211,17 +211,17 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
 // numeric, warp per row
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __restrict__ ctl, int bmw, Csr A, Csr B, RowTables tab,
+__global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __restrict__ ctl, int bmw, int accw, Csr A, Csr B, RowTables tab,
                                                                     const i64* __restrict__ rowptr, int* __restrict__ Ccrd,
                                                                     T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (ctl->status != 0) return;
     const int n = ctl->n_warp_rows;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // per warp: DENSE_WARP_ACC values, bmw bitmap words, bmw word ranks (bmw = widest row of this launch)
-    T* acc = reinterpret_cast<T*>(smem_raw) + warp * DENSE_WARP_ACC;
-    unsigned* bm = reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) + warp * bmw;
-    unsigned short* pre = reinterpret_cast<unsigned short*>(reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * DENSE_WARP_ACC) +
+    // per warp: accw values, bmw bitmap words, bmw word ranks (the largest / widest row of this launch)
+    T* acc = reinterpret_cast<T*>(smem_raw) + warp * accw;
+    unsigned* bm = reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * accw) + warp * bmw;
+    unsigned short* pre = reinterpret_cast<unsigned short*>(reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * accw) +
                                                             DW_WARPS * bmw) + warp * bmw;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         const unsigned span = (unsigned)nw * 32u;
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const i64 out0 = rowptr[row];
-        const int cnt = (int)(rowptr[row + 1] - out0);
+        const int cnt = min((int)(rowptr[row + 1] - out0), accw);
         // reload the bitmap; rank of each word's first bit = chunk rank + prefix inside the chunk
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
         for (int w0 = 0; w0 < nw; w0 += 32) {
@@ -279,26 +279,26 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                     // entry e
                     if (rel0 < span) {
                         const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a0, v0));
+                        if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a0, v0));
                     }
                     for (int t = lane + 32; t < len0; t += 32) {
                         const unsigned rel = (unsigned)(__ldg(B.crd + qs0 + t) - base);
                         if (rel < span) {
                             const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                            if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a0, __ldg(Bval + qs0 + t)));
+                            if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a0, __ldg(Bval + qs0 + t)));
                         }
                     }
                     __syncwarp();
                     // entry e + 1
                     if (rel1 < span) {
                         const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
-                        if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a1, v1));
+                        if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a1, v1));
                     }
                     for (int t = lane + 32; t < len1; t += 32) {
                         const unsigned rel = (unsigned)(__ldg(B.crd + qs1 + t) - base);
                         if (rel < span) {
                             const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                            if (slot < DENSE_WARP_ACC) acc[slot] = add_rn(acc[slot], mul_rn(a1, __ldg(Bval + qs1 + t)));
+                            if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a1, __ldg(Bval + qs1 + t)));
                         }
                     }
                     __syncwarp();
@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                     const unsigned rel = (unsigned)(__ldg(B.crd + qs + t) - base);
                     if (rel < span) {
                         const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                        if (slot < DENSE_WARP_ACC) atomicAdd(&acc[slot], mul_rn(a, __ldg(Bval + qs + t)));
+                        if (slot < accw) atomicAdd(&acc[slot], mul_rn(a, __ldg(Bval + qs + t)));
                     }
                 }
             }
@@ -635,25 +635,28 @@ cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B)
 }
 
 template <typename T>
-static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, int bmw, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
+static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, int bmw, int accw, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd,
+                              void* Cval) {
     int per_sm = 0;
-    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * DENSE_WARP_ACC + 6 * (size_t)bmw);
+    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * (size_t)accw + 6 * (size_t)bmw);
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(dense_num_warp_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_num_warp_kernel<T>, DW_THREADS, smem)) != cudaSuccess) return e;
     const i64 work = n_host >= 0 ? ((i64)n_host + DW_WARPS - 1) / DW_WARPS : -1;
-    dense_num_warp_kernel<T><<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, bmw, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
+    dense_num_warp_kernel<T><<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, bmw, accw, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
     ++c.launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, const Csr& A, const Csr& B,
+cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, int max_cnt, const Csr& A, const Csr& B,
                                   const i64* rowptr, int* Ccrd, void* Cval) {
     // bitmap words reserved per warp: the widest dense row of this pass, at most the class limit
     int bmw = max_span_words > 0 ? ((max_span_words + 31) & ~31) : DENSE_WARP_BM_WORDS;
     if (bmw > DENSE_WARP_BM_WORDS) bmw = DENSE_WARP_BM_WORDS;
-    return c.is_f64 ? num_warp_t<double>(c, n_host, bmw, A, B, rowptr, Ccrd, Cval)
-                    : num_warp_t<float>(c, n_host, bmw, A, B, rowptr, Ccrd, Cval);
+    int accw = max_cnt > 0 ? ((max_cnt + 31) & ~31) : DENSE_WARP_ACC;     // values reserved per warp
+    if (accw > DENSE_WARP_ACC) accw = DENSE_WARP_ACC;
+    return c.is_f64 ? num_warp_t<double>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval)
+                    : num_warp_t<float>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval);
 }
 
 template <typename T>

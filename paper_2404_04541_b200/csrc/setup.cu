@@ -244,7 +244,7 @@ cudaError_t launch_bin_rows(const LaunchCtx& c, int m) {
 // row's A entries (all units of a row add into the same outputs).
 __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, ClassParams prm, DevCtl* ctl) {
     __shared__ int ws[33];
-    __shared__ int s_wbase, s_ubase;
+    __shared__ int s_wbase, s_ubase, s_wmax;
     __shared__ i64 s_wp, s_wn;
     int off, n4, n5, n6, o5, o6;
     class_range(ctl, CLS_DENSE_WARP, off, n4);
@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
     for (i64 b0 = (i64)blockIdx.x * blockDim.x; b0 < n; b0 += (i64)gridDim.x * blockDim.x) {
         const i64 r = b0 + threadIdx.x;
         int row = -1, cnt = 0, to_warp = 0, nu = 0;
-        if (threadIdx.x == 0) { s_wp = 0; s_wn = 0; }
+        if (threadIdx.x == 0) { s_wp = 0; s_wn = 0; s_wmax = 0; }
         if (r < n) {
             row = tab.perm[off + r];
             cnt = tab.cnt[row];
@@ -276,6 +276,7 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
                 tab.row_unit0[row] = -1;
                 atomicAdd((u64*)&s_wp, (u64)tab.ub[row]);
                 atomicAdd((u64*)&s_wn, (u64)cnt);
+                atomicMax(&s_wmax, cnt);
             } else {
                 const int u0 = s_ubase + upos;
                 if (u0 + nu > prm.unit_cap) {
@@ -291,6 +292,7 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
         if (threadIdx.x == 0 && s_wp) {
             atomicAdd((u64*)&ctl->dense_warp_products, (u64)s_wp);
             atomicAdd((u64*)&ctl->dense_warp_nnz, (u64)s_wn);
+            atomicMax(&ctl->max_warp_cnt, s_wmax);
         }
         __syncthreads();
     }

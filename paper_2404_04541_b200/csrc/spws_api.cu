@@ -31,6 +31,7 @@ struct spws_plan_s {
     int64_t m = 0;
     void* scratch = nullptr;
     int max_span_words = 0;     // widest dense bitmap of the last symbolic pass
+    int max_warp_cnt = 0;       // most outputs of a warp-numeric row
     int64_t bin_rows[NCLASS] = {};  // rows per internal class of the last symbolic pass
     // optional per-kernel timing: ev[g] is recorded after group g; ev_start[] before each pass
     bool profiling = false;
@@ -499,6 +500,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     plan->stats.dense_warp_nnz = hc.dense_warp_nnz;
     plan->stats.bitmap_bytes = (int64_t)hc.bm_words_used * 4;
     plan->max_span_words = hc.max_span_words;
+    plan->max_warp_cnt = hc.max_warp_cnt;
     plan->stats.launches_symbolic = c.launches;
     if (plan->kind == 0) {
         C->n[0] = C->dims[0];
@@ -552,7 +554,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         mark(plan, SPWS_T_NUM_ISM_SMEM);
     }
     if (s.dense_warp_rows > 0) {
-        CUDA_TRY(launch_dense_num_warp(c, (int)s.dense_warp_rows, plan->max_span_words, S.A, S.B, rowptr, crd, C->val));
+        CUDA_TRY(launch_dense_num_warp(c, (int)s.dense_warp_rows, plan->max_span_words, plan->max_warp_cnt, S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_DENSE_WARP);
     }
     if (s.dense_units > 0) {
