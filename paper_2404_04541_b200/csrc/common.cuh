@@ -23,6 +23,7 @@ enum RowClass : int {
     CLS_ISM_GLOBAL = 9  // accumulation array in shared memory, all array in global memory
 };
 constexpr int NUM_SLOT = 16;   // work_counter[cls] in the symbolic pass, work_counter[NUM_SLOT + cls] in the numeric pass
+constexpr int EMIT_SLOT = 30;  // work_counter slot of the coordinate emission of the CTA dense route
 // index of a class in the public statistics (the three register classes are reported as one)
 __host__ __device__ inline int public_class(int cls) { return cls == 0 ? 0 : (cls <= 3 ? 1 : cls - 2); }
 

@@ -559,7 +559,14 @@ __global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __re
     const int n_units = ctl->n_units;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int* stage = s_stage[warp];
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    __shared__ int s_u;
+    for (;;) {                                          // rows differ a lot in set bits: deal them out dynamically
+        __syncthreads();
+        if (threadIdx.x == 0) s_u = atomicAdd(&ctl->work_counter[EMIT_SLOT], 4);
+        __syncthreads();
+        const int u_first = s_u;
+        if (u_first >= n_units) break;
+      for (int u = u_first; u < min(n_units, u_first + 4); ++u) {
         const int row = tab.unit_row[u];
         if (u != tab.row_unit0[row]) continue;
         const int base = tab.jmin[row];
@@ -602,6 +609,7 @@ __global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __re
                 __syncwarp();
             }
         }
+      }
     }
 }
 
@@ -676,8 +684,12 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int phase, int n_units_host, in
     else if (phase == 1)
         k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab,
                                                                                  rowptr, Ccrd, (T*)Cval);
-    else
-        dense_emit_crd_kernel<<<persistent_grid(c, 8, n_units_host), DE_THREADS, 0, c.stream>>>(c.ctl, c.tab, rowptr, Ccrd);
+    else {
+        // rows are dealt out by grid stride, so the grid must be exactly what is resident at once
+        int emit_per_sm = 0;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&emit_per_sm, dense_emit_crd_kernel, DE_THREADS, 0)) != cudaSuccess) return e;
+        dense_emit_crd_kernel<<<persistent_grid(c, emit_per_sm, n_units_host), DE_THREADS, 0, c.stream>>>(c.ctl, c.tab, rowptr, Ccrd);
+    }
     ++c.launches;
     return cudaGetLastError();
 }
