@@ -546,27 +546,27 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
     }
 }
 
-// Coordinates of the CTA-unit rows: a warp expands one 32-word chunk of the saved bitmap at a
-// time (its outputs are the contiguous range that starts at the chunk's saved rank) into a small
-// shared-memory stage and stores it with contiguous writes.
+// Coordinates of the CTA-unit rows.  A warp takes a row at a time and walks its saved bitmap in
+// groups of four 32-word chunks; the outputs of a group are the contiguous range that starts at
+// the first chunk's saved rank, so the group is expanded into a small shared-memory stage and
+// stored with contiguous writes.  The loads of the next group (and the ranks of the one after)
+// are issued before the current group is expanded.
 constexpr int DE_THREADS = 256;
 constexpr int DE_WARPS = DE_THREADS / 32;
+constexpr int DE_STAGE = 1024;       // coordinates a warp stages at once (one full chunk)
 
 __global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __restrict__ ctl, RowTables tab,
                                                                     const i64* __restrict__ rowptr, int* __restrict__ Ccrd) {
-    __shared__ int s_stage[DE_WARPS][1024];
+    __shared__ int s_stage[DE_WARPS][DE_STAGE];
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int* stage = s_stage[warp];
-    __shared__ int s_u;
     for (;;) {                                          // rows differ a lot in set bits: deal them out dynamically
-        __syncthreads();
-        if (threadIdx.x == 0) s_u = atomicAdd(&ctl->work_counter[EMIT_SLOT], 4);
-        __syncthreads();
-        const int u_first = s_u;
-        if (u_first >= n_units) break;
-      for (int u = u_first; u < min(n_units, u_first + 4); ++u) {
+        int u = 0;
+        if (lane == 0) u = atomicAdd(&ctl->work_counter[EMIT_SLOT], 1);
+        u = __shfl_sync(0xffffffffu, u, 0);
+        if (u >= n_units) break;
         const int row = tab.unit_row[u];
         if (u != tab.row_unit0[row]) continue;
         const int base = tab.jmin[row];
@@ -574,42 +574,70 @@ __global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __re
         const int nch = chunks_of(nw);
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
         const i64 out0 = rowptr[row];
-        for (int c0 = warp * 4; c0 < nch; c0 += DE_WARPS * 4) {      // four chunks' loads in flight
-            // ranks at the starts of chunks c0 .. c0+4 (lanes 0..4); equal neighbours = empty chunk
-            const int cnt_row = (int)(rowptr[row + 1] - out0);
-            int my_rank = cnt_row;
-            if (lane < 5 && c0 + lane < nch) my_rank = (int)src[nw + c0 + lane];
-            const int next_rank = __shfl_down_sync(0xffffffffu, my_rank, 1);
-            const int my_n = next_rank - my_rank;            // outputs of chunk c0 + lane (lanes 0..3)
-            unsigned words[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int w = ((c0 + x) << 5) + lane;
-                const int nx = __shfl_sync(0xffffffffu, my_n, x);
-                words[x] = (w < nw && nx > 0) ? src[w] : 0u;
-            }
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int n = __shfl_sync(0xffffffffu, my_n, x);
-                const int rank0 = __shfl_sync(0xffffffffu, my_rank, x);
-                if (n <= 0 || c0 + x >= nch) continue;
-                unsigned word = words[x];
-                const int pc = __popc(word);
-                const int incl = warp_incl_scan(pc);
-                int slot = incl - pc;
-                const int col0 = base + (((c0 + x) << 5) + lane << 5);
-                while (word) {
-                    const int b = __ffs(word) - 1;
-                    word &= word - 1;
-                    stage[slot++] = col0 + b;
+        const int cnt_row = (int)(rowptr[row + 1] - out0);
+
+        // lanes 0..4 hold the ranks at the starts of chunks c0 .. c0+4 (the row's count past the end)
+        auto load_ranks = [&](int c0) {
+            int r = cnt_row;
+            if (lane < 5 && c0 + lane < nch) r = (int)src[nw + c0 + lane];
+            return r;
+        };
+        // word `lane` of chunk c0+x unless that chunk is empty (equal ranks at both ends)
+        auto load_word = [&](int c0, int x, int ranks) {
+            const int n = __shfl_sync(0xffffffffu, ranks, x + 1) - __shfl_sync(0xffffffffu, ranks, x);
+            const int w = ((c0 + x) << 5) + lane;
+            return (w < nw && n > 0) ? src[w] : 0u;
+        };
+        int rk = load_ranks(0);
+        unsigned w0 = load_word(0, 0, rk), w1 = load_word(0, 1, rk), w2 = load_word(0, 2, rk), w3 = load_word(0, 3, rk);
+        int rk_next = load_ranks(4);
+        for (int c0 = 0; c0 < nch; c0 += 4) {
+            const unsigned n0 = load_word(c0 + 4, 0, rk_next), n1 = load_word(c0 + 4, 1, rk_next);
+            const unsigned n2 = load_word(c0 + 4, 2, rk_next), n3 = load_word(c0 + 4, 3, rk_next);
+            const int rk_next2 = load_ranks(c0 + 8);
+
+            const int r0 = __shfl_sync(0xffffffffu, rk, 0);
+            const int n_all = __shfl_sync(0xffffffffu, rk, 4) - r0;
+            if (n_all > 0) {
+                // exclusive ranks of the four words of this lane inside their chunks: two scans of
+                // two 16-bit counts each
+                const int p0 = __popc(w0), p1 = __popc(w1), p2 = __popc(w2), p3 = __popc(w3);
+                const unsigned sa = (unsigned)warp_incl_scan(p0 | (p1 << 16)), sb = (unsigned)warp_incl_scan(p2 | (p3 << 16));
+                const int e0 = (int)(sa & 0xffffu) - p0, e1 = (int)(sa >> 16) - p1;
+                const int e2 = (int)(sb & 0xffffu) - p2, e3 = (int)(sb >> 16) - p3;
+                const int col = base + (((c0 << 5) + lane) << 5);
+                auto expand = [&](unsigned word, int slot, int col0) {
+                    while (word) {
+                        const int b = __ffs(word) - 1;
+                        word &= word - 1;
+                        stage[slot++] = col0 + b;
+                    }
+                };
+                auto flush = [&](int rank0, int n) {
+                    __syncwarp();
+                    const i64 o = out0 + rank0;
+                    for (int y = lane; y < n; y += 32) Ccrd[o + y] = stage[y];
+                    __syncwarp();
+                };
+                if (n_all <= DE_STAGE) {
+                    expand(w0, e0, col);
+                    expand(w1, __shfl_sync(0xffffffffu, rk, 1) - r0 + e1, col + 1024);
+                    expand(w2, __shfl_sync(0xffffffffu, rk, 2) - r0 + e2, col + 2048);
+                    expand(w3, __shfl_sync(0xffffffffu, rk, 3) - r0 + e3, col + 3072);
+                    flush(r0, n_all);
+                } else {
+                    const int r1 = __shfl_sync(0xffffffffu, rk, 1), r2 = __shfl_sync(0xffffffffu, rk, 2);
+                    const int r3 = __shfl_sync(0xffffffffu, rk, 3), r4 = r0 + n_all;
+                    expand(w0, e0, col);        flush(r0, r1 - r0);
+                    expand(w1, e1, col + 1024); flush(r1, r2 - r1);
+                    expand(w2, e2, col + 2048); flush(r2, r3 - r2);
+                    expand(w3, e3, col + 3072); flush(r3, r4 - r3);
                 }
-                __syncwarp();
-                const i64 o = out0 + rank0;
-                for (int y = lane; y < n; y += 32) Ccrd[o + y] = stage[y];
-                __syncwarp();
             }
+            w0 = n0; w1 = n1; w2 = n2; w3 = n3;
+            rk = rk_next;
+            rk_next = rk_next2;
         }
-      }
     }
 }
 
