@@ -96,7 +96,7 @@ typedef struct {
                                  segment in global memory), power of two in [64, 8192];
                                  default 4096                                                      */
     int32_t dense_max_span;   /* widest column span (jmax - jmin + 1) a dense workspace may cover,
-                                 in [32, 2^20]; default 2^20.  Wider rows go to ISM (AUTO) or
+                                 in [32, 2^19]; default 2^19.  Wider rows go to ISM (AUTO) or
                                  fail with SPWS_WORKSPACE_TOO_LARGE (DENSE)                       */
     int32_t fallback_cap;     /* accumulation-array capacity (the paper's `cap`) of the global-
                                  memory ISM, power of two in [2, 2048]; default 2048              */

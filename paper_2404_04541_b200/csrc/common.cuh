@@ -32,7 +32,7 @@ constexpr int DENSE_WARP_BM_WORDS = 1024;  // bitmap words a warp-per-row worksp
 constexpr int DENSE_WARP_ACC = 256;        // outputs a warp-per-row numeric workspace may hold
 constexpr int DENSE_WARP_MAX_UB = 4096;    // products a single warp is given at most
 constexpr i64 DENSE_HUB_UB = 1ll << 17;    // rows with at least this many products are scheduled first
-constexpr int DENSE_MAX_SPAN_WORDS = 32768;// 2^20 columns: the widest bitmap one CTA can hold
+constexpr int DENSE_MAX_SPAN_WORDS = 16384;// 2^19 columns: the widest bitmap (8 bytes per word with its rank) one CTA holds
 
 enum DevStatus : int {
     DEV_OK = 0,

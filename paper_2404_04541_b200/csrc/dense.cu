@@ -16,10 +16,10 @@
 //   warp per row : bitmap <= 1024 words, <= 256 outputs.  A warp walks the A entries one at a
 //              time with its lanes across the B row, so no two lanes ever hit the same slot and
 //              the accumulator needs no atomics; sums are in loop order.
-//   CTA units    : any span up to 2^20 columns.  A row is cut into units of `unit_outputs`
-//              consecutive outputs (rank ranges), so units carry equal output counts however
-//              skewed the columns are; hub rows spread over many CTAs and write disjoint,
-//              ordered pieces of the row.  Shared-memory atomics combine the CTA's warps.
+//   CTA units    : any span up to 2^19 columns.  A unit is a row, or an equal share of the A
+//              entries of a row with very many products, so hub rows spread over many CTAs.
+//              The first `unit_outputs` outputs of the row accumulate in shared memory
+//              (atomics combine the CTA's warps), the rest in the row's value segment.
 #include "common.cuh"
 
 namespace spws {
@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 // in shared memory; outputs beyond accumulate straight into the row's value segment in global
 // memory (zeroed beforehand), which keeps any row to a single pass whatever its output count.
 // ---------------------------------------------------------------------------------------
-constexpr int DN_ENTRIES = 1024;     // A entries whose descriptors are staged per round
+constexpr int DN_ENTRIES = 768;      // A entries whose descriptors are staged per round
 constexpr int DN_TILE = 256;         // products a warp takes per fetch
 
 // Zero the value segments of the rows that several units add into (a row with a single unit
@@ -370,12 +370,10 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
                                                                    int* __restrict__ Ccrd, T* __restrict__ Cval) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
-    unsigned* bm = reinterpret_cast<unsigned*>(acc + CAP);                           // smem_words
-    int* crank = reinterpret_cast<int*>(bm + smem_words);                            // smem_words / 32 + 1: rank at chunk start
-    unsigned short* pre = reinterpret_cast<unsigned short*>(crank + smem_words / 32 + 1);   // rank of word start inside its chunk
+    // per bitmap word: .x = the word, .y = outputs of the row before it (one load gives a rank)
+    uint2* bmr = reinterpret_cast<uint2*>(acc + CAP);                                // smem_words
     // staged descriptors of up to DN_ENTRIES A entries: B-row start, A value, running product count
-    i64* d_qs = reinterpret_cast<i64*>(smem_raw + ((sizeof(T) * (size_t)CAP + 4 * (size_t)smem_words + 4 * (size_t)(smem_words / 32 + 1) +
-                                                     2 * (size_t)smem_words + 15) & ~(size_t)15));
+    i64* d_qs = reinterpret_cast<i64*>(smem_raw + ((sizeof(T) * (size_t)CAP + 8 * (size_t)smem_words + 15) & ~(size_t)15));
     T* d_a = reinterpret_cast<T*>(d_qs + DN_ENTRIES);
     int* d_pre = reinterpret_cast<int*>(d_a + DN_ENTRIES);                           // DN_ENTRIES + 1
     __shared__ int s_next, s_tile;
@@ -408,22 +406,31 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
         if (nun == 1)                                   // outputs beyond the shared-memory part start at zero
             for (int x = CAP + tid; x < cnt; x += DN_THREADS) gacc[x] = 0;
 
-        // the row's bitmap, the rank at every chunk start and the rank of every word inside its chunk
+        // the row's bitmap with the rank of every word's first bit (the symbolic pass saved the
+        // rank at every chunk start).  A warp takes eight chunks at a time, all loads first.
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        for (int c = warp; c < nch; c += DN_WARPS) {
-            const int w = (c << 5) + lane;
-            const unsigned word = (w < nw) ? src[w] : 0u;
-            const int pc = __popc(word);
-            const int incl = warp_incl_scan(pc);
-            if (w < nw) { bm[w] = word; pre[w] = (unsigned short)(incl - pc); }
-            if (lane == 0) crank[c] = (int)src[nw + c];
+        for (int c0 = warp; c0 < nch; c0 += DN_WARPS * 8) {
+            unsigned word[8], rank_c[8];
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const int c = c0 + x * DN_WARPS, w = (c << 5) + lane;
+                word[x] = (w < nw) ? src[w] : 0u;
+                rank_c[x] = (c < nch) ? src[nw + c] : 0u;
+            }
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const int c = c0 + x * DN_WARPS, w = (c << 5) + lane;
+                const int pc = __popc(word[x]);
+                const int incl = warp_incl_scan(pc);
+                if (w < nw) bmr[w] = make_uint2(word[x], rank_c[x] + (unsigned)(incl - pc));
+            }
         }
         __syncthreads();
 
 #define SPWS_DENSE_ADD(REL, VAL)                                                                          \
         if ((REL) < span_bits) {                                                                          \
-            const unsigned w_ = (REL) >> 5;                                                               \
-            const int r_ = crank[w_ >> 5] + pre[w_] + __popc(bm[w_] & ((1u << ((REL) & 31)) - 1u));        \
+            const uint2 br_ = bmr[(REL) >> 5];                                                            \
+            const int r_ = (int)br_.y + __popc(br_.x & ((1u << ((REL) & 31)) - 1u));                      \
             if (r_ < CAP) atomicAdd(&acc[r_], (VAL));                                                     \
             else if (r_ < cnt) atomicAdd(gacc + r_, (VAL));                                               \
         }
@@ -458,72 +465,92 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
                 if (2 * tid + 1 < nE) d_pre[2 * tid + 1] = excl + len2[0];
                 if (tid == 0) { d_pre[nE] = total; s_tile = 0; }
                 __syncthreads();
-                for (;;) {
-                    int t0 = 0;
-                    if (lane == 0) t0 = atomicAdd(&s_tile, DN_TILE);
-                    t0 = __shfl_sync(0xffffffffu, t0, 0);
-                    if (t0 >= total) break;
-                    const int t1 = min(total, t0 + DN_TILE);
-                    int e = 0;
-                    {   // entry that holds product t0: the last one whose running count is <= t0
-                        int lo = 0, hi = nE;
-                        while (hi - lo > 1) {
-                            const int mid = (lo + hi) >> 1;
-                            if (d_pre[mid] <= t0) lo = mid; else hi = mid;
-                        }
-                        e = lo;
+                // Every warp walks the product stream tile by tile.  The loads of a step are
+                // issued before the previous step is ranked and added, so gather latency and
+                // accumulation overlap inside a warp as well as across warps.
+                int t0 = 0, t1 = 0, e = 0;              // stream position, end of the tile in hand, entry at t0
+                auto next_tile = [&]() -> bool {
+                    int s = 0;
+                    if (lane == 0) s = atomicAdd(&s_tile, DN_TILE);
+                    t0 = __shfl_sync(0xffffffffu, s, 0);
+                    if (t0 >= total) return false;
+                    t1 = min(total, t0 + DN_TILE);
+                    int lo = 0, hi = nE;                // the last entry whose running count is <= t0
+                    while (hi - lo > 1) {
+                        const int mid = (lo + hi) >> 1;
+                        if (d_pre[mid] <= t0) lo = mid; else hi = mid;
                     }
-                    if (!long_rows) {
-                        // short B rows: every lane walks its own products (t0 + lane, + 32, ...) and
-                        // advances its own entry index, so lanes stay busy across row boundaries
-                        int my_e = e;
-                        for (int t = t0 + lane; t < t1; t += 64) {      // two products in flight per lane
-                            while (d_pre[my_e + 1] <= t) ++my_e;
-                            const i64 q0 = d_qs[my_e] + (t - d_pre[my_e]);
-                            const T a0 = d_a[my_e];
-                            const int t2 = t + 32;
-                            const bool two = t2 < t1;
-                            i64 q1 = q0;
-                            T a1 = 0;
-                            if (two) {
-                                while (d_pre[my_e + 1] <= t2) ++my_e;
-                                q1 = d_qs[my_e] + (t2 - d_pre[my_e]);
-                                a1 = d_a[my_e];
-                            }
-                            const unsigned rel0 = (unsigned)(__ldg(B.crd + q0) - base);
-                            const unsigned rel1 = two ? (unsigned)(__ldg(B.crd + q1) - base) : 0xffffffffu;
-                            const T v0 = a0 * __ldg(Bval + q0);
-                            const T v1 = a1 * __ldg(Bval + q1);
-                            SPWS_DENSE_ADD(rel0, v0)
-                            SPWS_DENSE_ADD(rel1, v1)
-                        }
-                        continue;
-                    }
-                    while (t0 < t1) {
-                        const int e_end = d_pre[e + 1];
-                        if (e_end <= t0) { ++e; continue; }
-                        const int seg_end = min(t1, e_end);
-                        const int off = t0 - d_pre[e], n = seg_end - t0;
+                    e = lo;
+                    return true;
+                };
+                if (long_rows) {
+                    // a step = up to 128 consecutive products of one B row, four per lane
+                    auto fetch = [&](unsigned (&rel)[4], T (&b)[4], T& a) -> bool {
+                        if (t0 >= t1 && !next_tile()) return false;
+                        while (d_pre[e + 1] <= t0) ++e;
+                        const int off = t0 - d_pre[e];
+                        const int n = min(min(t1, d_pre[e + 1]) - t0, 128);
                         const int* __restrict__ ck = B.crd + d_qs[e] + off;
                         const T* __restrict__ vk = Bval + d_qs[e] + off;
-                        const T a = d_a[e];
-                        int t = lane;
-                        for (; t + 96 < n; t += 128) {    // four products in flight per lane
-                            const unsigned rel0 = (unsigned)(__ldg(ck + t) - base), rel1 = (unsigned)(__ldg(ck + t + 32) - base);
-                            const unsigned rel2 = (unsigned)(__ldg(ck + t + 64) - base), rel3 = (unsigned)(__ldg(ck + t + 96) - base);
-                            const T v0 = a * __ldg(vk + t), v1 = a * __ldg(vk + t + 32);
-                            const T v2 = a * __ldg(vk + t + 64), v3 = a * __ldg(vk + t + 96);
-                            SPWS_DENSE_ADD(rel0, v0)
-                            SPWS_DENSE_ADD(rel1, v1)
-                            SPWS_DENSE_ADD(rel2, v2)
-                            SPWS_DENSE_ADD(rel3, v3)
+                        a = d_a[e];
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            const int idx = lane + 32 * x;
+                            rel[x] = idx < n ? (unsigned)(__ldg(ck + idx) - base) : 0xffffffffu;
+                            b[x] = idx < n ? __ldg(vk + idx) : (T)0;
                         }
-                        for (; t < n; t += 32) {
-                            const unsigned rel0 = (unsigned)(__ldg(ck + t) - base);
-                            const T v0 = a * __ldg(vk + t);
-                            SPWS_DENSE_ADD(rel0, v0)
+                        t0 += n;
+                        return true;
+                    };
+                    unsigned relc[4] = {0, 0, 0, 0}, reln[4] = {0, 0, 0, 0};
+                    T bc[4] = {0, 0, 0, 0}, bn[4] = {0, 0, 0, 0};
+                    T ac = 0, an = 0;
+                    bool have = fetch(relc, bc, ac);
+                    while (have) {
+                        const bool more = fetch(reln, bn, an);
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) { SPWS_DENSE_ADD(relc[x], ac * bc[x]) }
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) { relc[x] = reln[x]; bc[x] = bn[x]; }
+                        ac = an;
+                        have = more;
+                    }
+                } else {
+                    // short B rows: a step = 64 consecutive products of the stream, two per lane;
+                    // every lane advances its own entry index across row boundaries
+                    int my_e = 0;
+                    auto fetch = [&](unsigned (&rel)[2], T (&b)[2], T (&a)[2]) -> bool {
+                        if (t0 >= t1) {
+                            if (!next_tile()) return false;
+                            my_e = e;
                         }
-                        t0 = seg_end;
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            const int t = t0 + lane + 32 * x;
+                            rel[x] = 0xffffffffu;
+                            b[x] = 0;
+                            a[x] = 0;
+                            if (t < t1) {
+                                while (d_pre[my_e + 1] <= t) ++my_e;
+                                const i64 q = d_qs[my_e] + (t - d_pre[my_e]);
+                                a[x] = d_a[my_e];
+                                rel[x] = (unsigned)(__ldg(B.crd + q) - base);
+                                b[x] = __ldg(Bval + q);
+                            }
+                        }
+                        t0 = min(t1, t0 + 64);
+                        return true;
+                    };
+                    unsigned relc[2] = {0, 0}, reln[2] = {0, 0};
+                    T bc[2] = {0, 0}, bn[2] = {0, 0}, ac[2] = {0, 0}, an[2] = {0, 0};
+                    bool have = fetch(relc, bc, ac);
+                    while (have) {
+                        const bool more = fetch(reln, bn, an);
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) { SPWS_DENSE_ADD(relc[x], ac[x] * bc[x]) }
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) { relc[x] = reln[x]; bc[x] = bn[x]; ac[x] = an[x]; }
+                        have = more;
                     }
                 }
                 __syncthreads();
@@ -700,7 +727,7 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int phase, int n_units_host, in
                              const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
     const int CAP = c.prm.unit_outputs;
     const i64 unit_products = dense_unit_products(total_products);
-    const size_t smem = ((sizeof(T) * (size_t)CAP + (size_t)words * 4 + (size_t)(words / 32 + 1) * 4 + (size_t)words * 2 + 15) & ~(size_t)15) +
+    const size_t smem = ((sizeof(T) * (size_t)CAP + (size_t)words * 8 + 15) & ~(size_t)15) +
                         (size_t)DN_ENTRIES * (8 + sizeof(T)) + (size_t)(DN_ENTRIES + 1) * 4 + 16;
     cudaError_t e;
     int per_sm = 0;

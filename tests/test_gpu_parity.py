@@ -218,6 +218,33 @@ def test_wide_columns_with_many_products(ctx, oracle_mod, policy):
     check_spgemm(ctx, oracle_mod, Abig, B, policy)
 
 
+def test_dense_cta_widest_span_and_just_beyond(ctx, oracle_mod):
+    """Rows whose outputs cover almost 2^19 columns (the widest dense workspace one CTA holds, with
+    the whole bitmap and its ranks in shared memory) and rows a little wider, which must fall back
+    to the insert-sort-merge workspace in global memory."""
+    ncols = 600_000
+    B = uniform_rows_csr(96, ncols, 128, 31)
+    crd, pos = B.crd, B.pos
+    # rows 0..63 of B are clipped to the first 2^19 columns; rows 64..95 keep all 600 000
+    out_pos, out_crd, out_val = [0], [], []
+    for k in range(B.nrows):
+        c = crd[pos[k]:pos[k + 1]]
+        v = B.val[pos[k]:pos[k + 1]]
+        if k < 64:
+            sel = c < (1 << 19)
+            c, v = c[sel], v[sel]
+        out_crd.append(c); out_val.append(v); out_pos.append(out_pos[-1] + c.size)
+    Bc = CSR(B.nrows, ncols, np.asarray(out_pos, dtype=np.int64), np.concatenate(out_crd).astype(np.int32),
+             np.concatenate(out_val))
+    Bc.val[:] = np.round(Bc.val * 16) / 16
+    a_pos = np.array([0, 64, 160], dtype=np.int64)                     # row 0: narrow B rows, row 1: all B rows
+    a_crd = np.concatenate([np.arange(64), np.arange(96)]).astype(np.int32)
+    a_val = (1 + (np.arange(160) % 7) / 8.0).astype(np.float64)
+    A = CSR(2, 96, a_pos, a_crd, a_val)
+    stats = check_spgemm(ctx, oracle_mod, A, Bc, "auto")
+    assert sum(stats["rows_per_class"][DENSE]) == 1 and stats["rows_per_class"][GLOBAL] == 1
+
+
 def test_dense_policy_refuses_prohibitive_workspace(ctx):
     from paper_2404_04541_b200 import binding
     c = config_inputs("wide26", reduced=True)
