@@ -31,6 +31,12 @@ constexpr int DC_WARPS = DC_THREADS / 32;
 constexpr int DN_THREADS = 512;            // numeric CTA kernel
 constexpr int DN_WARPS = DN_THREADS / 32;
 
+// A warp-route row whose bitmap is mostly empty words saves only the non-empty ones; bm_off then
+// carries a flag and the number of saved words above the slot offset.
+constexpr i64 BM_COMPACT = 1ll << 62;
+constexpr int BM_NZW_SHIFT = 44;
+constexpr i64 BM_OFF_MASK = (1ll << BM_NZW_SHIFT) - 1;
+
 // A dense row's slot in the arena: nw bitmap words, then for every chunk of 32 words the rank of
 // the chunk's first bit (an exclusive prefix of the chunk popcounts).
 __device__ __forceinline__ int chunks_of(int nw) { return (nw + 31) >> 5; }
@@ -53,6 +59,8 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
     class_range(ctl, CLS_DENSE_WARP, off, n);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned* bm = s_bm[warp];
+    for (int w = lane; w < DENSE_WARP_BM_WORDS; w += 32) bm[w] = 0;     // every row leaves its bitmap clear
+    __syncwarp();
     for (;;) {
         int r = 0;
         if (lane == 0) r = atomicAdd(&ctl->work_counter[CLS_DENSE_WARP], 1);
@@ -63,8 +71,6 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
         const int nw = (tab.jmax[row] - base) / 32 + 1;
         const unsigned span = (unsigned)nw * 32u;
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
-        for (int w = lane; w < nw; w += 32) bm[w] = 0;
-        __syncwarp();
         const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
         if (gs == 32) {
             // descriptors of 32 A entries at a time (one per lane), then the first 32 elements of
@@ -115,18 +121,46 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
             }
         }
         __syncwarp();
-        unsigned* out = tab.bm_arena + tab.bm_off[row];
-        int carry = 0;
+        // outputs and non-empty words of the row
+        int cnt = 0, nzw = 0;
         for (int w0 = 0; w0 < nw; w0 += 32) {
             const int w = w0 + lane;
             const unsigned word = (w < nw) ? bm[w] : 0u;
-            if (w < nw) out[w] = word;
-            int c = __popc(word);
-            for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
-            if (lane == 0) out[nw + (w0 >> 5)] = (unsigned)carry;
-            carry += c;
+            cnt += __popc(word);
+            nzw += __popc(__ballot_sync(0xffffffffu, word != 0u));
         }
-        if (lane == 0) tab.cnt[row] = carry;
+        for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+        const i64 slot = tab.bm_off[row];
+        unsigned* out = tab.bm_arena + slot;
+        if (cnt <= DENSE_WARP_ACC && 2 * nzw <= nw + chunks_of(nw)) {
+            // compact form for the warp numeric kernel: only the non-empty words, as (bits, word index)
+            uint2* out2 = reinterpret_cast<uint2*>(out);
+            int at = 0;
+            for (int w0 = 0; w0 < nw; w0 += 32) {
+                const int w = w0 + lane;
+                const unsigned word = (w < nw) ? bm[w] : 0u;
+                const unsigned ball = __ballot_sync(0xffffffffu, word != 0u);
+                if (word != 0u) {
+                    out2[at + __popc(ball & ((1u << lane) - 1u))] = make_uint2(word, (unsigned)w);
+                    bm[w] = 0;
+                }
+                at += __popc(ball);
+            }
+            if (lane == 0) tab.bm_off[row] = slot | ((i64)nzw << BM_NZW_SHIFT) | BM_COMPACT;
+        } else {
+            // full form: every word, then the rank at every 32-word chunk start
+            int carry = 0;
+            for (int w0 = 0; w0 < nw; w0 += 32) {
+                const int w = w0 + lane;
+                const unsigned word = (w < nw) ? bm[w] : 0u;
+                if (w < nw) { out[w] = word; bm[w] = 0; }
+                int c = __popc(word);
+                for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
+                if (lane == 0) out[nw + (w0 >> 5)] = (unsigned)carry;
+                carry += c;
+            }
+        }
+        if (lane == 0) tab.cnt[row] = cnt;
         __syncwarp();
     }
 }
@@ -218,13 +252,14 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
     if (ctl->status != 0) return;
     const int n = ctl->n_warp_rows;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // per warp: accw values, bmw bitmap words, bmw word ranks (the largest / widest row of this launch)
-    T* acc = reinterpret_cast<T*>(smem_raw) + warp * accw;
-    unsigned* bm = reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * accw) + warp * bmw;
-    unsigned short* pre = reinterpret_cast<unsigned short*>(reinterpret_cast<unsigned*>(reinterpret_cast<T*>(smem_raw) + DW_WARPS * accw) +
-                                                            DW_WARPS * bmw) + warp * bmw;
+    // per warp: a table of bmw bitmap words, each with the number of outputs before it (one load
+    // ranks a column), and accw values (sized from the widest / largest row of this launch)
+    uint2* tbl = reinterpret_cast<uint2*>(smem_raw) + warp * bmw;
+    T* acc = reinterpret_cast<T*>(reinterpret_cast<uint2*>(smem_raw) + DW_WARPS * bmw) + warp * accw;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
+    for (int w = lane; w < bmw; w += 32) tbl[w] = make_uint2(0u, 0u);       // every row leaves its table clear
+    __syncwarp();
     for (;;) {
         int r = 0;
         if (lane == 0) r = atomicAdd(&ctl->work_counter[NUM_SLOT + CLS_DENSE_WARP], 1);
@@ -237,14 +272,31 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const i64 out0 = rowptr[row];
         const int cnt = min((int)(rowptr[row + 1] - out0), accw);
-        // reload the bitmap; rank of each word's first bit = chunk rank + prefix inside the chunk
-        const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        for (int w0 = 0; w0 < nw; w0 += 32) {
-            const int w = w0 + lane;
-            const unsigned word = (w < nw) ? src[w] : 0u;
-            const int c = __popc(word);
-            const int incl = warp_incl_scan(c);
-            if (w < nw) { bm[w] = word; pre[w] = (unsigned short)((int)src[nw + (w0 >> 5)] + incl - c); }
+        const i64 slot = tab.bm_off[row];
+        const bool compact = (slot & BM_COMPACT) != 0;
+        const int nzw = (int)((slot & ~BM_COMPACT) >> BM_NZW_SHIFT);
+        const unsigned* src = tab.bm_arena + (slot & BM_OFF_MASK);
+        const uint2* src2 = reinterpret_cast<const uint2*>(src);
+        if (compact) {
+            // the saved non-empty words in column order: ranks by a running prefix of their bit counts
+            int carry = 0;
+            for (int i0 = 0; i0 < nzw; i0 += 32) {
+                const int i = i0 + lane;
+                const uint2 e = (i < nzw) ? src2[i] : make_uint2(0u, 0u);
+                const int c = __popc(e.x);
+                const int incl = warp_incl_scan(c);
+                if (i < nzw && e.y < (unsigned)nw) tbl[e.y] = make_uint2(e.x, (unsigned)(carry + incl - c));
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+            }
+        } else {
+            // the whole bitmap; rank of each word's first bit = chunk rank + prefix inside the chunk
+            for (int w0 = 0; w0 < nw; w0 += 32) {
+                const int w = w0 + lane;
+                const unsigned word = (w < nw) ? src[w] : 0u;
+                const int c = __popc(word);
+                const int incl = warp_incl_scan(c);
+                if (w < nw) tbl[w] = make_uint2(word, src[nw + (w0 >> 5)] + (unsigned)(incl - c));
+            }
         }
         for (int x = lane; x < cnt; x += 32) acc[x] = 0;
         __syncwarp();
@@ -278,27 +330,31 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                     if (lane < len1) { rel1 = (unsigned)(__ldg(B.crd + qs1 + lane) - base); v1 = __ldg(Bval + qs1 + lane); }
                     // entry e
                     if (rel0 < span) {
-                        const int slot = pre[rel0 >> 5] + __popc(bm[rel0 >> 5] & ((1u << (rel0 & 31)) - 1u));
-                        if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a0, v0));
+                        const uint2 t = tbl[rel0 >> 5];
+                        const int slot_ = (int)t.y + __popc(t.x & ((1u << (rel0 & 31)) - 1u));
+                        if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a0, v0));
                     }
                     for (int t = lane + 32; t < len0; t += 32) {
                         const unsigned rel = (unsigned)(__ldg(B.crd + qs0 + t) - base);
                         if (rel < span) {
-                            const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                            if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a0, __ldg(Bval + qs0 + t)));
+                            const uint2 tw = tbl[rel >> 5];
+                            const int slot_ = (int)tw.y + __popc(tw.x & ((1u << (rel & 31)) - 1u));
+                            if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a0, __ldg(Bval + qs0 + t)));
                         }
                     }
                     __syncwarp();
                     // entry e + 1
                     if (rel1 < span) {
-                        const int slot = pre[rel1 >> 5] + __popc(bm[rel1 >> 5] & ((1u << (rel1 & 31)) - 1u));
-                        if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a1, v1));
+                        const uint2 t = tbl[rel1 >> 5];
+                        const int slot_ = (int)t.y + __popc(t.x & ((1u << (rel1 & 31)) - 1u));
+                        if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a1, v1));
                     }
                     for (int t = lane + 32; t < len1; t += 32) {
                         const unsigned rel = (unsigned)(__ldg(B.crd + qs1 + t) - base);
                         if (rel < span) {
-                            const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                            if (slot < accw) acc[slot] = add_rn(acc[slot], mul_rn(a1, __ldg(Bval + qs1 + t)));
+                            const uint2 tw = tbl[rel >> 5];
+                            const int slot_ = (int)tw.y + __popc(tw.x & ((1u << (rel & 31)) - 1u));
+                            if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a1, __ldg(Bval + qs1 + t)));
                         }
                     }
                     __syncwarp();
@@ -316,22 +372,41 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                 for (int t = gl; t < len; t += gs) {
                     const unsigned rel = (unsigned)(__ldg(B.crd + qs + t) - base);
                     if (rel < span) {
-                        const int slot = pre[rel >> 5] + __popc(bm[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                        if (slot < accw) atomicAdd(&acc[slot], mul_rn(a, __ldg(Bval + qs + t)));
+                        const uint2 tw = tbl[rel >> 5];
+                        const int slot_ = (int)tw.y + __popc(tw.x & ((1u << (rel & 31)) - 1u));
+                        if (slot_ < accw) atomicAdd(&acc[slot_], mul_rn(a, __ldg(Bval + qs + t)));
                     }
                 }
             }
             __syncwarp();
         }
-        // copy out: values are already in output order; set bits give the coordinates
+        // copy out: values are already in output order; set bits give the coordinates; the table
+        // words the row used are cleared on the way
         for (int x = lane; x < cnt; x += 32) Cval[out0 + x] = acc[x];
-        for (int w = lane; w < nw; w += 32) {
-            unsigned word = bm[w];
-            i64 o = out0 + pre[w];
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                Ccrd[o++] = base + (w << 5) + b;
+        if (compact) {
+            for (int i = lane; i < nzw; i += 32) {
+                const uint2 e = src2[i];
+                if (e.y >= (unsigned)nw) continue;
+                unsigned word = e.x;
+                i64 o = out0 + tbl[e.y].y;
+                tbl[e.y] = make_uint2(0u, 0u);
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+                    Ccrd[o++] = base + (int)(e.y << 5) + b;
+                }
+            }
+        } else {
+            for (int w = lane; w < nw; w += 32) {
+                const uint2 t = tbl[w];
+                unsigned word = t.x;
+                i64 o = out0 + t.y;
+                tbl[w] = make_uint2(0u, 0u);
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+                    Ccrd[o++] = base + (w << 5) + b;
+                }
             }
         }
         __syncwarp();
@@ -701,7 +776,7 @@ template <typename T>
 static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, int bmw, int accw, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd,
                               void* Cval) {
     int per_sm = 0;
-    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * (size_t)accw + 6 * (size_t)bmw);
+    const size_t smem = (size_t)DW_WARPS * (sizeof(T) * (size_t)accw + 8 * (size_t)bmw);
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(dense_num_warp_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_num_warp_kernel<T>, DW_THREADS, smem)) != cudaSuccess) return e;
