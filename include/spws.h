@@ -101,7 +101,7 @@ typedef struct {
     int32_t fallback_cap;     /* accumulation-array capacity (the paper's `cap`) of the global-
                                  memory ISM, power of two in [2, 2048]; default 2048              */
     float dense_span_words_per_product; /* AUTO prefers DENSE over the shared-memory ISM when
-                                 span/32 <= this * products; default 4                            */
+                                 span/32 <= this * products; default 8                            */
     int32_t reserved[5];
 } spws_options_t;
 

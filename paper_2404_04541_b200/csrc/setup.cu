@@ -92,17 +92,29 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         i64 u = 0;
         int lo = 0x7fffffff, hi = -1;
         bool bad = false;
-        for (i64 p = ps + gl; p < pe; p += G) {
-            const int k = __ldg(A.crd + p);
-            if ((unsigned)k < (unsigned)B.nrows) {
-                const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
-                if (qe > qs) {
-                    u += qe - qs;
-                    lo = min(lo, __ldg(B.crd + qs));
-                    hi = max(hi, __ldg(B.crd + qe - 1));
+        // four entries per lane and step, each level of loads issued for all four before the
+        // next level needs it: a row with very many entries is a chain of dependent loads otherwise
+        for (i64 p0 = ps + gl; p0 < pe; p0 += 4 * G) {
+            int k[4];
+            i64 qs[4], qe[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const i64 p = p0 + (i64)x * G;
+                k[x] = p < pe ? __ldg(A.crd + p) : -1;
+                if (p < pe && (unsigned)k[x] >= (unsigned)B.nrows) bad = true;
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                qs[x] = qe[x] = 0;
+                if ((unsigned)k[x] < (unsigned)B.nrows) { qs[x] = __ldg(B.pos + k[x]); qe[x] = __ldg(B.pos + k[x] + 1); }
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                if (qe[x] > qs[x]) {
+                    u += qe[x] - qs[x];
+                    lo = min(lo, __ldg(B.crd + qs[x]));
+                    hi = max(hi, __ldg(B.crd + qe[x] - 1));
                 }
-            } else {
-                bad = true;
             }
         }
 #pragma unroll

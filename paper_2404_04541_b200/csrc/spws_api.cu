@@ -341,7 +341,7 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
     if (o.dense_unit_outputs == 0) o.dense_unit_outputs = 4096;
     if (o.dense_max_span == 0) o.dense_max_span = 1 << 19;
     if (o.fallback_cap == 0) o.fallback_cap = 2048;
-    if (o.dense_span_words_per_product == 0.0f) o.dense_span_words_per_product = 4.0f;
+    if (o.dense_span_words_per_product == 0.0f) o.dense_span_words_per_product = 8.0f;
     if (o.validate != 0 && o.validate != 1) return SPWS_INVALID_ARGUMENT;
     if (o.ism_warp_cap < 1 || o.ism_warp_cap > 32) return SPWS_INVALID_ARGUMENT;
     if (!is_pow2(o.ism_cta_cap) || o.ism_cta_cap < 64 || o.ism_cta_cap > 4096) return SPWS_INVALID_ARGUMENT;
