@@ -33,6 +33,7 @@ WORKLOAD_TEXT = {
     "stencil64": "FEM-like SpGEMM C=A*A, 27-point stencil on 64^3, fp64",
     "uniform8": "SpGEMM C=A*A, 2048x2048, 8 nnz/row, fp64",
     "wide26": "wide-output SpGEMM, A 65536 x 2^26, B 2^26 x 2^26, 4 nnz/row, fp32",
+    "ttm4096": "3-tensor times matrix C(i,j,l)=A(i,j,k)B(k,l), A 4096^3 CSF with 2^21 nnz, B 4096^2 CSR 8 nnz/row, fp64",
 }
 NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per product of the two kernels that
@@ -154,6 +155,8 @@ def run_reference(args):
     oracle.build()
     cfg = config_inputs(args.workload, seed=args.seed)
     A, B = cfg["A"], cfg["B"]
+    if cfg["kind"] == "ttm":                     # the 3-tensor form is the matrix form over the (i,j) fibres
+        A = A.fibres_as_csr()
     threads = oracle.hardware_threads()
     rows, psample, total = sized_oracle_sample(A, B, threads, 6.0)
     for _ in range(args.warmup):
@@ -179,7 +182,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="rmat18",
-                    help="rmat18 (default), stencil64, uniform8, wide26, or rmatNN / stencilNN at another size")
+                    help="rmat18 (default), stencil64, uniform8, wide26, ttm4096, or rmatNN / stencilNN at another size")
     ap.add_argument("--policy", default="auto")
     ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
     ap.add_argument("--seed", type=int, default=1)
@@ -208,29 +211,39 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = config_inputs(args.workload, seed=args.seed + rank)
-    A, B = cfg["A"], cfg["B"]
+    is_ttm = cfg["kind"] == "ttm"
+    T3 = cfg["A"] if is_ttm else None           # the CSF operand of the 3-tensor form
+    # the 3-tensor form works on the (i,j) fibres as rows: sizes, bytes and the oracle sample use that matrix
+    A, B = (T3.fibres_as_csr() if is_ttm else cfg["A"]), cfg["B"]
     V = 8 if cfg["dtype"] == np.float64 else 4
     vt = torch.float64 if V == 8 else torch.float32
     ctx = api.Context(dev)
-    dA = api.DeviceCSR.from_host(A, device=dev)
-    dB = dA if B is A else api.DeviceCSR.from_host(B, device=dev)
     options = {}
     for kv in args.opt:
         name, value = kv.split("=", 1)
         options[name] = float(value) if "." in value else int(value)
-    plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, cfg["dtype"], args.policy, **options)
+    if is_ttm:
+        dA = api.DeviceCSF3.from_host(T3, dev)
+        dB = api.DeviceCSR.from_host(B, device=dev)
+        plan = ctx.plan(api.EXPR_TTM, (binding.SPWS_CSF3, binding.SPWS_CSF3, binding.SPWS_CSR), cfg["dtype"], args.policy, **options)
+        symbolic, numeric, last = ctx.ttm_symbolic, ctx.ttm_numeric, 2
+    else:
+        dA = api.DeviceCSR.from_host(A, device=dev)
+        dB = dA if B is A else api.DeviceCSR.from_host(B, device=dev)
+        plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, cfg["dtype"], args.policy, **options)
+        symbolic, numeric, last = ctx.spgemm_symbolic, ctx.spgemm_numeric, 1
     plan.set_profiling(True)
 
     # a first pass sizes C; its buffers are reused by every step (allocation is outside the timed region)
-    c, state = ctx.spgemm_symbolic(plan, dA, dB)
-    nnzC = c.n[1]
+    c, state = symbolic(plan, dA, dB)
+    nnzC = c.n[last]
     crd = torch.empty(nnzC, dtype=torch.int32, device=dev)
     val = torch.empty(nnzC, dtype=vt, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)       # > L2 (126 MB)
 
     def step():
-        cc, st = ctx.spgemm_symbolic(plan, dA, dB)
-        ctx.spgemm_numeric(plan, cc, st, crd=crd, val=val)
+        cc, st = symbolic(plan, dA, dB)
+        numeric(plan, cc, st, crd=crd, val=val)
 
     for _ in range(args.warmup):
         step()
@@ -314,7 +327,8 @@ def main():
             "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "policy": args.policy, "options": options,
                        "seed": args.seed, "rows": int(A.nrows), "nnzA": int(A.nnz), "products": int(products),
                        "nnzC": int(nnzC), "l2": "512 MiB buffer written between timed steps",
-                       "timed": "spws_symbolic + spws_numeric; C buffers preallocated"},
+                       "timed": "spws_symbolic + spws_numeric; C buffers preallocated",
+                       **({"rows_are": "the (i,j) fibres of A"} if is_ttm else {})},
             "effective_gbs": eff_gbs, "algorithmic_bytes_per_step": abytes,
             "hbm_frac_nominal_8tbs": eff_gbs / NOMINAL_HBM_GBS, "hbm_frac_measured": eff_gbs / peak,
             "roofline": roofline, "kernel_ms": avg, "rows_per_class": stats["rows_per_class"],
@@ -324,24 +338,50 @@ def main():
             "gpu_launches": (stats["launches_symbolic"] + stats["launches_numeric"]) * args.steps,
             "clocks": clocks}
 
-    # ---- end to end through the host-buffer entry point (H2D of A, D2H of C inside the timed region)
-    if not args.no_e2e and B is A:
+    # ---- end to end through the host-buffer entry point (H2D of the operands, D2H of C inside the timed region)
+    if not args.no_e2e:
         try:
-            pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-            hp, hc, hv = pin(A.pos), pin(A.crd), pin(A.val)
-            cpos = torch.empty(A.nrows + 1, dtype=torch.int64).pin_memory()
-            ccrd = torch.empty(nnzC, dtype=torch.int32).pin_memory()
-            cval = torch.empty(nnzC, dtype=vt).pin_memory()
-            a = binding.csr_arrays(A.nrows, A.ncols, hp.numpy(), hc.numpy(), hv.numpy())
-            cc = binding.csr_arrays(A.nrows, A.ncols, cpos.numpy(), ccrd.numpy(), cval.numpy())
-            in_bytes = hp.numel() * 8 + hc.numel() * 4 + hv.numel() * V
-            ws = plan.workspace_size(dA.arrays(), dA.arrays())
-            arena_bytes = in_bytes + (A.nrows + 1) * 8 + ws + nnzC * (4 + V) + (1 << 20)
+            keep = []
+
+            def pin(a):
+                t = torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+                keep.append(t)
+                return t.numpy()
+
+            def pinned_out(n, dtype):
+                t = torch.empty(max(int(n), 1), dtype=dtype).pin_memory()
+                keep.append(t)
+                return t.numpy()
+
+            def host_csr(M):
+                return binding.csr_arrays(M.nrows, M.ncols, pin(M.pos), pin(M.crd), pin(M.val))
+
+            hb = host_csr(B)
+            if is_ttm:
+                ha = binding.csf3_arrays(T3.dims, pin(T3.pos0), pin(T3.crd0), pin(T3.pos1), pin(T3.crd1), pin(T3.pos2),
+                                         pin(T3.crd2), pin(T3.val))
+                n_i, n_ij = T3.n_i, T3.n_ij
+                cc = binding.TensorArrays(3, (T3.dims[0], T3.dims[1], B.ncols),
+                                          [pinned_out(2, torch.int64), pinned_out(n_i + 1, torch.int64), pinned_out(n_ij + 1, torch.int64)],
+                                          [pinned_out(n_i, torch.int32), pinned_out(n_ij, torch.int32), pinned_out(nnzC, torch.int32)],
+                                          pinned_out(nnzC, vt), [n_i, n_ij, nnzC])
+                in_bytes = (16 + n_i * 4 + (n_i + 1) * 8 + n_ij * 4 + (n_ij + 1) * 8 + T3.nnz * (4 + V)
+                            + (B.nrows + 1) * 8 + B.nnz * (4 + V))
+                out_fixed = 16 + n_i * 4 + (n_i + 1) * 8 + n_ij * 4 + (n_ij + 1) * 8
+            else:
+                ha = hb if B is A else host_csr(A)
+                cc = binding.csr_arrays(A.nrows, B.ncols, pinned_out(A.nrows + 1, torch.int64), pinned_out(nnzC, torch.int32),
+                                        pinned_out(nnzC, vt))
+                cc.n = [A.nrows, nnzC, 0]
+                in_bytes = (A.nrows + 1) * 8 + A.nnz * (4 + V) + (0 if B is A else (B.nrows + 1) * 8 + B.nnz * (4 + V))
+                out_fixed = (A.nrows + 1) * 8
+            ws = plan.workspace_size(dA.arrays(), dB.arrays())
+            arena_bytes = in_bytes + 2 * out_fixed + ws + nnzC * (4 + V) + (1 << 20)
             arena = torch.empty(arena_bytes + 256, dtype=torch.uint8, device=dev)
             aptr = ctx._aligned_ptr(arena)
             plan.set_profiling(False)
             for _ in range(2):
-                st, sizes, need = plan.execute_host(a, a, cc, aptr, arena_bytes)
+                st, sizes, need = plan.execute_host(ha, hb, cc, aptr, arena_bytes)
                 if st != 0:
                     raise RuntimeError(f"execute_host: {binding.status_string(st)} (needs {need} bytes)")
             n_e2e = max(1, min(args.steps, 3))
@@ -351,13 +391,13 @@ def main():
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             for _ in range(n_e2e):
-                st, sizes, need = plan.execute_host(a, a, cc, aptr, arena_bytes)
+                st, sizes, need = plan.execute_host(ha, hb, cc, aptr, arena_bytes)
             e1.record()
             torch.cuda.synchronize()
             e2e_ms = torch.tensor([e0.elapsed_time(e1) / n_e2e], dtype=torch.float64, device=dev)
             if world > 1:
                 dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-            out_bytes = (A.nrows + 1) * 8 + nnzC * (4 + V)
+            out_bytes = out_fixed + nnzC * (4 + V)
             line["e2e"] = {"value": 2.0 * all_products / (float(e2e_ms[0]) * 1e-3) / 1e9, "unit": UNIT,
                            "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
                            "ms_per_step": float(e2e_ms[0]), "steps": n_e2e,

@@ -124,6 +124,34 @@ class Context:
                 plan.close()
 
     # ------------------------------------------------------------------ TTM
+    def ttm_symbolic(self, plan: B_.Plan, A: DeviceCSF3, B: DeviceCSR):
+        """Symbolic pass of the 3-tensor form: allocates C's upper levels (bounded by A's) and returns
+        (C arrays with sizes filled in, state for ttm_numeric)."""
+        a, b = A.arrays(), B.arrays()
+        nbytes = plan.workspace_size(a, b)
+        sc = self.scratch(nbytes)
+        n_i, n_ij = a.n[0], a.n[1]
+        i64, i32, dev = torch.int64, torch.int32, self.device
+        pos0 = torch.empty(2, dtype=i64, device=dev)
+        crd0 = torch.empty(n_i, dtype=i32, device=dev)
+        pos1 = torch.empty(n_i + 1, dtype=i64, device=dev)
+        crd1 = torch.empty(n_ij, dtype=i32, device=dev)
+        pos2 = torch.empty(n_ij + 1, dtype=i64, device=dev)
+        c = B_.TensorArrays(3, (A.dims[0], A.dims[1], B.ncols), [pos0, pos1, pos2], [crd0, crd1, None], None,
+                            [n_i, n_ij, 0])
+        sizes = plan.symbolic(a, b, c, self._aligned_ptr(sc), nbytes)
+        return c, (a, b, sc, nbytes, sizes)
+
+    def ttm_numeric(self, plan: B_.Plan, c: B_.TensorArrays, state, crd=None, val=None) -> DeviceCSF3:
+        a, b, sc, nbytes, sizes = state
+        nnz = sizes[2]
+        vt = torch.float64 if plan.np_dtype == np.float64 else torch.float32
+        c.crd[2] = crd if crd is not None else torch.empty(nnz, dtype=torch.int32, device=self.device)
+        c.val = val if val is not None else torch.empty(nnz, dtype=vt, device=self.device)
+        plan.numeric(a, b, c, self._aligned_ptr(sc), nbytes)
+        return DeviceCSF3(c.dims, c.pos[0], c.crd[0][:sizes[0]], c.pos[1][:sizes[0] + 1], c.crd[1][:sizes[1]],
+                          c.pos[2][:sizes[1] + 1], c.crd[2][:nnz], c.val[:nnz])
+
     def ttm(self, A: DeviceCSF3, B: DeviceCSR, policy="auto", plan: B_.Plan | None = None, **options):
         """C(i,j,l) = sum_k A(i,j,k) B(k,l) with A, C in CSF; returns (C, stats)."""
         own = plan is None
@@ -131,25 +159,8 @@ class Context:
             dt = np.float64 if A.val.dtype == torch.float64 else np.float32
             plan = self.plan(EXPR_TTM, (B_.SPWS_CSF3, B_.SPWS_CSF3, B_.SPWS_CSR), dt, policy, **options)
         try:
-            a, b = A.arrays(), B.arrays()
-            nbytes = plan.workspace_size(a, b)
-            sc = self.scratch(nbytes)
-            n_i, n_ij = a.n[0], a.n[1]
-            i64, i32, dev = torch.int64, torch.int32, self.device
-            pos0 = torch.empty(2, dtype=i64, device=dev)
-            crd0 = torch.empty(n_i, dtype=i32, device=dev)
-            pos1 = torch.empty(n_i + 1, dtype=i64, device=dev)
-            crd1 = torch.empty(n_ij, dtype=i32, device=dev)
-            pos2 = torch.empty(n_ij + 1, dtype=i64, device=dev)
-            c = B_.TensorArrays(3, (A.dims[0], A.dims[1], B.ncols), [pos0, pos1, pos2], [crd0, crd1, None], None,
-                                [n_i, n_ij, 0])
-            sizes = plan.symbolic(a, b, c, self._aligned_ptr(sc), nbytes)
-            nnz = sizes[2]
-            c.crd[2] = torch.empty(nnz, dtype=i32, device=dev)
-            c.val = torch.empty(nnz, dtype=A.val.dtype, device=dev)
-            plan.numeric(a, b, c, self._aligned_ptr(sc), nbytes)
-            C = DeviceCSF3(c.dims, pos0, crd0[:sizes[0]], pos1[:sizes[0] + 1], crd1[:sizes[1]], pos2[:sizes[1] + 1],
-                           c.crd[2], c.val)
+            c, state = self.ttm_symbolic(plan, A, B)
+            C = self.ttm_numeric(plan, c, state)
             return C, plan.get_stats()
         finally:
             if own:

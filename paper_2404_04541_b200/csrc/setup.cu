@@ -87,6 +87,10 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
     const i64 group = ((i64)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const i64 ngroups = ((i64)gridDim.x * blockDim.x) / G;
     i64 my_products = 0, my_max = 0, my_max_global = 0;
+    // rows and products of the class of this group's last rows: neighbouring rows mostly share a
+    // class, so the shared-memory histogram is touched only when the class changes
+    int run_cls = -1, run_rows = 0, my_span_words = 0;
+    i64 run_products = 0;
     for (i64 row = group; row < A.nrows; row += ngroups) {
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         i64 u = 0;
@@ -94,7 +98,24 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         bool bad = false;
         // four entries per lane and step, each level of loads issued for all four before the
         // next level needs it: a row with very many entries is a chain of dependent loads otherwise
-        for (i64 p0 = ps + gl; p0 < pe; p0 += 4 * G) {
+        i64 p0 = ps + gl;
+        if (pe - ps <= G) {                         // the common short row: one entry per lane
+            if (p0 < pe) {
+                const int k = __ldg(A.crd + p0);
+                if ((unsigned)k < (unsigned)B.nrows) {
+                    const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                    if (qe > qs) {
+                        u = qe - qs;
+                        lo = __ldg(B.crd + qs);
+                        hi = __ldg(B.crd + qe - 1);
+                    }
+                } else {
+                    bad = true;
+                }
+            }
+            p0 = pe;
+        }
+        for (; p0 < pe; p0 += 4 * G) {
             int k[4];
             i64 qs[4], qe[4];
 #pragma unroll
@@ -132,15 +153,29 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             tab.jmax[row] = hi;
             tab.cnt[row] = 0;
             tab.cls[row] = (unsigned char)cls;
-            atomicAdd(&s_hist[cls], 1);
-            if (u) atomicAdd((u64*)&s_cprod[cls], (u64)u);
+            if (cls != run_cls) {
+                if (run_rows) {
+                    atomicAdd(&s_hist[run_cls], run_rows);
+                    if (run_products) atomicAdd((u64*)&s_cprod[run_cls], (u64)run_products);
+                }
+                run_cls = cls;
+                run_rows = 0;
+                run_products = 0;
+            }
+            ++run_rows;
+            run_products += u;
             my_products += u;
             my_max = max(my_max, u);
             if (cls == CLS_ISM_GLOBAL) my_max_global = max(my_max_global, u);
             if (cls == CLS_DENSE_HUB || cls == CLS_DENSE_CTA || cls == CLS_DENSE_WARP)
-                atomicMax(&s_max_span_words, (hi - lo) / 32 + 1);
+                my_span_words = max(my_span_words, (hi - lo) / 32 + 1);
         }
     }
+    if (gl == 0 && run_rows) {
+        atomicAdd(&s_hist[run_cls], run_rows);
+        if (run_products) atomicAdd((u64*)&s_cprod[run_cls], (u64)run_products);
+    }
+    if (gl == 0 && my_span_words) atomicMax(&s_max_span_words, my_span_words);
     if (gl == 0 && my_products) atomicAdd((u64*)&s_products, (u64)my_products);
     if (gl == 0 && my_max) atomicMax(&s_max_ub, my_max);
     if (gl == 0 && my_max_global) atomicMax(&s_max_ub_global, my_max_global);
