@@ -41,10 +41,10 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/ (taken on a smaller case of the same recipe where noted; traffic grows in proportion
 # to the products).  Valid only for the kernel source the capture was taken on.
 PROFILED_TRAFFIC = {
-    "num_dense_cta": {"bytes_per_product": (1716242000 + 3979372000) / 1079487607, "source": "profiles/dense_num_cta_kernel_rmat17.md"},
-    "num_dense_warp": {"bytes_per_product": (848124672 + 346681344) / 181321496, "source": "profiles/dense_num_warp_kernel_stencil64.md"},
+    "num_dense_cta": {"bytes_per_product": (1906732000 + 4161497000) / 1085650666, "source": "profiles/dense_cta_kernels_rmat17.md"},
+    "num_dense_warp": {"bytes_per_product": (324897792 + 332786432) / 181321496, "source": "profiles/dense_warp_kernels_stencil64.md"},
 }
-PROFILED_SOURCE_SHA = "26431363493c3924"   # sha256 prefix of csrc/dense.cu at capture time
+PROFILED_SOURCE_SHA = "595e09683d98a368"   # sha256 prefix of csrc/dense.cu at capture time
 
 
 def algorithmic_bytes(m, nnzA, products, nnzC, V):
