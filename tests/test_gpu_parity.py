@@ -191,6 +191,40 @@ def test_warp_dense_route_reproduces_sequential_sum(ctx, oracle_mod):
     assert ok.all()
 
 
+def test_warp_dense_route_compact_and_full_bitmaps(ctx, oracle_mod):
+    """The warp dense route saves a row's bitmap either whole or as its non-empty words only.
+    One matrix makes rows of every kind under the forced dense policy: a few products over a wide
+    span (compact form), many products over a narrow span (whole bitmap: the list would not fit
+    the slot), more than 256 outputs (handed to the CTA numeric kernel, which reads the whole
+    bitmap), and empty rows."""
+    rng = np.random.default_rng(11)
+    n = 20000
+    B = uniform_rows_csr(n, n, 6, 5)
+    rows, cols = [], []
+    for i in range(96):
+        kind = i % 4
+        if kind == 0:
+            ks = rng.choice(n, size=3, replace=False)           # 18 products anywhere in 20000 columns
+        elif kind == 1:
+            ks = rng.choice(n, size=30, replace=False)          # 180 products, still sparse words
+        elif kind == 2:
+            ks = rng.choice(n, size=120, replace=False)         # ~700 outputs: beyond a warp's accumulator
+        else:
+            ks = np.array([], dtype=np.int64)
+        rows += [i] * len(ks)
+        cols += sorted(int(k) for k in ks)
+    A = CSR.from_coo(96, n, rows, cols, rng.uniform(-1, 1, len(rows)))
+    # a block of rows that all pick B rows with the same few columns: narrow span, dense words
+    Bn = CSR.from_coo(64, 40, np.repeat(np.arange(64), 20), np.tile(np.arange(0, 40, 2), 64), rng.uniform(-1, 1, 64 * 20))
+    An = uniform_rows_csr(50, 64, 9, 6)
+    for (X, Y) in ((A, B), (An, Bn)):
+        stats = check_spgemm(ctx, oracle_mod, X, Y, "dense")
+        assert stats["rows_per_class"][4] > 0
+    # the wide case must have used both numeric kernels
+    stats = check_spgemm(ctx, oracle_mod, A, B, "dense")
+    assert 0 < stats["dense_warp_rows"] < 72 and stats["dense_units"] > 0
+
+
 # ------------------------------------------------------------------ benchmark configurations
 @pytest.mark.parametrize("policy", POLICIES)
 @pytest.mark.parametrize("cfg", ["uniform8", "rmat18", "stencil64"])
