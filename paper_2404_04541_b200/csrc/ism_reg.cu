@@ -32,6 +32,27 @@ __global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ pe
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const int base = jmin[row];
 
+        if (pe - ps == 1) {
+            // A row with ONE entry (the commonest fibre of a hyper-sparse 3-tensor): its products
+            // are the picked B row itself, already sorted and free of duplicates, so Insert, Sort
+            // and Merge are the identity and the lanes copy the scaled B row to the output.
+            const int k = __ldg(A.crd + ps);
+            i64 qs = 0;
+            int len = 0;
+            if ((unsigned)k < (unsigned)B.nrows) {
+                qs = __ldg(B.pos + k);
+                len = min((int)(__ldg(B.pos + k + 1) - qs), G);
+            }
+            if (!NUMERIC) {
+                if (gl == 0) cnt[row] = len;
+            } else if (gl < len) {
+                const i64 o = rowptr[row] + gl;
+                Ccrd[o] = __ldg(B.crd + qs + gl);
+                Cval[o] = mul_rn(__ldg(Aval + ps), __ldg(Bval + qs + gl));
+            }
+            continue;
+        }
+
         // ---- Insert: lane gl receives product number gl
         unsigned packed = 0xffffffffu;
         T val = 0;
