@@ -27,9 +27,23 @@ __global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ pe
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
 
+    // the row id and its A range are loaded one iteration ahead: with a handful of products per row
+    // the kernel is a chain of dependent loads otherwise
+    int row_n = 0;
+    i64 ps_n = 0, pe_n = 0;
+    if (group < n) {
+        row_n = __ldg(rows + group);
+        ps_n = __ldg(A.pos + row_n);
+        pe_n = __ldg(A.pos + row_n + 1);
+    }
     for (i64 r = group; r < n; r += ngroups) {
-        const int row = rows[r];
-        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        const int row = row_n;
+        const i64 ps = ps_n, pe = pe_n;
+        if (r + ngroups < n) {
+            row_n = __ldg(rows + r + ngroups);
+            ps_n = __ldg(A.pos + row_n);
+            pe_n = __ldg(A.pos + row_n + 1);
+        }
         const int base = jmin[row];
 
         if (pe - ps == 1) {
