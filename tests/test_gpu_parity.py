@@ -405,6 +405,65 @@ def test_ttm_config(ctx, oracle_mod, reduced):
     assert stats["products"] == 8 * c["A"].nnz
 
 
+def test_ttm_equals_spgemm_of_the_fibre_matrix(ctx):
+    """Hoisting the shared outer loops turns the 3-tensor form into the matrix form over the (i,j)
+    fibres: the last CSF level of the TTM result must equal the CSR result of the fibre matrix times
+    B on the same device path, bit for bit in structure and within rounding in value (fp32, fp64)."""
+    for dtype in (np.float32, np.float64):
+        A = uniform_csf3((48, 40, 64), 9000, 4)
+        A.val = A.val.astype(dtype)
+        B = random_csr(64, 500, 0.1, 9, empty_row_frac=0.3)
+        B.val = B.val.astype(dtype)
+        got, _ = run_ttm(ctx, A, B, "auto")
+        pos, crd, val, _ = run_spgemm(ctx, A.fibres_as_csr(), B, "auto")
+        keep = np.diff(pos) > 0                     # fibres without an output are dropped from C
+        assert np.array_equal(got["pos2"], np.concatenate([[0], np.cumsum(np.diff(pos)[keep])]))
+        assert np.array_equal(got["crd2"], crd)
+        tol = TOL[np.dtype(dtype)]                  # routes with atomics sum in a run-dependent order
+        assert np.allclose(got["val"], val, rtol=100 * tol, atol=100 * tol)
+        assert np.array_equal(got["crd1"], A.crd1[keep])
+
+
+def test_execute_host_ttm_and_distinct_operands(ctx, oracle_mod):
+    """The host-buffer entry point on the 3-tensor form and on a matrix product with B != A."""
+    import torch
+    from paper_2404_04541_b200 import api, binding
+    arena = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    A = uniform_csf3((32, 32, 64), 6000, 7)
+    B = random_csr(64, 200, 0.1, 8, empty_row_frac=0.4)
+    ref = oracle_mod.ttm(A, B)
+    plan = ctx.plan(api.EXPR_TTM, (binding.SPWS_CSF3, binding.SPWS_CSF3, binding.SPWS_CSR), np.float64)
+    a = binding.csf3_arrays(A.dims, A.pos0, A.crd0, A.pos1, A.crd1, A.pos2, A.crd2, A.val)
+    b = binding.csr_arrays(B.nrows, B.ncols, B.pos, B.crd, B.val)
+    nnz = ref.crd2.shape[0]
+    out = dict(pos0=np.empty(2, np.int64), crd0=np.empty(A.n_i, np.int32), pos1=np.empty(A.n_i + 1, np.int64),
+               crd1=np.empty(A.n_ij, np.int32), pos2=np.empty(A.n_ij + 1, np.int64), crd2=np.empty(nnz, np.int32),
+               val=np.empty(nnz, np.float64))
+    c = binding.TensorArrays(3, (A.dims[0], A.dims[1], B.ncols), [out["pos0"], out["pos1"], out["pos2"]],
+                             [out["crd0"], out["crd1"], out["crd2"]], out["val"], [A.n_i, A.n_ij, nnz])
+    st, sizes, _ = plan.execute_host(a, b, c, ctx._aligned_ptr(arena), arena.numel() - 256)
+    assert st == 0 and sizes == [ref.crd0.shape[0], ref.crd1.shape[0], nnz]
+    assert np.array_equal(out["pos0"], ref.pos0) and np.array_equal(out["crd0"][:sizes[0]], ref.crd0)
+    assert np.array_equal(out["pos1"][:sizes[0] + 1], ref.pos1) and np.array_equal(out["crd1"][:sizes[1]], ref.crd1)
+    assert np.array_equal(out["pos2"][:sizes[1] + 1], ref.pos2) and np.array_equal(out["crd2"], ref.crd2)
+    ok, _ = values_close(out["val"], ref.val_ref, ref.abs, 1e-12)
+    assert ok.all()
+    plan.close()
+    # matrix form, two different operands
+    M, N = random_csr(300, 64, 0.1, 12), B
+    mref = oracle_mod.spgemm(M, N)
+    plan = ctx.plan(api.EXPR_SPGEMM, (0, 0, 0), np.float64)
+    cpos, ccrd, cval = np.empty(301, np.int64), np.empty(mref.nnz, np.int32), np.empty(mref.nnz, np.float64)
+    cm = binding.csr_arrays(300, N.ncols, cpos, ccrd, cval)
+    st, sizes, _ = plan.execute_host(binding.csr_arrays(300, 64, M.pos, M.crd, M.val), b, cm, ctx._aligned_ptr(arena),
+                                     arena.numel() - 256)
+    assert st == 0 and sizes[1] == mref.nnz
+    assert np.array_equal(cpos, mref.pos) and np.array_equal(ccrd, mref.crd)
+    ok, _ = values_close(cval, mref.val_ref, mref.abs, 1e-12)
+    assert ok.all()
+    plan.close()
+
+
 # ------------------------------------------------------------------ boundary behaviour
 def test_error_statuses(ctx):
     import torch
