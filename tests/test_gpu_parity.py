@@ -225,6 +225,53 @@ def test_warp_dense_route_compact_and_full_bitmaps(ctx, oracle_mod):
     assert 0 < stats["dense_warp_rows"] < 72 and stats["dense_units"] > 0
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_randomized_shapes_policies_and_thresholds(ctx, oracle_mod, seed):
+    """Seeded random sweep: shapes from 1 x 1 to a few thousand rows and up to 2^20 columns, uniform /
+    power-law / stencil / heavy-row structure, both value types, every policy, and route thresholds
+    drawn at random, each case against the oracle (structure exact, values within the tolerance)."""
+    rng = np.random.default_rng(seed)
+    for _ in range(16):
+        kind = int(rng.integers(0, 5))
+        dtype = np.float64 if rng.random() < 0.7 else np.float32
+        s = int(rng.integers(1, 1 << 30))
+        if kind == 0:
+            m, k, n = int(rng.integers(1, 400)), int(rng.integers(1, 400)), int(rng.integers(1, 70000))
+            A = random_csr(m, k, float(rng.uniform(0.01, 0.5)), s, empty_row_frac=float(rng.uniform(0, 0.3)))
+            B = random_csr(k, n, float(rng.uniform(0.0005, 0.05)), s + 1, empty_row_frac=float(rng.uniform(0, 0.3)))
+        elif kind == 1:
+            A = B = rmat_csr(int(rng.integers(6, 13)), int(rng.integers(2, 24)), s)
+        elif kind == 2:
+            A = B = stencil27_csr(int(rng.integers(3, 13)), s)
+        elif kind == 3:
+            m, k = int(rng.integers(1, 3000)), int(rng.integers(1, 5000))
+            A = uniform_rows_csr(m, k, int(rng.integers(1, min(k, 40) + 1)), s)
+            n = int(rng.integers(64, 1 << 20))
+            B = uniform_rows_csr(k, n, int(rng.integers(1, min(n, 64) + 1)), s + 1)
+        else:                                       # a few very heavy rows over a wide span
+            k, n = int(rng.integers(500, 3000)), int(rng.integers(20000, 400000))
+            B = uniform_rows_csr(k, n, int(rng.integers(20, 200)), s + 1)
+            A = random_csr(int(rng.integers(2, 30)), k, float(rng.uniform(0.2, 1.0)), s)
+        A.val = A.val.astype(dtype)
+        B.val = B.val.astype(dtype)
+        policy = POLICIES[int(rng.integers(0, 3))]
+        if policy == "ism" and kind in (1, 4):
+            policy = "auto"                         # the global-memory ISM on very heavy rows is slow
+        opts = {}
+        if rng.random() < 0.5:
+            opts = dict(ism_warp_cap=int(rng.choice([4, 8, 16, 32])), ism_cta_cap=int(rng.choice([64, 256, 1024, 4096])),
+                        dense_unit_outputs=int(rng.choice([64, 256, 4096])), fallback_cap=int(rng.choice([2, 16, 256, 2048])))
+        if policy == "dense" and B.ncols > (1 << 19):
+            # a row may be wider than the widest dense workspace: the forced policy must then say so
+            from paper_2404_04541_b200 import binding
+            try:
+                check_spgemm(ctx, oracle_mod, A, B, policy, **opts)
+            except binding.SpwsError as e:
+                assert e.status == binding.SPWS_WORKSPACE_TOO_LARGE
+        else:
+            check_spgemm(ctx, oracle_mod, A, B, policy, **opts)
+
+
 # ------------------------------------------------------------------ benchmark configurations
 @pytest.mark.parametrize("policy", POLICIES)
 @pytest.mark.parametrize("cfg", ["uniform8", "rmat18", "stencil64"])
