@@ -15,16 +15,16 @@
 //                     map over l; fibres (and slices) with no output are not materialised, as
 //                     Compress only creates coordinates that exist (Fig. 8, Compress part).
 //   oracle_ism_rowwise / oracle_ism_outer :
-//                     Algorithm 1 taken step by step (Allocate; Insert; on full: Sort, Merge,
-//                     Insert again; tail Sort+Merge; Compress) with the Coord policy of Sec. 5.2
-//                     (append, no reduction on insert, lexicographic sort at flush) and an
-//                     out-of-place two-way Merge that reduces equal coordinates (Sec. 4.3).  The
-//                     row-wise form uses a first-order workspace per row; the outer form follows
-//                     the loop order k -> i -> j of the paper's running example (Sec. 2.1) with a
-//                     second-order workspace and the COO -> CSR Compress.  Reading of the
-//                     "Insert / if full / Insert again" protocol: an Insert into an accumulation
-//                     array that has no free slot stores nothing and raises `full`; the same
-//                     component is inserted again after the flush.
+//                     the insert-sort-merge workspace of Algorithm 1 under the coordinate-sort
+//                     policy of Sec. 5.2 (append without reduction; sort and reduce when the
+//                     bounded buffer is emptied; union with the sorted store of everything seen
+//                     so far, Sec. 4.3), as a second, independent route to the same result.  The
+//                     row-wise form gives every output row a first-order workspace; the outer form
+//                     feeds one second-order workspace in the order k -> i -> j of Sec. 2.1 and
+//                     converts the sorted coordinate list to CSR.  Reading of the algorithm's
+//                     "insert, and if that found the buffer full, flush and insert again": an
+//                     insert into a buffer without a free slot stores nothing; the same entry goes
+//                     in after the flush.
 //
 // Values: `val` is the double-precision sum taken in loop order (multiply, then add; built with
 // -ffp-contract=off); `val_ref` accumulates the same products in long double and rounds once;
@@ -108,82 +108,65 @@ void append(std::vector<T>& dst, const std::vector<T>& src) {
     dst.insert(dst.end(), src.begin(), src.end());
 }
 
-// ---- Algorithm 1 pieces (Coord policy) -------------------------------------------------
+// ---- Algorithm 1 with the coordinate-sort policy ---------------------------------------
+//
+// Written from the contract of Algorithm 1 (Sec. 4.2-4.3) and of the Coord policy (Sec. 5.2):
+// a bounded buffer of pending (coordinate, value) entries in arrival order, and one store of
+// settled entries that is always sorted by coordinate and free of duplicates.  An entry is
+// offered to the buffer; when the buffer has no room it is emptied first -- its entries are
+// put in coordinate order, equal coordinates are summed (this policy reduces at sort time, not
+// at insert time), and the result is united with the settled store, again summing equal
+// coordinates -- and the same entry is offered again.  What is still pending at the end is
+// emptied the same way.  The settled store is then the whole result in storage order.
 
-struct Component {
-    int32_t crd[2];
-    double val;
+struct Entry {
+    int32_t i, j;      // coordinate; first-order use keeps i = 0
+    double v;
 };
 
-inline bool crd_less(const Component& a, const Component& b) {
-    return a.crd[0] < b.crd[0] || (a.crd[0] == b.crd[0] && a.crd[1] < b.crd[1]);
-}
-inline bool crd_equal(const Component& a, const Component& b) {
-    return a.crd[0] == b.crd[0] && a.crd[1] == b.crd[1];
-}
+inline bool before(const Entry& a, const Entry& b) { return a.i != b.i ? a.i < b.i : a.j < b.j; }
+inline bool same_place(const Entry& a, const Entry& b) { return a.i == b.i && a.j == b.j; }
 
-struct AccArray {
-    std::vector<Component> slot;
-    size_t cap;
-    bool full = false;
-    explicit AccArray(size_t c) : cap(c) { slot.reserve(c); }
-    bool empty() const { return slot.empty(); }
-};
+class BoundedWorkspace {
+public:
+    explicit BoundedWorkspace(int64_t capacity) : capacity_(static_cast<size_t>(capacity)) { pending_.reserve(capacity_); }
 
-// Insert: append when a slot is free, otherwise store nothing and raise `full`.
-void Insert(const Component& c, AccArray& acc) {
-    if (acc.slot.size() < acc.cap) {
-        acc.slot.push_back(c);
-        acc.full = false;
-    } else {
-        acc.full = true;
+    void feed(const Entry& e) {
+        if (pending_.size() == capacity_) settle();      // no room: nothing is stored, empty the buffer ...
+        pending_.push_back(e);                           // ... and take the same entry afterwards
     }
-}
 
-// Sort: lexicographic order of the coordinates; equal coordinates are then adjacent and are
-// reduced here (the Coord policy does not reduce on insert).
-void Sort(AccArray& acc) {
-    std::stable_sort(acc.slot.begin(), acc.slot.end(), crd_less);
-    std::vector<Component> uniq;
-    for (const Component& c : acc.slot) {
-        if (!uniq.empty() && crd_equal(uniq.back(), c)) uniq.back().val += c.val;
-        else uniq.push_back(c);
-    }
-    acc.slot.swap(uniq);
-}
-
-// Merge: out-of-place two-way merge of the sorted accumulation array into the sorted all
-// array, reducing equal coordinates; clears the accumulation array.
-void Merge(AccArray& acc, std::vector<Component>& all) {
-    std::vector<Component> out;
-    out.reserve(all.size() + acc.slot.size());
-    size_t x = 0, y = 0;
-    while (x < all.size() && y < acc.slot.size()) {
-        if (crd_equal(all[x], acc.slot[y])) {
-            Component c = all[x++];
-            c.val += acc.slot[y++].val;
-            out.push_back(c);
-        } else if (crd_less(all[x], acc.slot[y])) {
-            out.push_back(all[x++]);
-        } else {
-            out.push_back(acc.slot[y++]);
+    // Moves everything pending into the settled store.
+    void settle() {
+        if (pending_.empty()) return;
+        // order by coordinate, keeping arrival order among equals, then sum runs of equals
+        std::stable_sort(pending_.begin(), pending_.end(), before);
+        size_t kept = 0;
+        for (size_t x = 0; x < pending_.size(); ++x) {
+            if (kept > 0 && same_place(pending_[kept - 1], pending_[x])) pending_[kept - 1].v += pending_[x].v;
+            else pending_[kept++] = pending_[x];
         }
+        pending_.resize(kept);
+        // union of two duplicate-free sorted sequences into a fresh one; a coordinate present in
+        // both becomes settled value + pending value
+        std::vector<Entry> joined(settled_.size() + pending_.size());
+        std::merge(settled_.begin(), settled_.end(), pending_.begin(), pending_.end(), joined.begin(), before);
+        kept = 0;
+        for (size_t x = 0; x < joined.size(); ++x) {
+            if (kept > 0 && same_place(joined[kept - 1], joined[x])) joined[kept - 1].v += joined[x].v;
+            else joined[kept++] = joined[x];
+        }
+        joined.resize(kept);
+        settled_.swap(joined);
+        pending_.clear();
     }
-    while (x < all.size()) out.push_back(all[x++]);
-    while (y < acc.slot.size()) out.push_back(acc.slot[y++]);
-    all.swap(out);
-    acc.slot.clear();
-    acc.full = false;
-}
 
-void insert_with_flush(const Component& c, AccArray& acc, std::vector<Component>& all) {
-    Insert(c, acc);
-    if (acc.full) {
-        Sort(acc);
-        Merge(acc, all);
-        Insert(c, acc);
-    }
-}
+    const std::vector<Entry>& settled() const { return settled_; }
+
+private:
+    size_t capacity_;
+    std::vector<Entry> pending_, settled_;
+};
 
 }  // namespace
 
@@ -267,63 +250,46 @@ void* oracle_ttm(int64_t n_i, const int32_t* Acrd0, const int64_t* Apos1, const 
     return R;
 }
 
-// Algorithm 1, first-order workspace per output row (key = j), capacity `cap` >= 1.
+// Algorithm 1, one first-order workspace per output row (coordinate = j), capacity `cap` >= 1.
 void* oracle_ism_rowwise(int64_t m, const int64_t* Apos, const int32_t* Acrd, const double* Aval,
                          const int64_t* Bpos, const int32_t* Bcrd, const double* Bval, int64_t cap) {
     Result* R = new Result;
     R->pos.push_back(0);
     for (int64_t i = 0; i < m; ++i) {
-        AccArray acc(static_cast<size_t>(cap));               // Allocate
-        std::vector<Component> all;
+        BoundedWorkspace ws(cap);
         for (int64_t p = Apos[i]; p < Apos[i + 1]; ++p) {
             const int32_t k = Acrd[p];
-            for (int64_t q = Bpos[k]; q < Bpos[k + 1]; ++q) {
-                Component c;
-                c.crd[0] = 0;
-                c.crd[1] = Bcrd[q];
-                c.val = Aval[p] * Bval[q];
-                insert_with_flush(c, acc, all);
-            }
+            for (int64_t q = Bpos[k]; q < Bpos[k + 1]; ++q) ws.feed(Entry{0, Bcrd[q], Aval[p] * Bval[q]});
         }
-        if (!acc.empty()) { Sort(acc); Merge(acc, all); }
-        for (const Component& c : all) { R->crd.push_back(c.crd[1]); R->val.push_back(c.val); }  // Compress
+        ws.settle();
+        for (const Entry& e : ws.settled()) { R->crd.push_back(e.j); R->val.push_back(e.v); }
         R->pos.push_back(static_cast<int64_t>(R->crd.size()));
     }
     R->val_ref = R->val;
     return R;
 }
 
-// Algorithm 1, second-order workspace, loop order k -> i -> j.  At holds A by columns, i.e.
-// the CSR arrays of A transposed (K rows): row k lists the i with A(i,k) != 0.
+// Algorithm 1 with ONE second-order workspace (coordinate = (i, j)) for the whole product, fed
+// in the outer-product order of Sec. 2.1: for each k, every stored A(i,k) times every stored
+// B(k,j).  At holds A by columns, i.e. the CSR arrays of A transposed (K rows): row k lists the
+// i with A(i,k) != 0.  The settled store is the result in coordinate (COO) form; turning it into
+// CSR needs the number of entries of each row, prefix-summed.
 void* oracle_ism_outer(int64_t m, int64_t K, const int64_t* Atpos, const int32_t* Atcrd, const double* Atval,
                        const int64_t* Bpos, const int32_t* Bcrd, const double* Bval, int64_t cap) {
-    AccArray acc(static_cast<size_t>(cap));
-    std::vector<Component> all;
-    for (int64_t k = 0; k < K; ++k) {
-        for (int64_t p = Atpos[k]; p < Atpos[k + 1]; ++p) {
-            Component c;
-            c.crd[0] = Atcrd[p];
-            for (int64_t q = Bpos[k]; q < Bpos[k + 1]; ++q) {
-                c.crd[1] = Bcrd[q];
-                c.val = Atval[p] * Bval[q];
-                insert_with_flush(c, acc, all);
-            }
-        }
-    }
-    if (!acc.empty()) { Sort(acc); Merge(acc, all); }
-    // Compress: COO -> CSR.  Count the components of each row segment, then prefix-sum.
+    BoundedWorkspace ws(cap);
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t p = Atpos[k]; p < Atpos[k + 1]; ++p)
+            for (int64_t q = Bpos[k]; q < Bpos[k + 1]; ++q) ws.feed(Entry{Atcrd[p], Bcrd[q], Atval[p] * Bval[q]});
+    ws.settle();
     Result* R = new Result;
-    R->pos.assign(static_cast<size_t>(m) + 1, 0);
-    size_t w = 0;
-    while (w < all.size()) {
-        const int32_t i = all[w].crd[0];
-        size_t end = w + 1;
-        while (end < all.size() && all[end].crd[0] == i) ++end;
-        R->pos[static_cast<size_t>(i) + 1] = static_cast<int64_t>(end - w);
-        w = end;
+    std::vector<int64_t> per_row(static_cast<size_t>(m), 0);
+    for (const Entry& e : ws.settled()) {
+        ++per_row[static_cast<size_t>(e.i)];
+        R->crd.push_back(e.j);
+        R->val.push_back(e.v);
     }
-    for (int64_t r = 1; r <= m; ++r) R->pos[r] += R->pos[r - 1];
-    for (const Component& c : all) { R->crd.push_back(c.crd[1]); R->val.push_back(c.val); }
+    R->pos.assign(1, 0);
+    for (int64_t r = 0; r < m; ++r) R->pos.push_back(R->pos.back() + per_row[static_cast<size_t>(r)]);
     R->val_ref = R->val;
     return R;
 }
