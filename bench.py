@@ -300,8 +300,6 @@ def main():
         kbytes = (dense_p - dw_p) * (4 + V) + (dense_n - dw_n) * V
     elif top == "num_dense_emit":                   # writes the coordinates
         kbytes = (dense_n - dw_n) * 4
-    elif top == "num_dense_zero":
-        kbytes = 0
     elif top == "sym_dense_warp":
         kbytes = pc[4] * 4
     elif top == "sym_dense_cta":

@@ -142,11 +142,11 @@ enum {
     SPWS_T_NUM_ISM_SMEM_S = 10,
     SPWS_T_NUM_ISM_SMEM = 11,
     SPWS_T_NUM_DENSE_WARP = 12,
-    SPWS_T_NUM_DENSE_ZERO = 13, /* clears the value segments the CTA dense kernel adds into        */
+    SPWS_T_NUM_DENSE_EMIT = 13, /* coordinates of the CTA dense rows; clears the value segments
+                                 that several work units add into                                  */
     SPWS_T_NUM_DENSE_CTA = 14,
-    SPWS_T_NUM_DENSE_EMIT = 15, /* coordinates of the CTA dense rows                               */
-    SPWS_T_NUM_ISM_GLOBAL = 16,
-    SPWS_T_COUNT = 17
+    SPWS_T_NUM_ISM_GLOBAL = 15,
+    SPWS_T_COUNT = 16
 };
 
 spws_status_t spws_create(spws_handle_t* handle);
@@ -226,7 +226,8 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
  * fixed 64 KiB array that is part of the library image and therefore sits on every GPU that
  * loads the library until the process exits.  It calls no allocation routine of any kind.
  *
- * counts : DEVICE, int32, n entries (row i's number of stored outputs).
+ * counts : DEVICE, int32, n entries (row i's number of stored outputs), each >= 0; all sums are
+ *          carried in 64 bits, so any non-negative int32 counts are admissible.
  * pos    : DEVICE, int64, n+1 entries, written by the call; pos[n] is the total.
  * n      : 0 <= n <= SPWS_STATIC_MAX_ROWS; a larger n is refused with SPWS_SCRATCH_TOO_SMALL and
  *          nothing is launched.

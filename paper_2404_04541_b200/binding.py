@@ -38,7 +38,7 @@ EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create",
 STATIC_MAX_ROWS = 16777216
 TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense_warp",
                  "sym_dense_cta", "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem",
-                 "num_dense_warp", "num_dense_zero", "num_dense_cta", "num_dense_emit", "num_ism_global")
+                 "num_dense_warp", "num_dense_emit", "num_dense_cta", "num_ism_global")
 # class index of each per-class kernel group (rows_per_class / products_per_class / nnz_per_class)
 CLASS_NAMES = ("empty", "ism_reg", "ism_smem_s", "ism_smem", "dense_warp", "dense_hub", "dense_cta", "ism_global")
 

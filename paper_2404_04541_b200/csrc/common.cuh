@@ -24,6 +24,7 @@ enum RowClass : int {
 };
 constexpr int NUM_SLOT = 16;   // work_counter[cls] in the symbolic pass, work_counter[NUM_SLOT + cls] in the numeric pass
 constexpr int EMIT_SLOT = 30;  // work_counter slot of the coordinate emission of the CTA dense route
+constexpr int BW_SLOT = 31;    // work_counter slot of the word-list build
 // index of a class in the public statistics (the three register classes are reported as one)
 __host__ __device__ inline int public_class(int cls) { return cls == 0 ? 0 : (cls <= 3 ? 1 : cls - 2); }
 
@@ -33,6 +34,11 @@ constexpr int DENSE_WARP_ACC = 256;        // outputs a warp-per-row numeric wor
 constexpr int DENSE_WARP_MAX_UB = 4096;    // products a single warp is given at most
 constexpr i64 DENSE_HUB_UB = 1ll << 17;    // rows with at least this many products are scheduled first
 constexpr int DENSE_MAX_SPAN_WORDS = 16384;// 2^19 columns: the widest bitmap (8 bytes per word with its rank) one CTA holds
+// Word lists of long B rows (symbolic pass of the CTA dense route): a B row with at least
+// BW_MIN_LEN entries whose entries share bitmap words is also kept as (word index, bits) pairs,
+// so that a row that picks it sets one word per pair instead of one bit per entry.
+constexpr int BW_MIN_LEN = 256;
+constexpr i64 BW_MAX_NNZ = 1ll << 26;      // lists are built only for a B with at most this many entries
 
 enum DevStatus : int {
     DEV_OK = 0,
@@ -55,7 +61,7 @@ struct DevCtl {
     int n_warp_rows;        // numeric dense warp rows
     int max_span_words;     // widest bitmap among the dense rows
     int max_warp_cnt;       // most outputs of a row the warp numeric kernel takes
-    int pad_;
+    int n_long;             // B rows with at least BW_MIN_LEN entries (candidates for a word list)
     int class_count[NCLASS];
     int class_cursor[NCLASS];
     int work_counter[32];   // dynamic work distribution; cleared before each pass
@@ -178,12 +184,16 @@ struct LaunchCtx {
     char* rest;              // scratch after the fixed tables: bitmap arena, then the ISM-global arena
     size_t rest_bytes;
     int global_cap;          // accumulation-array capacity of CLS_ISM_GLOBAL
+    uint2* bw;               // word lists of long B rows, indexed like B's entries (null: not built)
+    int* bw_long;            // the long B rows, in arrival order
+    int bw_long_cap;
     mutable int launches;    // kernels enqueued through this context
 };
 
 // setup.cu
 cudaError_t launch_validate(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA, i64 nnzB);
 cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA);
+cudaError_t launch_bw_build(const LaunchCtx& c, const Csr& B);
 cudaError_t launch_bin_rows(const LaunchCtx& c, int m);
 cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr);
 cudaError_t launch_class_nnz(const LaunchCtx& c, int m);
@@ -200,7 +210,7 @@ cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B
 cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B);
 cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, int max_cnt, const Csr& A, const Csr& B,
                                   const i64* rowptr, int* Ccrd, void* Cval);
-// phase 0: clear the value segments units add into; 1: accumulate; 2: write the coordinates
+// phase 0: write the coordinates and clear the value segments several units add into; 1: accumulate
 cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host, int max_span_words, i64 total_products,
                                  const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,

@@ -19,7 +19,9 @@
 //   CTA units    : any span up to 2^19 columns.  A unit is a row, or an equal share of the A
 //              entries of a row with very many products, so hub rows spread over many CTAs.
 //              The first `unit_outputs` outputs of the row accumulate in shared memory
-//              (atomics combine the CTA's warps), the rest in the row's value segment.
+//              (atomics combine the CTA's warps), the rest in the row's value segment.  The
+//              coordinates of these rows are written by a kernel of their own, which also clears
+//              the value segments that several units add into.
 #include "common.cuh"
 
 namespace spws {
@@ -168,7 +170,8 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
 // ---------------------------------------------------------------------------------------
 // symbolic, CTA per row (hub rows first: classes HUB and CTA are adjacent in perm)
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, Csr A, Csr B, RowTables tab) {
+__global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, Csr A, Csr B, RowTables tab,
+                                                                   const uint2* __restrict__ bw) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned* bm = reinterpret_cast<unsigned*>(smem_raw);                 // smem_words
     int* chunk = reinterpret_cast<int*>(bm + smem_words);                  // smem_words / 32
@@ -190,6 +193,7 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
         const int base = tab.jmin[row];
         const int nw = min((tab.jmax[row] - base) / 32 + 1, smem_words);
         const unsigned span = (unsigned)nw * 32u;
+        const unsigned base_w = (unsigned)base >> 5;                     // base is a multiple of 32
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         for (int w = tid; w < nw; w += DC_THREADS) bm[w] = 0;
         __syncthreads();
@@ -200,6 +204,29 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
             if ((unsigned)k >= (unsigned)B.nrows) continue;
             const i64 qs = __ldg(B.pos + k);
             const int len = (int)(__ldg(B.pos + k + 1) - qs);
+            if (bw && len >= BW_MIN_LEN) {
+                // a long B row with a word list: one atomic per (word, bits) pair, and the lanes
+                // of a warp hold distinct words
+                const int np = (int)__ldg(&bw[qs].x);
+                if (np > 0) {
+                    const uint2* __restrict__ pk = bw + qs + 1;
+                    int t = gl;
+                    for (; t + 3 * gs < np; t += 4 * gs) {
+                        const uint2 e0 = __ldg(pk + t), e1 = __ldg(pk + t + gs), e2 = __ldg(pk + t + 2 * gs), e3 = __ldg(pk + t + 3 * gs);
+                        const unsigned w0 = e0.x - base_w, w1 = e1.x - base_w, w2 = e2.x - base_w, w3 = e3.x - base_w;
+                        if (w0 < (unsigned)nw) atomicOr(&bm[w0], e0.y);
+                        if (w1 < (unsigned)nw) atomicOr(&bm[w1], e1.y);
+                        if (w2 < (unsigned)nw) atomicOr(&bm[w2], e2.y);
+                        if (w3 < (unsigned)nw) atomicOr(&bm[w3], e3.y);
+                    }
+                    for (; t < np; t += gs) {
+                        const uint2 e0 = __ldg(pk + t);
+                        const unsigned w0 = e0.x - base_w;
+                        if (w0 < (unsigned)nw) atomicOr(&bm[w0], e0.y);
+                    }
+                    continue;
+                }
+            }
             const int* __restrict__ ck = B.crd + qs;
             int t = gl;
             for (; t + 3 * gs < len; t += 4 * gs) {     // four loads in flight per lane
@@ -422,23 +449,6 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 constexpr int DN_ENTRIES = 768;      // A entries whose descriptors are staged per round
 constexpr int DN_TILE = 256;         // products a warp takes per fetch
 
-// Zero the value segments of the rows that several units add into (a row with a single unit
-// clears its own overflow part inside the accumulate kernel).
-template <typename T>
-__global__ void __launch_bounds__(256) dense_zero_kernel(DevCtl* __restrict__ ctl, int CAP, i64 unit_products, RowTables tab,
-                                                         const i64* __restrict__ rowptr, T* __restrict__ Cval) {
-    if (ctl->status != 0) return;
-    const int n_units = ctl->n_units;
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-        const int row = tab.unit_row[u];
-        if (u != tab.row_unit0[row]) continue;
-        if (dense_units_of_row(tab.ub[row], unit_products) == 1) continue;
-        const i64 out0 = rowptr[row];
-        const int cnt = (int)(rowptr[row + 1] - out0);
-        for (int x = threadIdx.x; x < cnt; x += 256) Cval[out0 + x] = 0;
-    }
-}
-
 template <typename T>
 __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, i64 unit_products,
                                                                    Csr A, Csr B, RowTables tab, const i64* __restrict__ rowptr,
@@ -648,97 +658,115 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
     }
 }
 
-// Coordinates of the CTA-unit rows.  A warp takes a row at a time and walks its saved bitmap in
-// groups of four 32-word chunks; the outputs of a group are the contiguous range that starts at
-// the first chunk's saved rank, so the group is expanded into a small shared-memory stage and
-// stored with contiguous writes.  The loads of the next group (and the ranks of the one after)
-// are issued before the current group is expanded.
+// Coordinates of the CTA-unit rows, and the clearing of the value segments that several units
+// add into.  Runs before the accumulation kernel.  The saved bitmap carries the rank at every
+// 32-word chunk, so any stretch of a row can be expanded on its own: unit c of a row's n units
+// takes the c-th n-th of the row's 128-word groups, which spreads a hub row over as many warps as
+// it has units.  A warp takes one group at a time, four consecutive words per lane (one 16-byte
+// load); the lanes' bit counts are scanned once per group.  Unless the non-empty words of a group
+// are half full on average, every lane expands its own words into a small shared-memory stage at
+// their ranks and the stage goes out with contiguous stores; otherwise the warp takes one word
+// per step with a lane per bit.
 constexpr int DE_THREADS = 256;
 constexpr int DE_WARPS = DE_THREADS / 32;
-constexpr int DE_STAGE = 1024;       // coordinates a warp stages at once (one full chunk)
+constexpr int DE_STAGE = 2048;       // coordinates a warp stages at once (128 words, 16 bits each on average)
 
-__global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __restrict__ ctl, RowTables tab,
-                                                                    const i64* __restrict__ rowptr, int* __restrict__ Ccrd) {
-    __shared__ int s_stage[DE_WARPS][DE_STAGE];
+template <typename T>
+__global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __restrict__ ctl, i64 unit_products, RowTables tab,
+                                                                    const i64* __restrict__ rowptr, int* __restrict__ Ccrd,
+                                                                    T* __restrict__ Cval) {
+    __shared__ unsigned short s_stage[DE_WARPS][DE_STAGE];
     if (ctl->status != 0) return;
     const int n_units = ctl->n_units;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int* stage = s_stage[warp];
-    for (;;) {                                          // rows differ a lot in set bits: deal them out dynamically
+    unsigned short* stage = s_stage[warp];
+    for (;;) {
         int u = 0;
         if (lane == 0) u = atomicAdd(&ctl->work_counter[EMIT_SLOT], 1);
         u = __shfl_sync(0xffffffffu, u, 0);
         if (u >= n_units) break;
         const int row = tab.unit_row[u];
-        if (u != tab.row_unit0[row]) continue;
+        const int uidx = u - tab.row_unit0[row];
+        const int nun = dense_units_of_row(tab.ub[row], unit_products);
         const int base = tab.jmin[row];
         const int nw = (tab.jmax[row] - base) / 32 + 1;
         const int nch = chunks_of(nw);
+        const int ng = (nch + 3) >> 2;                                  // groups of four chunks = 128 words
+        const int g_lo = (int)((i64)ng * uidx / nun), g_hi = (int)((i64)ng * (uidx + 1) / nun);
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
+        const uint4* src4 = reinterpret_cast<const uint4*>(src);         // slots are 16-byte aligned
         const i64 out0 = rowptr[row];
         const int cnt_row = (int)(rowptr[row + 1] - out0);
+        const bool clear = nun > 1;                                      // several units add into this row's values
 
-        // lanes 0..4 hold the ranks at the starts of chunks c0 .. c0+4 (the row's count past the end)
-        auto load_ranks = [&](int c0) {
-            int r = cnt_row;
-            if (lane < 5 && c0 + lane < nch) r = (int)src[nw + c0 + lane];
-            return r;
-        };
-        // word `lane` of chunk c0+x unless that chunk is empty (equal ranks at both ends)
-        auto load_word = [&](int c0, int x, int ranks) {
-            const int n = __shfl_sync(0xffffffffu, ranks, x + 1) - __shfl_sync(0xffffffffu, ranks, x);
-            const int w = ((c0 + x) << 5) + lane;
-            return (w < nw && n > 0) ? src[w] : 0u;
-        };
-        int rk = load_ranks(0);
-        unsigned w0 = load_word(0, 0, rk), w1 = load_word(0, 1, rk), w2 = load_word(0, 2, rk), w3 = load_word(0, 3, rk);
-        int rk_next = load_ranks(4);
-        for (int c0 = 0; c0 < nch; c0 += 4) {
-            const unsigned n0 = load_word(c0 + 4, 0, rk_next), n1 = load_word(c0 + 4, 1, rk_next);
-            const unsigned n2 = load_word(c0 + 4, 2, rk_next), n3 = load_word(c0 + 4, 3, rk_next);
-            const int rk_next2 = load_ranks(c0 + 8);
-
-            const int r0 = __shfl_sync(0xffffffffu, rk, 0);
-            const int n_all = __shfl_sync(0xffffffffu, rk, 4) - r0;
-            if (n_all > 0) {
-                // exclusive ranks of the four words of this lane inside their chunks: two scans of
-                // two 16-bit counts each
-                const int p0 = __popc(w0), p1 = __popc(w1), p2 = __popc(w2), p3 = __popc(w3);
-                const unsigned sa = (unsigned)warp_incl_scan(p0 | (p1 << 16)), sb = (unsigned)warp_incl_scan(p2 | (p3 << 16));
-                const int e0 = (int)(sa & 0xffffu) - p0, e1 = (int)(sa >> 16) - p1;
-                const int e2 = (int)(sb & 0xffffu) - p2, e3 = (int)(sb >> 16) - p3;
-                const int col = base + (((c0 << 5) + lane) << 5);
-                auto expand = [&](unsigned word, int slot, int col0) {
-                    while (word) {
-                        const int b = __ffs(word) - 1;
-                        word &= word - 1;
-                        stage[slot++] = col0 + b;
-                    }
-                };
-                auto flush = [&](int rank0, int n) {
-                    __syncwarp();
-                    const i64 o = out0 + rank0;
-                    for (int y = lane; y < n; y += 32) Ccrd[o + y] = stage[y];
-                    __syncwarp();
-                };
-                if (n_all <= DE_STAGE) {
-                    expand(w0, e0, col);
-                    expand(w1, __shfl_sync(0xffffffffu, rk, 1) - r0 + e1, col + 1024);
-                    expand(w2, __shfl_sync(0xffffffffu, rk, 2) - r0 + e2, col + 2048);
-                    expand(w3, __shfl_sync(0xffffffffu, rk, 3) - r0 + e3, col + 3072);
-                    flush(r0, n_all);
-                } else {
-                    const int r1 = __shfl_sync(0xffffffffu, rk, 1), r2 = __shfl_sync(0xffffffffu, rk, 2);
-                    const int r3 = __shfl_sync(0xffffffffu, rk, 3), r4 = r0 + n_all;
-                    expand(w0, e0, col);        flush(r0, r1 - r0);
-                    expand(w1, e1, col + 1024); flush(r1, r2 - r1);
-                    expand(w2, e2, col + 2048); flush(r2, r3 - r2);
-                    expand(w3, e3, col + 3072); flush(r3, r4 - r3);
-                }
+        // words 128 g + 4 lane .. + 3 (zero past the end of the bitmap) and the ranks at both ends of group g
+        auto load_group = [&](int g, uint4& w, int& r0, int& r1) {
+            w = make_uint4(0u, 0u, 0u, 0u);
+            r0 = r1 = cnt_row;
+            if (g >= g_hi) return;
+            const int w0 = (g << 7) + (lane << 2);
+            if (w0 < nw) {
+                w = src4[(g << 5) + lane];
+                if (w0 + 1 >= nw) w.y = 0u;
+                if (w0 + 2 >= nw) w.z = 0u;
+                if (w0 + 3 >= nw) w.w = 0u;
             }
-            w0 = n0; w1 = n1; w2 = n2; w3 = n3;
-            rk = rk_next;
-            rk_next = rk_next2;
+            r0 = (int)src[nw + (g << 2)];
+            if ((g << 2) + 4 < nch) r1 = (int)src[nw + (g << 2) + 4];
+        };
+        uint4 w, wn;
+        int r0, r1, r0n, r1n;
+        load_group(g_lo, w, r0, r1);
+        for (int g = g_lo; g < g_hi; ++g) {
+            load_group(g + 1, wn, r0n, r1n);                             // next group's loads fly during this expansion
+            const int n = r1 - r0;
+            if (n > 0) {
+                const int p = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
+                const int e = warp_incl_scan(p) - p;
+                const int col = base + (((g << 7) + (lane << 2)) << 5);
+                const i64 o = out0 + r0;
+                const unsigned m0 = __ballot_sync(0xffffffffu, w.x != 0u), m1 = __ballot_sync(0xffffffffu, w.y != 0u);
+                const unsigned m2 = __ballot_sync(0xffffffffu, w.z != 0u), m3 = __ballot_sync(0xffffffffu, w.w != 0u);
+                const int nzw = __popc(m0) + __popc(m1) + __popc(m2) + __popc(m3);
+                if (n <= DE_STAGE && n < 16 * nzw) {
+                    // every lane expands its own four words into the stage at their ranks (as 16-bit
+                    // offsets from the group's first column), then the stage goes out with
+                    // contiguous stores
+                    int slot = e;
+                    auto expand = [&](unsigned word, int off0) {
+                        while (word) {
+                            const int b = __ffs(word) - 1;
+                            word &= word - 1;
+                            stage[slot++] = (unsigned short)(off0 + b);
+                        }
+                    };
+                    const int off = lane << 7;
+                    expand(w.x, off); expand(w.y, off + 32); expand(w.z, off + 64); expand(w.w, off + 96);
+                    __syncwarp();
+                    const int gcol0 = base + (g << 12);
+                    for (int y = lane; y < n; y += 32) Ccrd[o + y] = gcol0 + (int)stage[y];
+                    __syncwarp();
+                } else {
+                    // half-full words or fuller: the warp expands one non-empty word per step, lane
+                    // b testing bit b, so the word's outputs leave as one contiguous store
+                    const unsigned below = (1u << lane) - 1u;
+                    const int gcol = base + (g << 12) + lane;
+                    auto spread = [&](unsigned mine, int rank_mine, unsigned m, int x) {
+                        while (m) {
+                            const int L = __ffs(m) - 1;
+                            m &= m - 1;
+                            const unsigned word = __shfl_sync(0xffffffffu, mine, L);
+                            const int at = __shfl_sync(0xffffffffu, rank_mine, L);
+                            if ((word >> lane) & 1u) Ccrd[o + at + __popc(word & below)] = gcol + (((L << 2) + x) << 5);
+                        }
+                    };
+                    const int e1 = e + __popc(w.x), e2 = e1 + __popc(w.y), e3 = e2 + __popc(w.z);
+                    spread(w.x, e, m0, 0); spread(w.y, e1, m1, 1); spread(w.z, e2, m2, 2); spread(w.w, e3, m3, 3);
+                }
+                if (clear)
+                    for (int y = lane; y < n; y += 32) Cval[o + y] = (T)0;
+            }
+            w = wn; r0 = r0n; r1 = r1n;
         }
     }
 }
@@ -767,7 +795,7 @@ cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B)
     int per_sm = 0;
     if ((e = cudaFuncSetAttribute(dense_sym_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_sym_cta_kernel, DC_THREADS, smem)) != cudaSuccess) return e;
-    dense_sym_cta_kernel<<<persistent_grid(c, per_sm, -1), DC_THREADS, smem, c.stream>>>(c.ctl, c.dense_smem_words, A, B, c.tab);
+    dense_sym_cta_kernel<<<persistent_grid(c, per_sm, -1), DC_THREADS, smem, c.stream>>>(c.ctl, c.dense_smem_words, A, B, c.tab, c.bw);
     ++c.launches;
     return cudaGetLastError();
 }
@@ -809,16 +837,15 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int phase, int n_units_host, in
     auto k = dense_num_cta_kernel<T>;
     if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DN_THREADS, smem)) != cudaSuccess) return e;
-    if (phase == 0)
-        dense_zero_kernel<T><<<persistent_grid(c, 8, n_units_host), 256, 0, c.stream>>>(c.ctl, CAP, unit_products, c.tab, rowptr, (T*)Cval);
-    else if (phase == 1)
+    if (phase == 0) {
+        // units are dealt out dynamically, so the grid is what is resident at once
+        int emit_per_sm = 0;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&emit_per_sm, dense_emit_crd_kernel<T>, DE_THREADS, 0)) != cudaSuccess) return e;
+        const i64 work = n_units_host >= 0 ? ((i64)n_units_host + DE_WARPS - 1) / DE_WARPS : -1;
+        dense_emit_crd_kernel<T><<<persistent_grid(c, emit_per_sm, work), DE_THREADS, 0, c.stream>>>(c.ctl, unit_products, c.tab, rowptr, Ccrd, (T*)Cval);
+    } else {
         k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab,
                                                                                  rowptr, Ccrd, (T*)Cval);
-    else {
-        // rows are dealt out by grid stride, so the grid must be exactly what is resident at once
-        int emit_per_sm = 0;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&emit_per_sm, dense_emit_crd_kernel, DE_THREADS, 0)) != cudaSuccess) return e;
-        dense_emit_crd_kernel<<<persistent_grid(c, emit_per_sm, n_units_host), DE_THREADS, 0, c.stream>>>(c.ctl, c.tab, rowptr, Ccrd);
     }
     ++c.launches;
     return cudaGetLastError();

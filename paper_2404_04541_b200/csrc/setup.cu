@@ -147,6 +147,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         if (bad) raise_status(ctl, DEV_NONCANONICAL);
         if (gl == 0) {
             if (lo < 0 || hi >= B.ncols) { raise_status(ctl, DEV_NONCANONICAL); u = 0; }
+            if (u > 0) lo &= ~31;               // bitmap words of every row start at a multiple of 32 columns
             const int cls = classify_row(u, lo, hi, prm, ctl);
             tab.ub[row] = u;
             tab.jmin[row] = lo;
@@ -205,6 +206,90 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
     else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
     else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
     ++c.launches;
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Word lists of long B rows.  The list of row k lives in `bw` at the positions of the row's own
+// entries: bw[pos[k]] is a header (.x = number of pairs, 0 = no list), the pairs (.x = column / 32,
+// .y = the bits of the row's entries in that word) follow.  A list is kept only when it has at
+// most three quarters as many pairs as the row has entries.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) bw_find_long_kernel(Csr B, int* __restrict__ bw_long, int cap, DevCtl* ctl) {
+    for (i64 k = (i64)blockIdx.x * blockDim.x + threadIdx.x; k < B.nrows; k += (i64)gridDim.x * blockDim.x) {
+        if (B.pos[k + 1] - B.pos[k] >= BW_MIN_LEN) {
+            const int at = atomicAdd(&ctl->n_long, 1);
+            if (at < cap) bw_long[at] = (int)k;
+        }
+    }
+}
+
+constexpr int BWB_THREADS = 256;
+constexpr int BWB_ITEMS = 4;
+
+__global__ void __launch_bounds__(BWB_THREADS) bw_build_kernel(Csr B, const int* __restrict__ bw_long, int cap,
+                                                              uint2* __restrict__ bw, DevCtl* ctl) {
+    __shared__ int ws[33];
+    __shared__ int s_next;
+    const int n_long = min(ctl->n_long, cap);
+    const int tid = threadIdx.x;
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[BW_SLOT], 1);
+        __syncthreads();
+        if (s_next >= n_long) break;
+        const int k = bw_long[s_next];
+        const i64 qs = B.pos[k], qe = B.pos[k + 1];
+        const i64 len = qe - qs;
+        const int* __restrict__ crd = B.crd;
+        int carry = 0;                                   // pairs of the row before this tile
+        for (i64 t0 = qs; t0 < qe; t0 += BWB_THREADS * BWB_ITEMS) {
+            const i64 q0 = t0 + (i64)tid * BWB_ITEMS;
+            unsigned word[BWB_ITEMS], bits[BWB_ITEMS];
+            int nfirst = 0;
+            unsigned prev = (q0 > qs && q0 < qe) ? ((unsigned)__ldg(crd + q0 - 1) >> 5) : 0xffffffffu;
+#pragma unroll
+            for (int x = 0; x < BWB_ITEMS; ++x) {
+                const i64 q = q0 + x;
+                word[x] = 0xffffffffu;                   // not the first entry of a word
+                bits[x] = 0u;
+                if (q < qe) {
+                    const unsigned c = (unsigned)__ldg(crd + q);
+                    if ((c >> 5) != prev) {
+                        word[x] = c >> 5;
+                        unsigned b = 1u << (c & 31);
+                        for (i64 q2 = q + 1; q2 < qe; ++q2) {          // at most 31 more entries share the word
+                            const unsigned c2 = (unsigned)__ldg(crd + q2);
+                            if ((c2 >> 5) != word[x]) break;
+                            b |= 1u << (c2 & 31);
+                        }
+                        bits[x] = b;
+                        ++nfirst;
+                    }
+                    prev = c >> 5;
+                }
+            }
+            int total;
+            int at = carry + block_excl_scan<BWB_THREADS>(nfirst, ws, total);
+#pragma unroll
+            for (int x = 0; x < BWB_ITEMS; ++x)
+                if (word[x] != 0xffffffffu) {
+                    if (at + 1 < len) bw[qs + 1 + at] = make_uint2(word[x], bits[x]);
+                    ++at;
+                }
+            carry += total;
+        }
+        if (tid == 0) bw[qs] = make_uint2(4 * (i64)carry <= 3 * len ? (unsigned)carry : 0u, 0u);
+    }
+}
+
+cudaError_t launch_bw_build(const LaunchCtx& c, const Csr& B) {
+    if (!c.bw || B.nrows == 0) return cudaSuccess;
+    i64 want = ((i64)B.nrows + 255) / 256;
+    i64 cap = (i64)c.sm_count * 8;
+    bw_find_long_kernel<<<(int)(want < cap ? want : cap), 256, 0, c.stream>>>(B, c.bw_long, c.bw_long_cap, c.ctl);
+    bw_build_kernel<<<c.sm_count * 8, BWB_THREADS, 0, c.stream>>>(B, c.bw_long, c.bw_long_cap, c.bw, c.ctl);
+    c.launches += 2;
     return cudaGetLastError();
 }
 
@@ -446,19 +531,30 @@ __global__ void __launch_bounds__(1024) scan_block_sums_kernel(i64* block_sums, 
     }
 }
 
+// The in-tile prefix is carried in 64 bits: a tile of 2048 counts may total 2^31 or more.
 __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int* __restrict__ in, int n, const i64* __restrict__ block_sums, i64* __restrict__ out) {
-    __shared__ int ws[33];
+    __shared__ i64 s_warp[SCAN_THREADS / 32];
     const i64 base = (i64)blockIdx.x * SCAN_TILE + (i64)threadIdx.x * SCAN_ITEMS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int v[SCAN_ITEMS];
-    int s = 0;
+    i64 s = 0;
 #pragma unroll
     for (int x = 0; x < SCAN_ITEMS; ++x) {
         v[x] = (base + x < n) ? in[base + x] : 0;
         s += v[x];
     }
-    int total;
-    const int excl = block_excl_scan<SCAN_THREADS>(s, ws, total);
-    i64 run = block_sums[blockIdx.x] + excl;
+    i64 incl = s;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const i64 t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    i64 before = 0;
+#pragma unroll
+    for (int w = 0; w < SCAN_THREADS / 32; ++w) before += (w < warp) ? s_warp[w] : 0;
+    i64 run = block_sums[blockIdx.x] + before + incl - s;
 #pragma unroll
     for (int x = 0; x < SCAN_ITEMS; ++x) {
         if (base + x < n) out[base + x] = run;
@@ -467,7 +563,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int* __r
 }
 
 cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out) {
-    const int nblocks = (n + SCAN_TILE - 1) / SCAN_TILE;
+    const int nblocks = (int)(((i64)n + SCAN_TILE - 1) / SCAN_TILE);
     if (nblocks > 0) scan_reduce_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums);
     scan_block_sums_kernel<<<1, 1024, 0, c.stream>>>(block_sums, nblocks, out + n, total_out);
     if (nblocks > 0) scan_apply_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums, out);

@@ -116,12 +116,13 @@ bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 // ---- scratch layout ------------------------------------------------------------------------
 struct Layout {
     size_t ctl, ub, rowptr_raw, cnt, jmin, jmax, cls, perm, bm_off, warp_rows, row_unit0, unit_row, block_sums,
-        flags, fpos, sflags, spos, rest, fixed_end;
+        flags, fpos, sflags, spos, bw_long, bw, rest, fixed_end;
     int unit_cap;
+    int bw_long_cap;            // 0: no word lists for this B
     int dense_smem_words;
 };
 
-Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) {
+Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, int64_t nnzB) {
     Layout L{};
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
@@ -152,6 +153,13 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i) 
         L.fpos = take(8 * ((size_t)m + 1));
         L.sflags = take(4 * (size_t)n_i);
         L.spos = take(8 * ((size_t)n_i + 1));
+    }
+    // word lists of long B rows (dense routes): one 8-byte slot per entry of B, used only at the
+    // positions of rows with at least BW_MIN_LEN entries
+    if (p->policy != SPWS_SPARSE_ISM && nnzB >= BW_MIN_LEN && nnzB <= BW_MAX_NNZ) {
+        L.bw_long_cap = (int)(nnzB / BW_MIN_LEN + 1);
+        L.bw_long = take(4 * (size_t)L.bw_long_cap);
+        L.bw = take(8 * (size_t)nnzB);
     }
     L.fixed_end = o;
     L.rest = o;
@@ -255,6 +263,11 @@ LaunchCtx make_ctx(const spws_plan_s* p, char* scratch, size_t scratch_bytes, co
     c.tab.unit_row = reinterpret_cast<int*>(scratch + L.unit_row);
     c.is_f64 = p->is_f64;
     c.global_cap = p->opt.fallback_cap;
+    if (L.bw_long_cap > 0) {
+        c.bw = reinterpret_cast<uint2*>(scratch + L.bw);
+        c.bw_long = reinterpret_cast<int*>(scratch + L.bw_long);
+        c.bw_long_cap = L.bw_long_cap;
+    }
     return c;
 }
 
@@ -410,7 +423,7 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S, false);   // pointers may still be unset when sizing
     if (st != SPWS_OK) return st;
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
     *bytes = L.fixed_end + rest_reserve(plan, S.m, S.ncols);
     return SPWS_OK;
 }
@@ -424,7 +437,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     if (st != SPWS_OK) return st;
     if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
     if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return SPWS_INVALID_ARGUMENT;
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
     if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
     char* sc = static_cast<char*>(scratch);
     LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
@@ -440,6 +453,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     // a1: upper bounds + classes; a2: binning
     mark_start(plan, 0);
     CUDA_TRY(launch_row_bounds(c, S.A, S.B, S.nnzA));
+    CUDA_TRY(launch_bw_build(c, S.B));
     mark(plan, SPWS_T_SYM_BOUNDS);
     CUDA_TRY(launch_bin_rows(c, (int)S.m));
     mark(plan, SPWS_T_SYM_BIN);
@@ -530,7 +544,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     const int last = plan->kind == 0 ? 1 : 2;
     if (C->n[last] < plan->stats.nnz) return SPWS_OUTPUT_TOO_SMALL;
     if (plan->stats.nnz > 0 && (!C->crd[last] || !C->val)) return SPWS_INVALID_ARGUMENT;
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
     if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
     char* sc = static_cast<char*>(scratch);
     LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
@@ -559,11 +573,9 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     }
     if (s.dense_units > 0) {
         CUDA_TRY(launch_dense_num_cta(c, 0, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
-        mark(plan, SPWS_T_NUM_DENSE_ZERO);
+        mark(plan, SPWS_T_NUM_DENSE_EMIT);
         CUDA_TRY(launch_dense_num_cta(c, 1, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_DENSE_CTA);
-        CUDA_TRY(launch_dense_num_cta(c, 2, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, crd, C->val));
-        mark(plan, SPWS_T_NUM_DENSE_EMIT);
     }
     if (bins[CLS_ISM_GLOBAL] > 0) {
         CUDA_TRY(launch_ism_global(c, true, (int)bins[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));

@@ -341,9 +341,14 @@ def test_full_uniform8(ctx, oracle_mod):
 
 
 def test_full_stencil64(ctx, oracle_mod):
+    """Values in [0.5, 1.5] cannot cancel, so every entry must pass the plain relative clause."""
     c = config_inputs("stencil64")
-    stats = check_spgemm(ctx, oracle_mod, c["A"], c["B"], "auto", threads=oracle_mod.hardware_threads())
-    assert stats["products"] == 566 ** 3 and stats["nnz"] == 314 ** 3
+    A = c["A"]
+    ref = oracle_mod.spgemm(A, A, threads=oracle_mod.hardware_threads())
+    pos, crd, val, stats = run_spgemm(ctx, A, A, "auto")
+    assert stats["products"] == 566 ** 3 and stats["nnz"] == 314 ** 3 == ref.nnz
+    second = assert_matches((pos, crd, val), ref, np.float64)
+    assert second == 0
 
 
 def test_full_wide26(ctx, oracle_mod):
@@ -411,6 +416,81 @@ def test_full_rmat18_sampled_rows_and_invariants(ctx, oracle_mod):
         assert ok.all()
 
 
+def test_full_rmat18_every_entry_streamed(ctx, oracle_mod):
+    """The whole power-law result against the oracle, entry by entry, in the launch configuration
+    the benchmark times.  Both sides are walked in blocks of rows so that neither 15 GB result has
+    to sit in host memory: the oracle computes a block, the matching slices of C come off the
+    device, structure must be identical and every value must pass the two-clause rule."""
+    from paper_2404_04541_b200 import api
+    c = config_inputs("rmat18")
+    A = c["A"]
+    dA = api.DeviceCSR.from_host(A)
+    C, stats = ctx.spgemm(dA, dA, policy="auto")
+    pos = C.pos.cpu().numpy()
+    threads = oracle_mod.hardware_threads()
+    # blocks of about 2^24 products (row boundaries), so that each oracle call stays small
+    lens = np.diff(A.pos)
+    ub = np.bincount(rows_of(A.pos), weights=lens[A.crd], minlength=A.nrows).astype(np.int64)
+    csum = np.concatenate([[0], np.cumsum(ub)])
+    cuts = np.unique(np.searchsorted(csum, np.arange(0, csum[-1], 1 << 25)))
+    cuts = np.unique(np.concatenate([cuts, [0, A.nrows]]))
+    products = entries = second = 0
+    for r0, r1 in zip(cuts[:-1], cuts[1:]):
+        ref = oracle_mod.spgemm(A, A, rows=np.arange(r0, r1), threads=threads)
+        s, e = int(pos[r0]), int(pos[r1])
+        assert np.array_equal(pos[r0:r1 + 1] - s, ref.pos), f"row pointer differs in rows {r0}..{r1}"
+        assert np.array_equal(C.crd[s:e].cpu().numpy(), ref.crd), f"column indices differ in rows {r0}..{r1}"
+        ok, sec = values_close(C.val[s:e].cpu().numpy(), ref.val_ref, ref.abs, 1e-12)
+        assert ok.all(), f"{(~ok).sum()} values out of tolerance in rows {r0}..{r1}"
+        products += int(ref.products.sum())
+        entries += ref.nnz
+        second += sec
+    assert products == stats["products"] and entries == stats["nnz"] == int(pos[-1])
+    print(f"rmat18: {entries} entries compared, {second} needed the sum|a*b| clause")
+
+
+# ------------------------------------------------------------------ row-sharded driver on the device
+def _sharded_worker(rank, world, port, out_dir):
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import torch
+    import torch.distributed as dist
+    from paper_2404_04541_b200 import api
+    from paper_2404_04541_b200 import dist as spd
+    from workloads import rmat_csr
+    torch.cuda.set_device(0)                        # every rank on the one device: ranks share nothing on the data path
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    A = rmat_csr(11, 12, 9)
+    ctx = api.Context("cuda:0")
+    res = spd.spgemm_sharded(A, A, spd.local_spgemm_cuda(ctx))
+    pos, crd, val = spd.gather_full(res, A.nrows)
+    np.savez(os.path.join(out_dir, f"rank{rank}.npz"), pos=pos, crd=crd, val=val, r0=res.row_begin, r1=res.row_end)
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [1, 2])
+def test_sharded_driver_with_the_cuda_local_product(oracle_mod, tmp_path, world):
+    """The row-sharded driver with the CUDA path as the local product (upload of a row block,
+    symbolic + numeric, row-pointer offsets from the size exchange) against the unsharded oracle."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    mp.spawn(_sharded_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    A = rmat_csr(11, 12, 9)
+    ref = oracle_mod.spgemm(A, A)
+    for r in range(world):
+        o = np.load(str(tmp_path / f"rank{r}.npz"))
+        assert np.array_equal(o["pos"], ref.pos) and np.array_equal(o["crd"], ref.crd)
+        ok, _ = values_close(o["val"], ref.val_ref, ref.abs, 1e-12)
+        assert ok.all()
+    if world == 2:
+        a, b = (np.load(str(tmp_path / f"rank{r}.npz")) for r in range(2))
+        assert a["r0"] == 0 and a["r1"] == b["r0"] and b["r1"] == A.nrows
+
+
 # ------------------------------------------------------------------ TTM
 def run_ttm(ctx, A, B, policy="auto", **options):
     from paper_2404_04541_b200 import api
@@ -445,10 +525,11 @@ def test_ttm_small_and_empty_fibres(ctx, oracle_mod, policy):
         check_ttm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
 
 
+@pytest.mark.parametrize("policy", POLICIES)
 @pytest.mark.parametrize("reduced", [True, False])
-def test_ttm_config(ctx, oracle_mod, reduced):
+def test_ttm_config(ctx, oracle_mod, reduced, policy):
     c = config_inputs("ttm4096", reduced=reduced)
-    stats = check_ttm(ctx, oracle_mod, c["A"], c["B"], "auto")
+    stats = check_ttm(ctx, oracle_mod, c["A"], c["B"], policy)
     assert stats["products"] == 8 * c["A"].nnz
 
 
