@@ -176,41 +176,20 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="rmat18",
-                    help="rmat18 (default), stencil64, uniform8, wide26, ttm4096, or rmatNN / stencilNN at another size")
-    ap.add_argument("--policy", default="auto")
-    ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
-    ap.add_argument("--seed", type=int, default=1)
-    ap.add_argument("--opt", action="append", default=[], help="plan option as name=value (repeatable)")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
-    WORKLOAD_TEXT.setdefault(args.workload, f"{args.workload} (same recipe as the named configuration, other size), fp64")
-    if args.impl == "reference":
-        run_reference(args)
-        return
-    if args.warmup < 3:
-        args.warmup = 3
+def percentile_stats(xs):
+    xs = sorted(xs)
+    return float(np.mean(xs)), float(xs[0]), float(np.median(xs))
 
+
+def measure(workload, args, dev, rank, world, dist, e2e=True, cpu_baseline=True):
+    """Times `args.steps` steps of symbolic + numeric on one workload; returns the fields of the
+    bench line that belong to the workload."""
     import torch
-    import torch.distributed as dist
     from paper_2404_04541_b200 import api, binding
     from workloads import config_inputs
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    cfg = config_inputs(args.workload, seed=args.seed + rank)
+    WORKLOAD_TEXT.setdefault(workload, f"{workload} (same recipe as the named configuration, other size), fp64")
+    cfg = config_inputs(workload, seed=args.seed + rank)
     is_ttm = cfg["kind"] == "ttm"
     T3 = cfg["A"] if is_ttm else None           # the CSF operand of the 3-tensor form
     # the 3-tensor form works on the (i,j) fibres as rows: sizes, bytes and the oracle sample use that matrix
@@ -240,10 +219,12 @@ def main():
     crd = torch.empty(nnzC, dtype=torch.int32, device=dev)
     val = torch.empty(nnzC, dtype=vt, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)       # > L2 (126 MB)
+    result = {}
 
     def step():
         cc, st = symbolic(plan, dA, dB)
-        numeric(plan, cc, st, crd=crd, val=val)
+        result["C"] = numeric(plan, cc, st, crd=crd, val=val)
+        result["c"], result["state"] = cc, st
 
     for _ in range(args.warmup):
         step()
@@ -251,7 +232,7 @@ def main():
     stats = plan.get_stats()
     products = stats["products"]
 
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(dev.index or 0)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -264,12 +245,14 @@ def main():
         step()
         ev[s][1].record()
         for g, ms in plan.get_timings().items():                         # synchronises the stream
-            group_ms[g] += ms
+            if not g.startswith("ceil_"):
+                group_ms[g] += ms
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
-    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = sum(step_ms)
     t = torch.tensor([total_ms, float(products), float(nnzC), float(A.nnz), float(A.nrows)], dtype=torch.float64, device=dev)
     if world > 1:
         tmax = t.clone()
@@ -278,13 +261,27 @@ def main():
         total_ms = float(tmax[0])
     all_products, all_nnzC, all_nnzA, all_m = float(t[1]), float(t[2]), float(t[3]), float(t[4])
     ms_per_step = total_ms / args.steps
+    _, ms_min, ms_median = percentile_stats(step_ms)
     value = 2.0 * all_products / (ms_per_step * 1e-3) / 1e9
     abytes = algorithmic_bytes(all_m, all_nnzA, all_products, all_nnzC, V)
     eff_gbs = abytes / (ms_per_step * 1e-3) / 1e9
 
+    # ---- iteration-only ceiling of the dense numeric kernels (outside the timed steps): the same
+    # traversal and gathers with the workspace stripped
+    ceil_ms = {"ceil_dense_warp": 0.0, "ceil_dense_cta": 0.0}
+    if stats["dense_units"] > 0 or stats["dense_warp_rows"] > 0:
+        n_ceil = max(1, min(args.steps, 5))
+        for s in range(1 + n_ceil):
+            flush.fill_(s & 0xff)
+            ctx.gather_ceiling(plan, result["c"], result["state"])
+            if s > 0:                                                    # first run is a warm-up
+                tm = plan.get_timings()
+                for g in ceil_ms:
+                    ceil_ms[g] += tm[g] / n_ceil
+
     # ---- roofline of the dominant kernel (this rank's launches)
     peak, peak_kind = measured_peak()
-    avg = {g: v / args.steps for g, v in group_ms.items()}
+    avg = {g: v / args.steps for g, v in group_ms.items() if not g.startswith("ceil_")}
     top = max(avg, key=avg.get)
     # algorithmic bytes of each per-class kernel group: numeric = index + value per product
     # gathered and per output written; symbolic = index per product gathered
@@ -315,29 +312,34 @@ def main():
         if hashlib.sha256(open(src, "rb").read()).hexdigest().startswith(PROFILED_SOURCE_SHA):
             traffic = PROFILED_TRAFFIC[top]["bytes_per_product"] * kunits
     achieved = kbytes / (avg[top] * 1e-3) / 1e9 if avg[top] > 0 else 0.0
+    ceiling = ceil_ms.get("ceil_" + top[len("num_"):]) if top.startswith("num_") else None
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                "kernel_ms": avg[top], "algorithmic_bytes": kbytes}
+                "kernel_ms": avg[top], "algorithmic_bytes": kbytes,
+                # what the counters say limits this kernel: B is L2-resident, DRAM sees C and the saved bitmaps only
+                "limiter": "SM load/store path (shared-memory atomics, L2 reductions, gather sectors), not DRAM",
+                "dram_frac": (traffic / (avg[top] * 1e-3) / 1e9 / peak) if traffic else None,
+                "ceiling_ms": ceiling, "kernel_over_ceiling": (avg[top] / ceiling) if ceiling else None,
+                "ceiling": "same traversal and gathers, workspace stripped (spws_gather_ceiling)"}
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64" if V == 8 else "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "policy": args.policy, "options": options,
-                       "seed": args.seed, "rows": int(A.nrows), "nnzA": int(A.nnz), "products": int(products),
-                       "nnzC": int(nnzC), "l2": "512 MiB buffer written between timed steps",
-                       "timed": "spws_symbolic + spws_numeric; C buffers preallocated",
-                       **({"rows_are": "the (i,j) fibres of A"} if is_ttm else {})},
-            "effective_gbs": eff_gbs, "algorithmic_bytes_per_step": abytes,
-            "hbm_frac_nominal_8tbs": eff_gbs / NOMINAL_HBM_GBS, "hbm_frac_measured": eff_gbs / peak,
-            "roofline": roofline, "kernel_ms": avg, "rows_per_class": stats["rows_per_class"],
-            "products_per_class": stats["products_per_class"], "nnz_per_class": stats["nnz_per_class"],
-            "dense_units": stats["dense_units"], "dense_warp_rows": stats["dense_warp_rows"],
-            "bitmap_bytes": stats["bitmap_bytes"],
-            "gpu_launches": (stats["launches_symbolic"] + stats["launches_numeric"]) * args.steps,
-            "clocks": clocks}
+    out = {"value": value, "ms_per_step": ms_per_step, "ms_min": ms_min, "ms_median": ms_median,
+           "dtype": "f64" if V == 8 else "f32",
+           "config": {"workload": WORKLOAD_TEXT[workload], "name": workload, "policy": args.policy, "options": options,
+                      "seed": args.seed, "rows": int(A.nrows), "nnzA": int(A.nnz), "products": int(products),
+                      "nnzC": int(nnzC), "l2": "512 MiB buffer written between timed steps",
+                      "timed": "spws_symbolic + spws_numeric; C buffers preallocated",
+                      **({"rows_are": "the (i,j) fibres of A"} if is_ttm else {})},
+           "effective_gbs": eff_gbs, "algorithmic_bytes_per_step": abytes,
+           "hbm_frac_nominal_8tbs": eff_gbs / NOMINAL_HBM_GBS, "hbm_frac_measured": eff_gbs / peak,
+           "roofline": roofline, "kernel_ms": avg, "ceiling_ms": ceil_ms, "rows_per_class": stats["rows_per_class"],
+           "products_per_class": stats["products_per_class"], "nnz_per_class": stats["nnz_per_class"],
+           "dense_units": stats["dense_units"], "dense_warp_rows": stats["dense_warp_rows"],
+           "bitmap_bytes": stats["bitmap_bytes"],
+           "gpu_launches": (stats["launches_symbolic"] + stats["launches_numeric"]) * args.steps,
+           "clocks": clocks}
 
     # ---- end to end through the host-buffer entry point (H2D of the operands, D2H of C inside the timed region)
-    if not args.no_e2e:
+    if e2e:
         try:
             keep = []
 
@@ -396,22 +398,99 @@ def main():
             if world > 1:
                 dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
             out_bytes = out_fixed + nnzC * (4 + V)
-            line["e2e"] = {"value": 2.0 * all_products / (float(e2e_ms[0]) * 1e-3) / 1e9, "unit": UNIT,
-                           "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
-                           "ms_per_step": float(e2e_ms[0]), "steps": n_e2e,
-                           "call": "spws_execute_host, pinned host buffers"}
+            out["e2e"] = {"value": 2.0 * all_products / (float(e2e_ms[0]) * 1e-3) / 1e9, "unit": UNIT,
+                          "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
+                          "ms_per_step": float(e2e_ms[0]), "steps": n_e2e,
+                          "call": "spws_execute_host, pinned host buffers"}
+            del arena
         except Exception as exc:  # report, do not hide
-            line["e2e"] = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
+            out["e2e"] = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
 
-    # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1); the same
+    # sampled rows of the device result are compared with it entry by entry
+    if cpu_baseline and rank == 0 and world == 1:
         import oracle
         oracle.build()
         threads = oracle.hardware_threads()
-        rows, psample, total = sized_oracle_sample(A, B, threads, 12.0)
-        dt, _ = time_oracle(A, B, rows, threads)
-        line["cpu_baseline"] = {"value": 2.0 * psample / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                "sample": f"{rows.size} random rows of {A.nrows}, {psample} of {total} products, {dt:.1f} s"}
+        rows, psample, total = sized_oracle_sample(A, B, threads, args.cpu_seconds)
+        t0 = time.perf_counter()
+        ref = oracle.spgemm(A, B, rows=rows, threads=threads)
+        dt = time.perf_counter() - t0
+        rows1, psample1, _ = oracle_sample(A, B, max(2e6, psample / max(dt, 1e-6) / max(threads, 1) * 3.0), seed=1)
+        dt1, _ = time_oracle(A, B, rows1, 1)
+        out["cpu_baseline"] = {"value": 2.0 * psample / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                               "sample": f"{rows.size} random rows of {A.nrows}, {psample} of {total} products, {dt:.1f} s",
+                               "single_thread": {"value": 2.0 * psample1 / dt1 / 1e9, "unit": UNIT, "cores": 1,
+                                                 "sample": f"{rows1.size} random rows, {psample1} products, {dt1:.1f} s"}}
+        # parity of the timed result on the sampled rows (structure exact; values under the two-clause rule)
+        C = result["C"]
+        pos = (C.pos2 if is_ttm else C.pos).cpu().numpy()
+        dcrd, dval = (C.crd2, C.val) if is_ttm else (C.crd, C.val)
+        tol = 1e-12 if V == 8 else 1e-5
+        entries = second = bad = 0
+        for tix, r in enumerate(rows):
+            s0, s1 = int(pos[r]), int(pos[r + 1])
+            u = slice(int(ref.pos[tix]), int(ref.pos[tix + 1]))
+            got_c = dcrd[s0:s1].cpu().numpy()
+            if got_c.shape[0] != u.stop - u.start or not np.array_equal(got_c, ref.crd[u]):
+                bad += 1
+                continue
+            err = np.abs(dval[s0:s1].cpu().numpy().astype(np.float64) - ref.val_ref[u])
+            first = err <= tol * np.abs(ref.val_ref[u])
+            sec = err <= tol * ref.abs[u]
+            bad += int((~(first | sec)).sum())
+            second += int((~first & sec).sum())
+            entries += u.stop - u.start
+        out["parity_sample"] = {"rows": int(rows.size), "entries": int(entries), "mismatches": int(bad),
+                                "second_clause_entries": int(second), "tolerance": tol}
+    plan.close()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="rmat18",
+                    help="rmat18 (default), stencil64, uniform8, wide26, ttm4096, or rmatNN / stencilNN at another size")
+    ap.add_argument("--policy", default="auto")
+    ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--opt", action="append", default=[], help="plan option as name=value (repeatable)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-targets", action="store_true", help="skip the second target configuration (stencil64)")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time of the oracle sample")
+    args = ap.parse_args()
+    WORKLOAD_TEXT.setdefault(args.workload, f"{args.workload} (same recipe as the named configuration, other size), fp64")
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    m = measure(args.workload, args, dev, rank, world, dist, e2e=not args.no_e2e, cpu_baseline=not args.no_cpu_baseline)
+    line = {"metric": METRIC, "value": m.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": m.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": m.pop("dtype"), "data": "synthetic", "config": m.pop("config")}
+    line.update(m)
+    # the other configuration with a roofline target, same protocol (default run only)
+    if args.workload == "rmat18" and not args.no_targets and not args.opt and args.policy == "auto":
+        torch.cuda.empty_cache()
+        t = measure("stencil64", args, dev, rank, world, dist, e2e=False, cpu_baseline=False)
+        line["targets"] = {"stencil64": {"metric": METRIC, "unit": UNIT, **t}}
 
     if rank == 0:
         print(json.dumps(line), flush=True)

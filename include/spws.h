@@ -146,7 +146,9 @@ enum {
                                  that several work units add into                                  */
     SPWS_T_NUM_DENSE_CTA = 14,
     SPWS_T_NUM_ISM_GLOBAL = 15,
-    SPWS_T_COUNT = 16
+    SPWS_T_CEIL_DENSE_WARP = 16, /* spws_gather_ceiling: the warp-per-row dense rows ...             */
+    SPWS_T_CEIL_DENSE_CTA = 17,  /* ... and the CTA-unit dense rows                                   */
+    SPWS_T_COUNT = 18
 };
 
 spws_status_t spws_create(spws_handle_t* handle);
@@ -203,6 +205,20 @@ spws_status_t spws_get_stats(spws_plan_t plan, spws_stats_t* stats);
  * did not run).  `n` is the capacity of `ms` and must be at least SPWS_T_COUNT. */
 spws_status_t spws_set_profiling(spws_plan_t plan, int enabled);
 spws_status_t spws_get_timings(spws_plan_t plan, float* ms, int n);
+
+/* Iteration-only lower bound of the dense-workspace numeric kernels (Sec. 7.2 measures, as a
+ * lower bound for any workspace, the generated code with the workspace stripped and only the
+ * sparse iteration kept).  Runs, on the rows the last spws_symbolic routed to the dense workspace,
+ * the same traversal as spws_numeric's two dense kernels -- same work units, same launch shape,
+ * same gathers of A's entries and of the B rows they pick -- without bitmap, rank or
+ * accumulation: every gathered column index is added into *index_sum and every product a*b into
+ * *value_sum (both DEVICE pointers, cleared by the call; the value sum is taken in an order that
+ * varies from run to run).  C is not written.  Call after spws_symbolic, with the same operands
+ * and scratch; asynchronous.  With profiling on, spws_get_timings reports the two kernels in
+ * SPWS_T_CEIL_DENSE_WARP / SPWS_T_CEIL_DENSE_CTA. */
+spws_status_t spws_gather_ceiling(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                                  const spws_tensor_t* C, void* scratch, size_t scratch_bytes,
+                                  uint64_t* index_sum, double* value_sum);
 
 /* Whole path with HOST tensors: copies A and B to the device, runs both passes, copies C back.
  * A, B, C hold host pointers; C's arrays must be allocated with capacities n[] (crd/val of the

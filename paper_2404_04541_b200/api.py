@@ -109,6 +109,15 @@ class Context:
         plan.numeric(a, b, c, self._aligned_ptr(sc), nbytes)
         return DeviceCSR(int(c.dims[0]), int(c.dims[1]), c.pos[1], c.crd[1][:nnz], c.val[:nnz])
 
+    def gather_ceiling(self, plan: B_.Plan, c: B_.TensorArrays, state):
+        """Runs the gather-only form of the dense numeric kernels after a symbolic pass; returns
+        (sum of gathered column indices, sum of products) as Python numbers."""
+        a, b, sc, nbytes = state[:4]
+        sums = torch.zeros(2, dtype=torch.int64, device=self.device)
+        plan.gather_ceiling(a, b, c, self._aligned_ptr(sc), nbytes, sums.data_ptr(), sums.data_ptr() + 8)
+        torch.cuda.synchronize(self.device)
+        return int(sums[0].item()), float(sums[1:].view(torch.float64).item())
+
     def spgemm(self, A: DeviceCSR, B: DeviceCSR, policy="auto", plan: B_.Plan | None = None, **options):
         """C = A*B in CSR; returns (C, stats)."""
         own = plan is None

@@ -33,12 +33,12 @@ POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPAR
 
 EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create", "spws_plan_destroy",
            "spws_check_expression", "spws_workspace_size", "spws_symbolic", "spws_numeric",
-           "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host",
+           "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host", "spws_gather_ceiling",
            "spws_row_pointer_static", "spws_status_string")
 STATIC_MAX_ROWS = 16777216
 TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense_warp",
                  "sym_dense_cta", "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem",
-                 "num_dense_warp", "num_dense_emit", "num_dense_cta", "num_ism_global")
+                 "num_dense_warp", "num_dense_emit", "num_dense_cta", "num_ism_global", "ceil_dense_warp", "ceil_dense_cta")
 # class index of each per-class kernel group (rows_per_class / products_per_class / nnz_per_class)
 CLASS_NAMES = ("empty", "ism_reg", "ism_smem_s", "ism_smem", "dense_warp", "dense_hub", "dense_cta", "ism_global")
 
@@ -94,6 +94,7 @@ def lib():
         L.spws_workspace_size.argtypes = [vp, T, T, ctypes.POINTER(sz)]
         L.spws_symbolic.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(ctypes.c_int64)]
         L.spws_numeric.argtypes = [vp, T, T, T, vp, sz]
+        L.spws_gather_ceiling.argtypes = [vp, T, T, T, vp, sz, vp, vp]
         L.spws_get_stats.argtypes = [vp, ctypes.POINTER(spws_stats_t)]
         L.spws_set_profiling.argtypes = [vp, i32]
         L.spws_get_timings.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32]
@@ -234,6 +235,14 @@ class Plan:
         a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
         _check(lib().spws_numeric(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
                                   ctypes.c_void_p(scratch_ptr), scratch_bytes), "spws_numeric")
+
+    def gather_ceiling(self, A, B, C, scratch_ptr: int, scratch_bytes: int, index_sum_ptr: int, value_sum_ptr: int):
+        """spws_gather_ceiling: the dense numeric kernels' traversal with the workspace stripped;
+        the two device words receive the sum of the gathered column indices and of the products."""
+        a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
+        _check(lib().spws_gather_ceiling(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                         ctypes.c_void_p(scratch_ptr), scratch_bytes, ctypes.c_void_p(index_sum_ptr),
+                                         ctypes.c_void_p(value_sum_ptr)), "spws_gather_ceiling")
 
     def get_stats(self) -> dict:
         s = spws_stats_t()

@@ -23,6 +23,7 @@ enum RowClass : int {
     CLS_ISM_GLOBAL = 9  // accumulation array in shared memory, all array in global memory
 };
 constexpr int NUM_SLOT = 16;   // work_counter[cls] in the symbolic pass, work_counter[NUM_SLOT + cls] in the numeric pass
+constexpr int CEIL_SLOT = 20;  // work_counter[CEIL_SLOT + cls] in the gather-only (iteration-only) kernels
 constexpr int EMIT_SLOT = 30;  // work_counter slot of the coordinate emission of the CTA dense route
 constexpr int BW_SLOT = 31;    // work_counter slot of the word-list build
 // index of a class in the public statistics (the three register classes are reported as one)
@@ -208,11 +209,13 @@ cudaError_t launch_ism_smem(const LaunchCtx& c, bool numeric, int cls, int n_hos
                             const i64* rowptr, int* Ccrd, void* Cval);
 cudaError_t launch_dense_sym_warp(const LaunchCtx& c, const Csr& A, const Csr& B);
 cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B);
+// chk_idx / chk_val non-null: the gather-only form of the same kernel (workspace stripped, checksums out)
 cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, int max_cnt, const Csr& A, const Csr& B,
-                                  const i64* rowptr, int* Ccrd, void* Cval);
+                                  const i64* rowptr, int* Ccrd, void* Cval, u64* chk_idx = nullptr, double* chk_val = nullptr);
 // phase 0: write the coordinates and clear the value segments several units add into; 1: accumulate
 cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host, int max_span_words, i64 total_products,
-                                 const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval);
+                                 const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval,
+                                 u64* chk_idx = nullptr, double* chk_val = nullptr);
 cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
                               const i64* rowptr, int* Ccrd, void* Cval);
 

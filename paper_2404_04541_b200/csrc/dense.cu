@@ -271,10 +271,13 @@ __global__ void __launch_bounds__(DC_THREADS) dense_sym_cta_kernel(DevCtl* __res
 // ---------------------------------------------------------------------------------------
 // numeric, warp per row
 // ---------------------------------------------------------------------------------------
-template <typename T>
+// CEIL = true: the same walk over rows, entries and B rows with the workspace stripped (Sec. 7.2,
+// iteration-only lower bound); the gathered indices and products go into two checksums.
+template <typename T, bool CEIL>
 __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __restrict__ ctl, int bmw, int accw, Csr A, Csr B, RowTables tab,
                                                                     const i64* __restrict__ rowptr, int* __restrict__ Ccrd,
-                                                                    T* __restrict__ Cval) {
+                                                                    T* __restrict__ Cval, u64* __restrict__ chk_idx,
+                                                                    double* __restrict__ chk_val) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (ctl->status != 0) return;
     const int n = ctl->n_warp_rows;
@@ -285,11 +288,14 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
     T* acc = reinterpret_cast<T*>(reinterpret_cast<uint2*>(smem_raw) + DW_WARPS * bmw) + warp * accw;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
-    for (int w = lane; w < bmw; w += 32) tbl[w] = make_uint2(0u, 0u);       // every row leaves its table clear
+    if (!CEIL)
+        for (int w = lane; w < bmw; w += 32) tbl[w] = make_uint2(0u, 0u);   // every row leaves its table clear
     __syncwarp();
+    u64 my_idx = 0;
+    double my_val = 0.0;
     for (;;) {
         int r = 0;
-        if (lane == 0) r = atomicAdd(&ctl->work_counter[NUM_SLOT + CLS_DENSE_WARP], 1);
+        if (lane == 0) r = atomicAdd(&ctl->work_counter[(CEIL ? CEIL_SLOT : NUM_SLOT) + CLS_DENSE_WARP], 1);
         r = __shfl_sync(0xffffffffu, r, 0);
         if (r >= n) break;
         const int row = tab.warp_rows[r];
@@ -304,7 +310,9 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         const int nzw = (int)((slot & ~BM_COMPACT) >> BM_NZW_SHIFT);
         const unsigned* src = tab.bm_arena + (slot & BM_OFF_MASK);
         const uint2* src2 = reinterpret_cast<const uint2*>(src);
-        if (compact) {
+        if (CEIL) {
+            // no workspace to set up
+        } else if (compact) {
             // the saved non-empty words in column order: ranks by a running prefix of their bit counts
             int carry = 0;
             for (int i0 = 0; i0 < nzw; i0 += 32) {
@@ -325,8 +333,23 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                 if (w < nw) tbl[w] = make_uint2(word, src[nw + (w0 >> 5)] + (unsigned)(incl - c));
             }
         }
-        for (int x = lane; x < cnt; x += 32) acc[x] = 0;
+        if (!CEIL)
+            for (int x = lane; x < cnt; x += 32) acc[x] = 0;
         __syncwarp();
+        // one product into the workspace: rank of its column, then add (plain when no other lane can
+        // hold the same column, atomic otherwise); stripped to the checksums when CEIL
+        auto put = [&](unsigned rel, T prod, bool shared_slot) {
+            if (CEIL) {
+                if (rel != 0xffffffffu) { my_idx += (u64)(rel + (unsigned)base); my_val += (double)prod; }
+            } else if (rel < span) {
+                const uint2 t = tbl[rel >> 5];
+                const int slot_ = (int)t.y + __popc(t.x & ((1u << (rel & 31)) - 1u));
+                if (slot_ < accw) {
+                    if (shared_slot) atomicAdd(&acc[slot_], prod);
+                    else acc[slot_] = add_rn(acc[slot_], prod);
+                }
+            }
+        };
         const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
         if (gs == 32) {
             // one A entry at a time, lanes across its B row: distinct columns, no atomics,
@@ -356,34 +379,14 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                     if (lane < len0) { rel0 = (unsigned)(__ldg(B.crd + qs0 + lane) - base); v0 = __ldg(Bval + qs0 + lane); }
                     if (lane < len1) { rel1 = (unsigned)(__ldg(B.crd + qs1 + lane) - base); v1 = __ldg(Bval + qs1 + lane); }
                     // entry e
-                    if (rel0 < span) {
-                        const uint2 t = tbl[rel0 >> 5];
-                        const int slot_ = (int)t.y + __popc(t.x & ((1u << (rel0 & 31)) - 1u));
-                        if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a0, v0));
-                    }
-                    for (int t = lane + 32; t < len0; t += 32) {
-                        const unsigned rel = (unsigned)(__ldg(B.crd + qs0 + t) - base);
-                        if (rel < span) {
-                            const uint2 tw = tbl[rel >> 5];
-                            const int slot_ = (int)tw.y + __popc(tw.x & ((1u << (rel & 31)) - 1u));
-                            if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a0, __ldg(Bval + qs0 + t)));
-                        }
-                    }
+                    put(rel0, mul_rn(a0, v0), false);
+                    for (int t = lane + 32; t < len0; t += 32)
+                        put((unsigned)(__ldg(B.crd + qs0 + t) - base), mul_rn(a0, __ldg(Bval + qs0 + t)), false);
                     __syncwarp();
                     // entry e + 1
-                    if (rel1 < span) {
-                        const uint2 t = tbl[rel1 >> 5];
-                        const int slot_ = (int)t.y + __popc(t.x & ((1u << (rel1 & 31)) - 1u));
-                        if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a1, v1));
-                    }
-                    for (int t = lane + 32; t < len1; t += 32) {
-                        const unsigned rel = (unsigned)(__ldg(B.crd + qs1 + t) - base);
-                        if (rel < span) {
-                            const uint2 tw = tbl[rel >> 5];
-                            const int slot_ = (int)tw.y + __popc(tw.x & ((1u << (rel & 31)) - 1u));
-                            if (slot_ < accw) acc[slot_] = add_rn(acc[slot_], mul_rn(a1, __ldg(Bval + qs1 + t)));
-                        }
-                    }
+                    put(rel1, mul_rn(a1, v1), false);
+                    for (int t = lane + 32; t < len1; t += 32)
+                        put((unsigned)(__ldg(B.crd + qs1 + t) - base), mul_rn(a1, __ldg(Bval + qs1 + t)), false);
                     __syncwarp();
                 }
             }
@@ -396,17 +399,12 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
                 const i64 qs = __ldg(B.pos + k);
                 const int len = (int)(__ldg(B.pos + k + 1) - qs);
                 const T a = __ldg(Aval + p);
-                for (int t = gl; t < len; t += gs) {
-                    const unsigned rel = (unsigned)(__ldg(B.crd + qs + t) - base);
-                    if (rel < span) {
-                        const uint2 tw = tbl[rel >> 5];
-                        const int slot_ = (int)tw.y + __popc(tw.x & ((1u << (rel & 31)) - 1u));
-                        if (slot_ < accw) atomicAdd(&acc[slot_], mul_rn(a, __ldg(Bval + qs + t)));
-                    }
-                }
+                for (int t = gl; t < len; t += gs)
+                    put((unsigned)(__ldg(B.crd + qs + t) - base), mul_rn(a, __ldg(Bval + qs + t)), true);
             }
             __syncwarp();
         }
+        if (CEIL) continue;
         // copy out: values are already in output order; set bits give the coordinates; the table
         // words the row used are cleared on the way
         for (int x = lane; x < cnt; x += 32) Cval[out0 + x] = acc[x];
@@ -438,6 +436,13 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
         }
         __syncwarp();
     }
+    if (CEIL) {
+        for (int d = 16; d > 0; d >>= 1) {
+            my_idx += __shfl_xor_sync(0xffffffffu, my_idx, d);
+            my_val += __shfl_xor_sync(0xffffffffu, my_val, d);
+        }
+        if (lane == 0) { atomicAdd(chk_idx, my_idx); atomicAdd(chk_val, my_val); }
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -449,10 +454,14 @@ __global__ void __launch_bounds__(DW_THREADS) dense_num_warp_kernel(DevCtl* __re
 constexpr int DN_ENTRIES = 768;      // A entries whose descriptors are staged per round
 constexpr int DN_TILE = 256;         // products a warp takes per fetch
 
-template <typename T>
+// CEIL = true is the same traversal with the workspace stripped (the iteration-only lower bound of
+// Sec. 7.2): units, descriptor rounds, product tiles and gathers as below, but no bitmap, no rank
+// and no accumulation; every gathered column index and product is folded into two checksums.
+template <typename T, bool CEIL>
 __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __restrict__ ctl, int smem_words, int CAP, i64 unit_products,
                                                                    Csr A, Csr B, RowTables tab, const i64* __restrict__ rowptr,
-                                                                   int* __restrict__ Ccrd, T* __restrict__ Cval) {
+                                                                   int* __restrict__ Ccrd, T* __restrict__ Cval,
+                                                                   u64* __restrict__ chk_idx, double* __restrict__ chk_val) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* acc = reinterpret_cast<T*>(smem_raw);                                        // CAP
     // per bitmap word: .x = the word, .y = outputs of the row before it (one load gives a rank)
@@ -468,11 +477,14 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const T* __restrict__ Aval = (const T*)A.val;
     const T* __restrict__ Bval = (const T*)B.val;
-    for (int x = tid; x < CAP; x += DN_THREADS) acc[x] = 0;
+    if (!CEIL)
+        for (int x = tid; x < CAP; x += DN_THREADS) acc[x] = 0;
+    u64 my_idx = 0;
+    double my_val = 0.0;
 
     for (;;) {
         __syncthreads();
-        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[NUM_SLOT + CLS_DENSE_CTA], 1);
+        if (tid == 0) s_next = atomicAdd(&ctl->work_counter[(CEIL ? CEIL_SLOT : NUM_SLOT) + CLS_DENSE_CTA], 1);
         __syncthreads();
         const int u = s_next;
         if (u >= n_units) break;
@@ -488,13 +500,13 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const i64 e_lo = ps + (pe - ps) * uidx / nun, e_hi = ps + (pe - ps) * (uidx + 1) / nun;
         T* const gacc = Cval + out0;
-        if (nun == 1)                                   // outputs beyond the shared-memory part start at zero
+        if (!CEIL && nun == 1)                          // outputs beyond the shared-memory part start at zero
             for (int x = CAP + tid; x < cnt; x += DN_THREADS) gacc[x] = 0;
 
         // the row's bitmap with the rank of every word's first bit (the symbolic pass saved the
         // rank at every chunk start).  A warp takes eight chunks at a time, all loads first.
         const unsigned* src = tab.bm_arena + tab.bm_off[row];
-        for (int c0 = warp; c0 < nch; c0 += DN_WARPS * 8) {
+        for (int c0 = warp; !CEIL && c0 < nch; c0 += DN_WARPS * 8) {
             unsigned word[8], rank_c[8];
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
@@ -513,7 +525,9 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
         __syncthreads();
 
 #define SPWS_DENSE_ADD(REL, VAL)                                                                          \
-        if ((REL) < span_bits) {                                                                          \
+        if (CEIL) {                                                                                       \
+            if ((REL) != 0xffffffffu) { my_idx += (u64)((REL) + (unsigned)base); my_val += (double)(VAL); } \
+        } else if ((REL) < span_bits) {                                                                   \
             const uint2 br_ = bmr[(REL) >> 5];                                                            \
             const int r_ = (int)br_.y + __popc(br_.x & ((1u << ((REL) & 31)) - 1u));                      \
             if (r_ < CAP) atomicAdd(&acc[r_], (VAL));                                                     \
@@ -645,7 +659,7 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
 
         // copy out the shared-memory part of the values (the coordinates are written by
         // dense_emit_crd_kernel)
-        const int n_smem = min(cnt, CAP);
+        const int n_smem = CEIL ? 0 : min(cnt, CAP);
         if (nun == 1) {
             for (int x = tid; x < n_smem; x += DN_THREADS) { gacc[x] = acc[x]; acc[x] = 0; }
         } else {
@@ -655,6 +669,13 @@ __global__ void __launch_bounds__(DN_THREADS, 2) dense_num_cta_kernel(DevCtl* __
                 if (v != (T)0) atomicAdd(gacc + x, v);
             }
         }
+    }
+    if (CEIL) {
+        for (int d = 16; d > 0; d >>= 1) {
+            my_idx += __shfl_xor_sync(0xffffffffu, my_idx, d);
+            my_val += __shfl_xor_sync(0xffffffffu, my_val, d);
+        }
+        if (lane == 0) { atomicAdd(chk_idx, my_idx); atomicAdd(chk_val, my_val); }
     }
 }
 
@@ -723,7 +744,6 @@ __global__ void __launch_bounds__(DE_THREADS) dense_emit_crd_kernel(DevCtl* __re
             if (n > 0) {
                 const int p = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
                 const int e = warp_incl_scan(p) - p;
-                const int col = base + (((g << 7) + (lane << 2)) << 5);
                 const i64 o = out0 + r0;
                 const unsigned m0 = __ballot_sync(0xffffffffu, w.x != 0u), m1 = __ballot_sync(0xffffffffu, w.y != 0u);
                 const unsigned m2 = __ballot_sync(0xffffffffu, w.z != 0u), m3 = __ballot_sync(0xffffffffu, w.w != 0u);
@@ -800,41 +820,45 @@ cudaError_t launch_dense_sym_cta(const LaunchCtx& c, const Csr& A, const Csr& B)
     return cudaGetLastError();
 }
 
-template <typename T>
+template <typename T, bool CEIL>
 static cudaError_t num_warp_t(const LaunchCtx& c, int n_host, int bmw, int accw, const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd,
-                              void* Cval) {
+                              void* Cval, u64* chk_idx, double* chk_val) {
     int per_sm = 0;
     const size_t smem = (size_t)DW_WARPS * (sizeof(T) * (size_t)accw + 8 * (size_t)bmw);
     cudaError_t e;
-    if ((e = cudaFuncSetAttribute(dense_num_warp_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_num_warp_kernel<T>, DW_THREADS, smem)) != cudaSuccess) return e;
+    auto k = dense_num_warp_kernel<T, CEIL>;
+    if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DW_THREADS, smem)) != cudaSuccess) return e;
     const i64 work = n_host >= 0 ? ((i64)n_host + DW_WARPS - 1) / DW_WARPS : -1;
-    dense_num_warp_kernel<T><<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, bmw, accw, A, B, c.tab, rowptr, Ccrd, (T*)Cval);
+    k<<<persistent_grid(c, per_sm, work), DW_THREADS, smem, c.stream>>>(c.ctl, bmw, accw, A, B, c.tab, rowptr, Ccrd, (T*)Cval, chk_idx, chk_val);
     ++c.launches;
     return cudaGetLastError();
 }
 
 cudaError_t launch_dense_num_warp(const LaunchCtx& c, int n_host, int max_span_words, int max_cnt, const Csr& A, const Csr& B,
-                                  const i64* rowptr, int* Ccrd, void* Cval) {
+                                  const i64* rowptr, int* Ccrd, void* Cval, u64* chk_idx, double* chk_val) {
     // bitmap words reserved per warp: the widest dense row of this pass, at most the class limit
     int bmw = max_span_words > 0 ? ((max_span_words + 31) & ~31) : DENSE_WARP_BM_WORDS;
     if (bmw > DENSE_WARP_BM_WORDS) bmw = DENSE_WARP_BM_WORDS;
     int accw = max_cnt > 0 ? ((max_cnt + 31) & ~31) : DENSE_WARP_ACC;     // values reserved per warp
     if (accw > DENSE_WARP_ACC) accw = DENSE_WARP_ACC;
-    return c.is_f64 ? num_warp_t<double>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval)
-                    : num_warp_t<float>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval);
+    if (chk_idx)      // same launch shape (shared memory reserved, hence occupancy) as the full kernel
+        return c.is_f64 ? num_warp_t<double, true>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval, chk_idx, chk_val)
+                        : num_warp_t<float, true>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval, chk_idx, chk_val);
+    return c.is_f64 ? num_warp_t<double, false>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval, nullptr, nullptr)
+                    : num_warp_t<float, false>(c, n_host, bmw, accw, A, B, rowptr, Ccrd, Cval, nullptr, nullptr);
 }
 
-template <typename T>
+template <typename T, bool CEIL>
 static cudaError_t num_cta_t(const LaunchCtx& c, int phase, int n_units_host, int words, i64 total_products, const Csr& A,
-                             const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
+                             const Csr& B, const i64* rowptr, int* Ccrd, void* Cval, u64* chk_idx, double* chk_val) {
     const int CAP = c.prm.unit_outputs;
     const i64 unit_products = dense_unit_products(total_products);
     const size_t smem = ((sizeof(T) * (size_t)CAP + (size_t)words * 8 + 15) & ~(size_t)15) +
                         (size_t)DN_ENTRIES * (8 + sizeof(T)) + (size_t)(DN_ENTRIES + 1) * 4 + 16;
     cudaError_t e;
     int per_sm = 0;
-    auto k = dense_num_cta_kernel<T>;
+    auto k = dense_num_cta_kernel<T, CEIL>;
     if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, DN_THREADS, smem)) != cudaSuccess) return e;
     if (phase == 0) {
@@ -845,18 +869,21 @@ static cudaError_t num_cta_t(const LaunchCtx& c, int phase, int n_units_host, in
         dense_emit_crd_kernel<T><<<persistent_grid(c, emit_per_sm, work), DE_THREADS, 0, c.stream>>>(c.ctl, unit_products, c.tab, rowptr, Ccrd, (T*)Cval);
     } else {
         k<<<persistent_grid(c, per_sm, n_units_host), DN_THREADS, smem, c.stream>>>(c.ctl, words, CAP, unit_products, A, B, c.tab,
-                                                                                 rowptr, Ccrd, (T*)Cval);
+                                                                                 rowptr, Ccrd, (T*)Cval, chk_idx, chk_val);
     }
     ++c.launches;
     return cudaGetLastError();
 }
 
 cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host, int max_span_words, i64 total_products,
-                                 const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval) {
+                                 const Csr& A, const Csr& B, const i64* rowptr, int* Ccrd, void* Cval, u64* chk_idx, double* chk_val) {
     int words = max_span_words > 0 ? max_span_words : c.dense_smem_words;
     words = (words + 31) & ~31;
-    return c.is_f64 ? num_cta_t<double>(c, phase, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval)
-                    : num_cta_t<float>(c, phase, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval);
+    if (chk_idx)      // same launch shape as the full kernel
+        return c.is_f64 ? num_cta_t<double, true>(c, 1, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval, chk_idx, chk_val)
+                        : num_cta_t<float, true>(c, 1, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval, chk_idx, chk_val);
+    return c.is_f64 ? num_cta_t<double, false>(c, phase, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval, nullptr, nullptr)
+                    : num_cta_t<float, false>(c, phase, n_units_host, words, total_products, A, B, rowptr, Ccrd, Cval, nullptr, nullptr);
 }
 
 }  // namespace spws

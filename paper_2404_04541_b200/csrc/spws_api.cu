@@ -36,9 +36,9 @@ struct spws_plan_s {
     // optional per-kernel timing: ev[g] is recorded after group g; ev_start[] before each pass
     bool profiling = false;
     cudaEvent_t ev[SPWS_T_COUNT] = {};
-    cudaEvent_t ev_start[2] = {};
+    cudaEvent_t ev_start[3] = {};
     bool ev_ran[SPWS_T_COUNT] = {};
-    bool ev_pass[2] = {};
+    bool ev_pass[3] = {};
 };
 
 namespace {
@@ -288,9 +288,12 @@ inline void mark(spws_plan_s* p, int group) {
     cudaEventRecord(p->ev[group], p->h->stream);
     p->ev_ran[group] = true;
 }
+// timing groups of pass 0 (symbolic), 1 (numeric), 2 (gather-only ceiling)
+const int PASS_GROUPS[4] = {0, SPWS_T_NUM_ISM_REG, SPWS_T_CEIL_DENSE_WARP, SPWS_T_COUNT};
+
 inline void mark_start(spws_plan_s* p, int pass) {
     if (!p->profiling) return;
-    const int g0 = pass == 0 ? 0 : SPWS_T_NUM_ISM_REG, g1 = pass == 0 ? SPWS_T_NUM_ISM_REG : SPWS_T_COUNT;
+    const int g0 = PASS_GROUPS[pass], g1 = PASS_GROUPS[pass + 1];
     for (int g = g0; g < g1; ++g) p->ev_ran[g] = false;
     cudaEventRecord(p->ev_start[pass], p->h->stream);
     p->ev_pass[pass] = true;
@@ -383,7 +386,7 @@ spws_status_t spws_set_profiling(spws_plan_t plan, int enabled) {
     if (!plan) return SPWS_INVALID_ARGUMENT;
     if (enabled && !plan->ev[0]) {
         for (int g = 0; g < SPWS_T_COUNT; ++g) CUDA_TRY(cudaEventCreate(&plan->ev[g]));
-        for (int g = 0; g < 2; ++g) CUDA_TRY(cudaEventCreate(&plan->ev_start[g]));
+        for (int g = 0; g < 3; ++g) CUDA_TRY(cudaEventCreate(&plan->ev_start[g]));
     }
     plan->profiling = enabled != 0;
     return SPWS_OK;
@@ -394,10 +397,10 @@ spws_status_t spws_get_timings(spws_plan_t plan, float* ms, int n) {
     for (int g = 0; g < SPWS_T_COUNT; ++g) ms[g] = 0.0f;
     if (!plan->ev[0]) return SPWS_BAD_SEQUENCE;
     CUDA_TRY(cudaStreamSynchronize(plan->h->stream));
-    for (int pass = 0; pass < 2; ++pass) {
+    for (int pass = 0; pass < 3; ++pass) {
         if (!plan->ev_pass[pass]) continue;
         cudaEvent_t prev = plan->ev_start[pass];
-        const int g0 = pass == 0 ? 0 : SPWS_T_NUM_ISM_REG, g1 = pass == 0 ? SPWS_T_NUM_ISM_REG : SPWS_T_COUNT;
+        const int g0 = PASS_GROUPS[pass], g1 = PASS_GROUPS[pass + 1];
         for (int g = g0; g < g1; ++g) {
             if (!plan->ev_ran[g]) continue;
             CUDA_TRY(cudaEventElapsedTime(&ms[g], prev, plan->ev[g]));
@@ -411,7 +414,7 @@ spws_status_t spws_plan_destroy(spws_plan_t plan) {
     if (!plan) return SPWS_INVALID_ARGUMENT;
     if (plan->ev[0]) {
         for (int g = 0; g < SPWS_T_COUNT; ++g) cudaEventDestroy(plan->ev[g]);
-        for (int g = 0; g < 2; ++g) cudaEventDestroy(plan->ev_start[g]);
+        for (int g = 0; g < 3; ++g) cudaEventDestroy(plan->ev_start[g]);
     }
     if (plan->host_ctl) cudaFreeHost(plan->host_ctl);
     delete plan;
@@ -582,6 +585,37 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         mark(plan, SPWS_T_NUM_ISM_GLOBAL);
     }
     plan->stats.launches_numeric = c.launches;
+    return SPWS_OK;
+}
+
+spws_status_t spws_gather_ceiling(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* C,
+                                  void* scratch, size_t scratch_bytes, uint64_t* index_sum, double* value_sum) {
+    if (!plan || !index_sum || !value_sum) return SPWS_INVALID_ARGUMENT;
+    if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
+    Shapes S{};
+    spws_status_t st = check_operands(plan, A, B, S);
+    if (st != SPWS_OK) return st;
+    if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
+    if (scratch != plan->scratch || S.m != plan->m) return SPWS_BAD_SEQUENCE;
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
+    const i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<const i64*>(sc + L.rowptr_raw);
+    CUDA_TRY(cudaMemsetAsync(c.ctl->work_counter + CEIL_SLOT, 0, sizeof(int) * NCLASS, c.stream));
+    CUDA_TRY(cudaMemsetAsync(index_sum, 0, sizeof(uint64_t), c.stream));
+    CUDA_TRY(cudaMemsetAsync(value_sum, 0, sizeof(double), c.stream));
+    mark_start(plan, 2);
+    const spws_stats_t& s = plan->stats;
+    u64* ci = reinterpret_cast<u64*>(index_sum);
+    if (s.dense_warp_rows > 0) {
+        CUDA_TRY(launch_dense_num_warp(c, (int)s.dense_warp_rows, plan->max_span_words, plan->max_warp_cnt, S.A, S.B, rowptr, nullptr, nullptr, ci, value_sum));
+        mark(plan, SPWS_T_CEIL_DENSE_WARP);
+    }
+    if (s.dense_units > 0) {
+        CUDA_TRY(launch_dense_num_cta(c, 1, (int)s.dense_units, plan->max_span_words, s.products, S.A, S.B, rowptr, nullptr, nullptr, ci, value_sum));
+        mark(plan, SPWS_T_CEIL_DENSE_CTA);
+    }
     return SPWS_OK;
 }
 

@@ -449,6 +449,38 @@ def test_full_rmat18_every_entry_streamed(ctx, oracle_mod):
     print(f"rmat18: {entries} entries compared, {second} needed the sum|a*b| clause")
 
 
+# ------------------------------------------------------------------ gather-only lower bound
+@pytest.mark.parametrize("name", ["rmat", "stencil", "heavy"])
+def test_gather_ceiling_visits_every_product_once(ctx, name):
+    """The iteration-only form of the dense numeric kernels must walk exactly the products of the
+    rows routed to the dense workspace: with the dense policy forced that is every product, so the
+    sum of the gathered column indices (exact) and of the products a*b (to rounding) have closed
+    forms in the operands."""
+    from paper_2404_04541_b200 import api, binding
+    if name == "rmat":
+        A = B = rmat_csr(12, 16, 3)
+    elif name == "stencil":
+        A = B = stencil27_csr(12, 4)
+    else:
+        B = uniform_rows_csr(4000, 30000, 200, 6)
+        A = random_csr(40, 4000, 0.3, 5)
+    dA = api.DeviceCSR.from_host(A)
+    dB = dA if B is A else api.DeviceCSR.from_host(B)
+    plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, np.float64, "dense")
+    c, state = ctx.spgemm_symbolic(plan, dA, dB)
+    for _ in range(2):                                               # repeatable: the call clears its own counters
+        idx_sum, val_sum = ctx.gather_ceiling(plan, c, state)
+        col_sum = np.bincount(rows_of(B.pos), weights=B.crd.astype(np.float64), minlength=B.nrows).astype(np.int64)
+        assert idx_sum == int(col_sum[A.crd].sum())
+        b1 = np.bincount(rows_of(B.pos), weights=B.val, minlength=B.nrows)
+        babs = np.bincount(rows_of(B.pos), weights=np.abs(B.val), minlength=B.nrows)
+        want, scale = float((A.val * b1[A.crd]).sum()), float((np.abs(A.val) * babs[A.crd]).sum())
+        assert abs(val_sum - want) <= 1e-12 * scale
+    stats = plan.get_stats()
+    assert stats["dense_units"] + stats["dense_warp_rows"] > 0
+    plan.close()
+
+
 # ------------------------------------------------------------------ row-sharded driver on the device
 def _sharded_worker(rank, world, port, out_dir):
     import os
