@@ -447,13 +447,80 @@ def measure(workload, args, dev, rank, world, dist, e2e=True, cpu_baseline=True)
     return out
 
 
+SWEEPS = {
+    # Sec. 7.2, first-order workspaces: row-wise SpGEMM C = A*B, A is I x K with I*K = 10^8 fixed, a tenth
+    # of the K coordinates non-empty with 1000 entries each in A (column k) and in B (row k); K swept
+    "sweep_first_order": [dict(I=10 ** 8 // K, K=K, J=10 ** 8 // K, live_k=K // 10, per_k=1000) for K in (2500, 5000, 10000, 20000)],
+    # Sec. 7.2, second-order workspaces: outer-product SpGEMM, I = K = J = 10^4, the number of non-empty
+    # coordinates of the contracted index swept, 1000 entries each
+    "sweep_second_order": [dict(I=10 ** 4, K=10 ** 4, J=10 ** 4, live_k=n, per_k=1000) for n in (1, 2, 5, 10, 25, 50, 100, 200, 400, 800, 1600)],
+}
+
+
+def run_sweep(name, args, dev):
+    """Dense against sparse workspace over the paper's synthetic shapes; one JSON line."""
+    import torch
+    from paper_2404_04541_b200 import api, binding
+    from workloads import crossover_operands
+
+    ctx = api.Context(dev)
+    second = name == "sweep_second_order"
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    points = []
+    for pt in SWEEPS[name]:
+        At, B = crossover_operands(pt["I"], pt["K"], pt["J"], pt["live_k"], pt["per_k"], args.seed)
+        dB = api.DeviceCSR.from_host(B, device=dev)
+        dA = api.DeviceCSR.from_host(At if second else At.transpose(), device=dev)
+        row = dict(pt)
+        for policy in ("dense", "ism", "auto"):
+            plan = ctx.plan(api.EXPR_OUTER if second else api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, np.float64, policy)
+            sym = ctx.outer_symbolic if second else ctx.spgemm_symbolic
+            try:
+                c, state = sym(plan, dA, dB)
+                nnzC = c.n[1]
+                crd = torch.empty(nnzC, dtype=torch.int32, device=dev)
+                val = torch.empty(nnzC, dtype=torch.float64, device=dev)
+                times = []
+                for s in range(1 + args.steps):
+                    flush.fill_(s & 0xff)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    cc, st = sym(plan, dA, dB)
+                    ctx.spgemm_numeric(plan, cc, st, crd=crd, val=val)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if s > 0:
+                        times.append(e0.elapsed_time(e1))
+                stats = plan.get_stats()
+                row["products"], row["nnzC"] = stats["products"], int(nnzC)
+                row[policy + "_ms"] = float(np.mean(times))
+                del crd, val
+            except binding.SpwsError as exc:
+                row[policy + "_ms"] = None
+                row[policy + "_error"] = binding.status_string(exc.status)
+            plan.close()
+        if row.get("dense_ms") and row.get("ism_ms"):
+            row["dense_over_sparse"] = row["dense_ms"] / row["ism_ms"]
+        points.append(row)
+        ctx._scratch = None
+        torch.cuda.empty_cache()
+    ratios = [p["dense_over_sparse"] for p in points if "dense_over_sparse" in p]
+    line = {"metric": "dense_vs_sparse_workspace_time_ratio", "unit": "ratio (dense ms / sparse ms)", "workload": name,
+            "value": None, "steps": args.steps, "dtype": "f64", "data": "synthetic", "points": points,
+            "sparse_faster_by_up_to": (max(ratios) if ratios else None),
+            "dense_faster_by_up_to": (1.0 / min(ratios) if ratios else None),
+            "paper_context": "sequential CPU code: sparse workspace up to 27.12x faster than dense, dense up to 7.58x faster than sparse"}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="rmat18",
-                    help="rmat18 (default), stencil64, uniform8, wide26, ttm4096, or rmatNN / stencilNN at another size")
+                    help="rmat18 (default), stencil64, uniform8, wide26, ttm4096, rmatNN / stencilNN at another size, "
+                         "or sweep_first_order / sweep_second_order (dense against sparse workspace, Sec. 7.2 shapes)")
     ap.add_argument("--policy", default="auto")
     ap.add_argument("--impl", default="spws", choices=["spws", "reference"])
     ap.add_argument("--seed", type=int, default=1)
@@ -478,6 +545,10 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    if args.workload in SWEEPS:
+        if rank == 0:
+            run_sweep(args.workload, args, dev)
+        return
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 

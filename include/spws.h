@@ -6,6 +6,8 @@
  *
  *   row-wise SpGEMM          C(i,j)   = sum_k A(i,k)   * B(k,j)    A, B, C in CSR
  *   tensor-times-matrix      C(i,j,l) = sum_k A(i,j,k) * B(k,l)    A, C in CSF, B in CSR
+ *   outer-product SpGEMM     C(i,j)   = sum_k A(k,i)   * B(k,j)    A, B, C in CSR, A stored by
+ *                                                                  its rows k (dims = {K, I})
  *
  * following the paper's statement of the problem: an expression over named index variables
  * (Sec. 3), a level format per operand (Sec. 2.1, Fig. 4) and a workspace policy (Sec. 6.1:
@@ -13,7 +15,13 @@
  * expressions are first-order scatters (Sec. 2.2): the loop order i -> k -> j differs from the
  * output order i -> j only by the reduction variable, so every output row (every (i,j) fibre,
  * after hoisting the shared outer loops, Sec. 6.2) owns a first-order workspace along the last
- * index.
+ * index.  The third expression is the paper's running example (Sec. 2.1): the reduction variable is
+ * the outermost loop, both output indices scatter, and ONE second-order workspace serves the whole
+ * result: sparse (Algorithm 1 on integer labels i*J + j, Sec. 5.2, with the accumulation array
+ * and the all array in the scratch buffer) under SPWS_SPARSE_ISM, an I x J value array with
+ * flags under SPWS_DENSE (SPWS_WORKSPACE_TOO_LARGE when the scratch given cannot hold it: the
+ * paper's dense workspace running out of memory, Sec. 7.2), and under SPWS_AUTO the dense one
+ * when it fits and the products number at least I*J/16.
  *
  * Work is split in two device passes (Sec. 5.4: a symbolic phase that precomputes the output
  * structure removes the all array):
@@ -102,7 +110,11 @@ typedef struct {
                                  memory ISM, power of two in [2, 2048]; default 2048              */
     float dense_span_words_per_product; /* AUTO prefers DENSE over the shared-memory ISM when
                                  span/32 <= this * products; default 8                            */
-    int32_t reserved[5];
+    int32_t outer_cap;        /* outer-product form: components the accumulation array of the
+                                 second-order sparse workspace holds (the paper's `cap`); when
+                                 full it is sorted, reduced and united with the all array.
+                                 0 (default): all products in one round                           */
+    int32_t reserved[4];
 } spws_options_t;
 
 typedef struct {
@@ -156,12 +168,14 @@ spws_status_t spws_destroy(spws_handle_t handle);
 /* `cuda_stream` is a cudaStream_t (NULL = the default stream). */
 spws_status_t spws_set_stream(spws_handle_t handle, void* cuda_stream);
 
-/* Parses `expr` -- "C(i,j)=A(i,k)*B(k,j)" or "C(i,j,l)=A(i,j,k)*B(k,l)" with any tensor and index
- * names and optional blanks -- and checks it against the formats: fmts[0] is the result's,
+/* Parses `expr` -- "C(i,j)=A(i,k)*B(k,j)", "C(i,j,l)=A(i,j,k)*B(k,l)" or "C(i,j)=A(k,i)*B(k,j)" with
+ * any tensor and index names and optional blanks -- and checks it against the formats: fmts[0] is the result's,
  * fmts[1], fmts[2] the operands' in the order written.  The expression is accepted when it has
  * exactly one reduction variable, the second operand is a CSR matrix indexed (reduction, last
  * output index), and the first operand's and result's level orders match the loop order
- * (Sec. 2.2 classification: first-order scatter).  Anything else: SPWS_UNSUPPORTED_EXPRESSION. */
+ * (Sec. 2.2 classification: first-order scatter), or when both operands are CSR matrices whose
+ * first index is the shared reduction variable (second-order scatter).  Anything else:
+ * SPWS_UNSUPPORTED_EXPRESSION. */
 spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spws_format_t fmts[3],
                                spws_dtype_t value_type, spws_policy_t policy,
                                const spws_options_t* options /* may be NULL */, spws_plan_t* plan);
@@ -169,11 +183,13 @@ spws_status_t spws_plan_destroy(spws_plan_t plan);
 
 /* The expression check of spws_plan_create on its own (host only, needs no device): the
  * classification of Sec. 2.2 applied to `expr` and `fmts`.  `kind` (may be NULL) receives 0 for
- * the matrix form, 1 for the 3-tensor form. */
+ * the matrix form, 1 for the 3-tensor form, 2 for the outer-product form. */
 spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3], int* kind);
 
 /* Upper bound of the scratch bytes spws_symbolic + spws_numeric need for these operands (reads
- * only dims and n[] of A and B; host-side, launches nothing).  It always suffices; the largest
+ * only dims and n[] of A and B; host-side, launches nothing -- except for the outer-product form,
+ * whose workspace is sized by the number of products: there the call needs A's and B's pos arrays
+ * on the device, counts the products with one kernel on the plan's stream and synchronises).  It always suffices; the largest
  * part is room for one occupancy bitmap per row (rows x min(columns, dense_max_span) / 8 bytes),
  * of which only the rows routed to the dense workspace use their exact span, so a smaller buffer
  * works for narrow rows and spws_symbolic reports SPWS_SCRATCH_TOO_SMALL when it does not.
@@ -191,7 +207,8 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
                             int64_t* sizes_out);
 
 /* Numeric pass.  C->crd[last] and C->val must now hold C->n[last] entries.  Asynchronous: returns
- * after enqueueing; a device-side failure is reported by the next spws_get_stats. */
+ * after enqueueing; a device-side failure is reported by the next spws_get_stats.  (The sparse
+ * workspace of the outer-product form synchronises once per round of its accumulation array.) */
 spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
                            spws_tensor_t* C, void* scratch, size_t scratch_bytes);
 

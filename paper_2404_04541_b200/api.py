@@ -13,6 +13,7 @@ from . import binding as B_
 
 EXPR_SPGEMM = "C(i,j) = A(i,k) * B(k,j)"
 EXPR_TTM = "C(i,j,l) = A(i,j,k) * B(k,l)"
+EXPR_OUTER = "C(i,j) = A(k,i) * B(k,j)"
 
 
 def _dev(a, dtype, device):
@@ -126,6 +127,31 @@ class Context:
             plan = self.plan(EXPR_SPGEMM, (B_.SPWS_CSR,) * 3, dt, policy, **options)
         try:
             c, state = self.spgemm_symbolic(plan, A, B)
+            C = self.spgemm_numeric(plan, c, state)
+            return C, plan.get_stats()
+        finally:
+            if own:
+                plan.close()
+
+    # ------------------------------------------------------------------ outer-product SpGEMM
+    def outer_symbolic(self, plan: B_.Plan, At: DeviceCSR, B: DeviceCSR):
+        """Symbolic pass of C(i,j) = sum_k A(k,i) B(k,j); `At` holds A by its rows k (K x I)."""
+        a, b = At.arrays(), B.arrays()
+        nbytes = plan.workspace_size(a, b)          # counts the products on the device
+        sc = self.scratch(nbytes)
+        pos = torch.empty(At.ncols + 1, dtype=torch.int64, device=self.device)
+        c = B_.csr_arrays(At.ncols, B.ncols, pos, None, None)
+        plan.symbolic(a, b, c, self._aligned_ptr(sc), nbytes)
+        return c, (a, b, sc, nbytes)
+
+    def spgemm_outer(self, At: DeviceCSR, B: DeviceCSR, policy="auto", plan: B_.Plan | None = None, **options):
+        """C = A^T-stored-by-rows times B through a second-order workspace; returns (C, stats)."""
+        own = plan is None
+        if own:
+            dt = np.float64 if At.val.dtype == torch.float64 else np.float32
+            plan = self.plan(EXPR_OUTER, (B_.SPWS_CSR,) * 3, dt, policy, **options)
+        try:
+            c, state = self.outer_symbolic(plan, At, B)
             C = self.spgemm_numeric(plan, c, state)
             return C, plan.get_stats()
         finally:

@@ -53,7 +53,7 @@ class spws_options_t(ctypes.Structure):
     _fields_ = [("validate", ctypes.c_int32), ("ism_warp_cap", ctypes.c_int32), ("ism_cta_cap", ctypes.c_int32),
                 ("dense_unit_outputs", ctypes.c_int32), ("dense_max_span", ctypes.c_int32),
                 ("fallback_cap", ctypes.c_int32), ("dense_span_words_per_product", ctypes.c_float),
-                ("reserved", ctypes.c_int32 * 5)]
+                ("outer_cap", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4)]
 
 
 class spws_stats_t(ctypes.Structure):

@@ -219,4 +219,16 @@ cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host
 cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
                               const i64* rowptr, int* Ccrd, void* Cval);
 
+// outer.cu: second-order workspaces of the outer-product form
+cudaError_t launch_outer_counts(const LaunchCtx& c, const Csr& At, const Csr& B, int* cnt);
+size_t outer_sort_scratch_bytes(i64 n);
+cudaError_t launch_outer_ism(const LaunchCtx& c, bool numeric, const Csr& At, const Csr& B, const i64* koff, i64 P, i64 cap, i64 J,
+                             int label_bits, u64* kA, void* vA, u64* kB, void* vB, int* head, i64* at, char* sort_tmp,
+                             i64* block_sums, i64* nnz_dev, i64* nnz_host_pinned, bool* result_first);
+cudaError_t launch_coo_pos(const LaunchCtx& c, const u64* ukeys, i64 nnz, i64 m, i64 J, i64* pos);
+cudaError_t launch_coo_out(const LaunchCtx& c, const u64* ukeys, const void* uvals, i64 nnz, i64 J, int* Ccrd, void* Cval);
+cudaError_t launch_outer_dense(const LaunchCtx& c, bool numeric, const Csr& At, const Csr& B, const i64* koff, i64 P, i64 m, i64 J,
+                               unsigned* dbits, void* dvals, int* cnt, const i64* pos, int* Ccrd, void* Cval);
+cudaError_t launch_outer_total(const LaunchCtx& c, const Csr& At, const Csr& B, u64* total_mapped_host);
+
 }  // namespace spws

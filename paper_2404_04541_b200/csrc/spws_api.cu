@@ -1,5 +1,6 @@
 // C ABI of the spws library: handles, plans, expression check, scratch layout and the launch
 // sequences of the symbolic and numeric passes.  Host code only.
+#include <algorithm>
 #include <cctype>
 #include <cstdio>
 #include <cstring>
@@ -20,7 +21,7 @@ struct spws_handle_s {
 
 struct spws_plan_s {
     spws_handle_t h = nullptr;
-    int kind = 0;               // 0 SpGEMM (CSR x CSR -> CSR), 1 TTM (CSF3 x CSR -> CSF3)
+    int kind = 0;               // 0 SpGEMM (CSR x CSR -> CSR), 1 TTM (CSF3 x CSR -> CSF3), 2 outer-product SpGEMM (A by rows k)
     int is_f64 = 1;
     int policy = SPWS_AUTO;
     spws_options_t opt{};
@@ -33,6 +34,9 @@ struct spws_plan_s {
     int max_span_words = 0;     // widest dense bitmap of the last symbolic pass
     int max_warp_cnt = 0;       // most outputs of a warp-numeric row
     int64_t bin_rows[NCLASS] = {};  // rows per internal class of the last symbolic pass
+    // outer-product form: what the last symbolic pass decided
+    int64_t outer_products = 0;
+    bool outer_dense = false;
     // optional per-kernel timing: ev[g] is recorded after group g; ev_start[] before each pass
     bool profiling = false;
     cudaEvent_t ev[SPWS_T_COUNT] = {};
@@ -80,10 +84,15 @@ bool distinct(const std::vector<std::string>& v) {
     return true;
 }
 
-// Accepts out(o_1..o_N) = x(o_1..o_{N-1}, r) * y(r, o_N), N = 2 or 3, with formats
-// (CSR, CSR, CSR) or (CSF3, CSF3, CSR): loop order o_1 -> .. -> r -> o_N, output order
-// o_1 -> .. -> o_N; they mismatch only by the reduction variable sitting one position from the
-// innermost index: a first-order scatter.  Returns the kind or -1.
+// Accepts
+//   out(o_1..o_N) = x(o_1..o_{N-1}, r) * y(r, o_N), N = 2 or 3, with formats (CSR, CSR, CSR) or
+//     (CSF3, CSF3, CSR): loop order o_1 -> .. -> r -> o_N, output order o_1 -> .. -> o_N; they
+//     mismatch only by the reduction variable sitting one position from the innermost index: a
+//     first-order scatter (kinds 0 and 1);
+//   out(o_1, o_2) = x(r, o_1) * y(r, o_2) with formats (CSR, CSR, CSR): loop order r -> o_1 -> o_2,
+//     the reduction variable outermost, so both output indices scatter: a second-order scatter
+//     (kind 2, the outer-product form).
+// Returns the kind or -1.
 int classify_expression(const char* expr, const spws_format_t fmts[3]) {
     const char* s = expr;
     Access out, x, y;
@@ -98,11 +107,16 @@ int classify_expression(const char* expr, const spws_format_t fmts[3]) {
     if (N != 2 && N != 3) return -1;
     if (x.idx.size() != N || y.idx.size() != 2) return -1;
     if (!distinct(out.idx) || !distinct(x.idx) || !distinct(y.idx)) return -1;
+    if (out.name == x.name || out.name == y.name) return -1;
+    if (N == 2 && x.idx[0] == y.idx[0] && x.idx[1] == out.idx[0] && y.idx[1] == out.idx[1] && x.idx[0] != out.idx[0] &&
+        x.idx[0] != out.idx[1]) {
+        if (fmts[0] != SPWS_CSR || fmts[1] != SPWS_CSR || fmts[2] != SPWS_CSR) return -1;
+        return 2;
+    }
     const std::string& r = x.idx[N - 1];
     for (size_t a = 0; a < N; ++a) if (out.idx[a] == r) return -1;           // r must be a reduction variable
     for (size_t a = 0; a + 1 < N; ++a) if (x.idx[a] != out.idx[a]) return -1;
     if (y.idx[0] != r || y.idx[1] != out.idx[N - 1]) return -1;
-    if (out.name == x.name || out.name == y.name) return -1;
     if (N == 2) {
         if (fmts[0] != SPWS_CSR || fmts[1] != SPWS_CSR || fmts[2] != SPWS_CSR) return -1;
         return 0;
@@ -196,6 +210,10 @@ spws_status_t check_operands(const spws_plan_s* p, const spws_tensor_t* A, const
         if (A->order != 2) return SPWS_INVALID_ARGUMENT;
         S.m = A->dims[0]; S.k = A->dims[1]; S.nnzA = A->n[1]; S.n_i = 0;
         S.A = Csr{LL(A->pos[1]), A->crd[1], A->val, (int)S.m, (int)S.k};
+    } else if (p->kind == 2) {                  // A stored by its rows k: dims = (K, I)
+        if (A->order != 2) return SPWS_INVALID_ARGUMENT;
+        S.m = A->dims[1]; S.k = A->dims[0]; S.nnzA = A->n[1]; S.n_i = 0;
+        S.A = Csr{LL(A->pos[1]), A->crd[1], A->val, (int)S.k, (int)S.m};
     } else {
         if (A->order != 3) return SPWS_INVALID_ARGUMENT;
         S.m = A->n[1]; S.k = A->dims[2]; S.nnzA = A->n[2]; S.n_i = A->n[0];
@@ -210,7 +228,7 @@ spws_status_t check_operands(const spws_plan_s* p, const spws_tensor_t* A, const
         return SPWS_INVALID_ARGUMENT;
     if (S.k != B->dims[0]) return SPWS_DIM_MISMATCH;
     if (!need_pointers) return SPWS_OK;
-    if (S.m > 0 && (!S.A.pos)) return SPWS_INVALID_ARGUMENT;
+    if ((p->kind == 2 ? S.k : S.m) > 0 && (!S.A.pos)) return SPWS_INVALID_ARGUMENT;
     if (S.nnzA > 0 && (!S.A.crd || !S.A.val)) return SPWS_INVALID_ARGUMENT;
     if (B->dims[0] > 0 && !S.B.pos) return SPWS_INVALID_ARGUMENT;
     if (S.nnzB > 0 && (!S.B.crd || !S.B.val)) return SPWS_INVALID_ARGUMENT;
@@ -219,9 +237,9 @@ spws_status_t check_operands(const spws_plan_s* p, const spws_tensor_t* A, const
 
 spws_status_t check_output_dims(const spws_plan_s* p, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* C) {
     if (!C) return SPWS_INVALID_ARGUMENT;
-    if (p->kind == 0) {
+    if (p->kind == 0 || p->kind == 2) {
         if (C->order != 2) return SPWS_INVALID_ARGUMENT;
-        if (C->dims[0] != A->dims[0] || C->dims[1] != B->dims[1]) return SPWS_DIM_MISMATCH;
+        if (C->dims[0] != A->dims[p->kind == 0 ? 0 : 1] || C->dims[1] != B->dims[1]) return SPWS_DIM_MISMATCH;
         if (!C->pos[1]) return SPWS_INVALID_ARGUMENT;
     } else {
         if (C->order != 3) return SPWS_INVALID_ARGUMENT;
@@ -299,6 +317,188 @@ inline void mark_start(spws_plan_s* p, int pass) {
     p->ev_pass[pass] = true;
 }
 
+// ---- outer-product form (kind 2): scratch layout and the two passes -------------------------
+struct OuterLayout {
+    size_t ctl, cnt, koff, block_sums, fixed_end;
+    // sparse workspace
+    size_t kA, kB, vA, vB, head, at, sort_tmp, ism_end;
+    // dense workspace
+    size_t dbits, dvals, dcnt, dense_end;
+    int64_t N;                  // entries of each (label, value) array
+};
+
+OuterLayout make_outer_layout(const spws_plan_s* p, int64_t I, int64_t K, int64_t J, int64_t P) {
+    OuterLayout L{};
+    const size_t V = p->is_f64 ? 8 : 4;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
+    const int64_t cap = p->opt.outer_cap > 0 ? p->opt.outer_cap : P;
+    L.N = P + (cap < P ? cap : 0);
+    const int64_t longest = std::max<int64_t>(std::max<int64_t>(K, I), L.N);
+    L.ctl = take(sizeof(DevCtl));
+    L.cnt = take(4 * (size_t)K);
+    L.koff = take(8 * ((size_t)K + 1));
+    L.block_sums = take(8 * ((size_t)longest / 2048 + 2));
+    L.fixed_end = o;
+    L.kA = take(8 * (size_t)L.N);
+    L.kB = take(8 * (size_t)L.N);
+    L.vA = take(V * (size_t)L.N);
+    L.vB = take(V * (size_t)L.N);
+    L.head = take(4 * (size_t)L.N);
+    L.at = take(8 * ((size_t)L.N + 1));
+    L.sort_tmp = take(outer_sort_scratch_bytes(L.N));
+    L.ism_end = o;
+    o = L.fixed_end;
+    const size_t row_words = (size_t)((J + 31) / 32);
+    L.dbits = take(4 * (size_t)I * row_words);
+    L.dvals = take(V * (size_t)I * (size_t)J);
+    L.dcnt = take(4 * (size_t)I);
+    L.dense_end = o;
+    return L;
+}
+
+int label_bits_of(int64_t I, int64_t J) {
+    const unsigned long long top = (unsigned long long)I * (unsigned long long)J;
+    int bits = 1;
+    while (bits < 64 && (top >> bits) != 0) ++bits;
+    return bits;
+}
+
+// products of the outer form, counted on the device into a word of the plan's pinned block
+spws_status_t outer_count_products(spws_plan_s* p, const Shapes& S, int64_t* P) {
+    LaunchCtx c{};
+    c.stream = p->h->stream;
+    c.sm_count = p->h->sm_count;
+    u64* word = reinterpret_cast<u64*>(&p->host_ctl->products);
+    *word = 0;
+    CUDA_TRY(launch_outer_total(c, S.A, S.B, word));
+    CUDA_TRY(cudaStreamSynchronize(c.stream));
+    *P = (int64_t)*word;
+    return SPWS_OK;
+}
+
+bool outer_wants_dense(const spws_plan_s* p, int64_t I, int64_t J, int64_t P, size_t scratch_bytes, const OuterLayout& L, spws_status_t* st) {
+    *st = SPWS_OK;
+    const bool fits = scratch_bytes >= L.dense_end;
+    if (p->policy == SPWS_DENSE) {
+        if (!fits) *st = SPWS_WORKSPACE_TOO_LARGE;
+        return true;
+    }
+    if (p->policy == SPWS_SPARSE_ISM) return false;
+    return fits && (double)P * 16.0 >= (double)I * (double)J;
+}
+
+spws_status_t outer_symbolic(spws_plan_s* plan, const Shapes& S, spws_tensor_t* C, void* scratch, size_t scratch_bytes, int64_t* sizes_out) {
+    const int64_t I = S.m, K = S.k, J = S.ncols;
+    if (I * J < 0 || (I > 0 && J > (int64_t)(0x7fffffffffffffffll / (I > 0 ? I : 1)))) return SPWS_INVALID_ARGUMENT;
+    int64_t P = 0;
+    spws_status_t st = outer_count_products(plan, S, &P);
+    if (st != SPWS_OK) return st;
+    if (P > 0x7fff0000ll) return SPWS_INTERNAL_OVERFLOW;            // product ordinals and scans are 31-bit here
+    const OuterLayout L = make_outer_layout(plan, I, K, J, P);
+    if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
+    const bool dense = outer_wants_dense(plan, I, J, P, scratch_bytes, L, &st);
+    if (st != SPWS_OK) return st;
+    if (!dense && scratch_bytes < L.ism_end) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c{};
+    c.stream = plan->h->stream;
+    c.sm_count = plan->h->sm_count;
+    c.ctl = reinterpret_cast<DevCtl*>(sc + L.ctl);
+    c.is_f64 = plan->is_f64;
+    cudaStream_t stream = c.stream;
+    CUDA_TRY(cudaMemsetAsync(c.ctl, 0, sizeof(DevCtl), stream));
+    mark_start(plan, 0);
+    int* cnt = reinterpret_cast<int*>(sc + L.cnt);
+    i64* koff = reinterpret_cast<i64*>(sc + L.koff);
+    i64* block_sums = reinterpret_cast<i64*>(sc + L.block_sums);
+    CUDA_TRY(launch_outer_counts(c, S.A, S.B, cnt));
+    CUDA_TRY(launch_scan_counts(c, cnt, (int)K, koff, block_sums, &c.ctl->products));
+    mark(plan, SPWS_T_SYM_BOUNDS);
+    i64* pos = LL(C->pos[1]);
+    int64_t nnz = 0;
+    if (dense) {
+        const size_t row_words = (size_t)((J + 31) / 32);
+        CUDA_TRY(cudaMemsetAsync(sc + L.dbits, 0, 4 * (size_t)I * row_words, stream));
+        CUDA_TRY(launch_outer_dense(c, false, S.A, S.B, koff, P, I, J, reinterpret_cast<unsigned*>(sc + L.dbits), nullptr,
+                                    reinterpret_cast<int*>(sc + L.dcnt), nullptr, nullptr, nullptr));
+        CUDA_TRY(launch_scan_counts(c, reinterpret_cast<int*>(sc + L.dcnt), (int)I, pos, block_sums, &c.ctl->nnz));
+        mark(plan, SPWS_T_SYM_DENSE_CTA);
+    } else {
+        bool first = true;
+        i64* nnz_host = reinterpret_cast<i64*>(&plan->host_ctl->nnz);
+        const int64_t cap = plan->opt.outer_cap > 0 ? plan->opt.outer_cap : (P > 0 ? P : 1);
+        CUDA_TRY(launch_outer_ism(c, false, S.A, S.B, koff, P, cap, J, label_bits_of(I, J), reinterpret_cast<u64*>(sc + L.kA), nullptr,
+                                  reinterpret_cast<u64*>(sc + L.kB), nullptr, reinterpret_cast<int*>(sc + L.head),
+                                  reinterpret_cast<i64*>(sc + L.at), sc + L.sort_tmp, block_sums, &c.ctl->nnz, nnz_host, &first));
+        nnz = *nnz_host;
+        CUDA_TRY(cudaMemcpyAsync(&c.ctl->nnz, nnz_host, sizeof(i64), cudaMemcpyHostToDevice, stream));
+        CUDA_TRY(launch_coo_pos(c, reinterpret_cast<u64*>(sc + (first ? L.kA : L.kB)), nnz, I, J, pos));
+        mark(plan, SPWS_T_SYM_ISM_GLOBAL);
+    }
+    CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    const DevCtl& hc = *plan->host_ctl;
+    plan->stats = spws_stats_t{};
+    plan->stats.device_status = hc.status;
+    if (hc.status != 0) return from_dev_status(hc.status);
+    plan->stats.rows = I;
+    plan->stats.products = P;
+    plan->stats.nnz = hc.nnz;
+    plan->stats.rows_per_class[dense ? public_class(CLS_DENSE_CTA) : public_class(CLS_ISM_GLOBAL)] = I;
+    plan->stats.products_per_class[dense ? public_class(CLS_DENSE_CTA) : public_class(CLS_ISM_GLOBAL)] = P;
+    plan->stats.nnz_per_class[dense ? public_class(CLS_DENSE_CTA) : public_class(CLS_ISM_GLOBAL)] = hc.nnz;
+    plan->stats.launches_symbolic = c.launches;
+    plan->outer_products = P;
+    plan->outer_dense = dense;
+    C->n[0] = C->dims[0];
+    C->n[1] = hc.nnz;
+    C->n[2] = 0;
+    if (sizes_out) { sizes_out[0] = C->n[0]; sizes_out[1] = C->n[1]; sizes_out[2] = 0; }
+    plan->symbolic_ok = true;
+    plan->m = S.m;
+    plan->scratch = scratch;
+    return SPWS_OK;
+}
+
+spws_status_t outer_numeric(spws_plan_s* plan, const Shapes& S, spws_tensor_t* C, void* scratch, size_t scratch_bytes) {
+    const int64_t I = S.m, K = S.k, J = S.ncols, P = plan->outer_products;
+    if (C->n[1] < plan->stats.nnz) return SPWS_OUTPUT_TOO_SMALL;
+    if (plan->stats.nnz > 0 && (!C->crd[1] || !C->val)) return SPWS_INVALID_ARGUMENT;
+    const OuterLayout L = make_outer_layout(plan, I, K, J, P);
+    if (scratch_bytes < (plan->outer_dense ? L.dense_end : L.ism_end)) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c{};
+    c.stream = plan->h->stream;
+    c.sm_count = plan->h->sm_count;
+    c.ctl = reinterpret_cast<DevCtl*>(sc + L.ctl);
+    c.is_f64 = plan->is_f64;
+    const size_t V = plan->is_f64 ? 8 : 4;
+    i64* koff = reinterpret_cast<i64*>(sc + L.koff);
+    i64* block_sums = reinterpret_cast<i64*>(sc + L.block_sums);
+    mark_start(plan, 1);
+    if (plan->outer_dense) {
+        const size_t row_words = (size_t)((J + 31) / 32);
+        CUDA_TRY(cudaMemsetAsync(sc + L.dbits, 0, 4 * (size_t)I * row_words, c.stream));
+        CUDA_TRY(cudaMemsetAsync(sc + L.dvals, 0, V * (size_t)I * (size_t)J, c.stream));
+        CUDA_TRY(launch_outer_dense(c, true, S.A, S.B, koff, P, I, J, reinterpret_cast<unsigned*>(sc + L.dbits), sc + L.dvals, nullptr,
+                                    LL(C->pos[1]), C->crd[1], C->val));
+        mark(plan, SPWS_T_NUM_DENSE_CTA);
+    } else {
+        bool first = true;
+        i64* nnz_host = reinterpret_cast<i64*>(&plan->host_ctl->nnz);
+        const int64_t cap = plan->opt.outer_cap > 0 ? plan->opt.outer_cap : (P > 0 ? P : 1);
+        CUDA_TRY(launch_outer_ism(c, true, S.A, S.B, koff, P, cap, J, label_bits_of(I, J), reinterpret_cast<u64*>(sc + L.kA), sc + L.vA,
+                                  reinterpret_cast<u64*>(sc + L.kB), sc + L.vB, reinterpret_cast<int*>(sc + L.head),
+                                  reinterpret_cast<i64*>(sc + L.at), sc + L.sort_tmp, block_sums, &c.ctl->kept[0], nnz_host, &first));
+        if (*nnz_host != plan->stats.nnz) return SPWS_BAD_SEQUENCE;     // operands differ from the symbolic pass's
+        CUDA_TRY(launch_coo_out(c, reinterpret_cast<u64*>(sc + (first ? L.kA : L.kB)), sc + (first ? L.vA : L.vB), *nnz_host, J, C->crd[1], C->val));
+        mark(plan, SPWS_T_NUM_ISM_GLOBAL);
+    }
+    plan->stats.launches_numeric = c.launches;
+    return SPWS_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -365,6 +565,7 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
     if (o.dense_max_span < 32 || o.dense_max_span > (1 << 19)) return SPWS_INVALID_ARGUMENT;
     if (!is_pow2(o.fallback_cap) || o.fallback_cap < 2 || o.fallback_cap > 2048) return SPWS_INVALID_ARGUMENT;
     if (!(o.dense_span_words_per_product > 0.0f)) return SPWS_INVALID_ARGUMENT;
+    if (o.outer_cap < 0) return SPWS_INVALID_ARGUMENT;
     spws_plan_s* p = new (std::nothrow) spws_plan_s;
     if (!p) return SPWS_INVALID_ARGUMENT;
     p->h = handle;
@@ -424,8 +625,18 @@ spws_status_t spws_plan_destroy(spws_plan_t plan) {
 spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, size_t* bytes) {
     if (!plan || !bytes) return SPWS_INVALID_ARGUMENT;
     Shapes S{};
-    spws_status_t st = check_operands(plan, A, B, S, false);   // pointers may still be unset when sizing
+    spws_status_t st = check_operands(plan, A, B, S, plan->kind != 2);   // pointers may still be unset when sizing
     if (st != SPWS_OK) return st;
+    if (plan->kind == 2) {                      // sized by the number of products, counted on the device
+        int64_t P = 0;
+        if ((st = outer_count_products(plan, S, &P)) != SPWS_OK) return st;
+        const OuterLayout OL = make_outer_layout(plan, S.m, S.k, S.ncols, P);
+        const size_t dense_ok = (double)S.m * (double)S.ncols <= 2.0e9 ? OL.dense_end : 0;     // a dense workspace beyond 2^31 cells is never offered
+        *bytes = plan->policy == SPWS_SPARSE_ISM ? OL.ism_end
+                 : plan->policy == SPWS_DENSE ? OL.dense_end
+                 : std::max(OL.ism_end, (double)P * 16.0 >= (double)S.m * (double)S.ncols ? dense_ok : (size_t)0);
+        return SPWS_OK;
+    }
     const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
     *bytes = L.fixed_end + rest_reserve(plan, S.m, S.ncols);
     return SPWS_OK;
@@ -440,6 +651,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     if (st != SPWS_OK) return st;
     if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
     if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind == 2) return outer_symbolic(plan, S, C, scratch, scratch_bytes, sizes_out);
     const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
     if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
     char* sc = static_cast<char*>(scratch);
@@ -544,6 +756,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     if (st != SPWS_OK) return st;
     if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
     if (scratch != plan->scratch || S.m != plan->m) return SPWS_BAD_SEQUENCE;
+    if (plan->kind == 2) return outer_numeric(plan, S, C, scratch, scratch_bytes);
     const int last = plan->kind == 0 ? 1 : 2;
     if (C->n[last] < plan->stats.nnz) return SPWS_OUTPUT_TOO_SMALL;
     if (plan->stats.nnz > 0 && (!C->crd[last] || !C->val)) return SPWS_INVALID_ARGUMENT;
@@ -591,6 +804,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
 spws_status_t spws_gather_ceiling(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* C,
                                   void* scratch, size_t scratch_bytes, uint64_t* index_sum, double* value_sum) {
     if (!plan || !index_sum || !value_sum) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind == 2) return SPWS_UNSUPPORTED_EXPRESSION;    // the first-order dense kernels do not run for the outer form
     if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S);
@@ -651,7 +865,7 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
     // device images of the operands
     spws_tensor_t dA = *A, dB = *B, dC = *C;
     const int lastA = plan->kind == 0 ? 1 : 2;
-    const bool same = (plan->kind == 0) && A->pos[1] == B->pos[1] && A->crd[1] == B->crd[1] && A->val == B->val;
+    const bool same = (plan->kind != 1) && A->pos[1] == B->pos[1] && A->crd[1] == B->crd[1] && A->val == B->val;
     struct Copy { void* dst; const void* src; size_t bytes; };
     std::vector<Copy> h2d;
     auto stage = [&](const void* src, size_t bytes) -> void* {
@@ -659,8 +873,8 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
         h2d.push_back(Copy{d, src, bytes});
         return d;
     };
-    if (plan->kind == 0) {
-        dA.pos[1] = (int64_t*)stage(A->pos[1], 8 * ((size_t)S.m + 1));
+    if (plan->kind != 1) {
+        dA.pos[1] = (int64_t*)stage(A->pos[1], 8 * ((size_t)A->dims[0] + 1));
         dA.crd[1] = (int32_t*)stage(A->crd[1], 4 * (size_t)S.nnzA);
     } else {
         dA.pos[0] = (int64_t*)stage(A->pos[0], 16);
@@ -679,7 +893,7 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
         dB.val = stage(B->val, V * (size_t)S.nnzB);
     }
     (void)lastA;
-    if (plan->kind == 0) {
+    if (plan->kind != 1) {
         dC.pos[1] = (int64_t*)carve(8 * ((size_t)S.m + 1));
     } else {
         dC.pos[0] = (int64_t*)carve(16);
@@ -688,19 +902,23 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
         dC.crd[1] = (int32_t*)carve(4 * (size_t)A->n[1]);
         dC.pos[2] = (int64_t*)carve(8 * ((size_t)A->n[1] + 1));
     }
-    size_t ws_bytes = 0;
-    if ((st = spws_workspace_size(plan, A, B, &ws_bytes)) != SPWS_OK) return st;
+    if (!fits) {
+        if (arena_needed) *arena_needed = o;      // lower bound: scratch and C's entries are not counted yet
+        return SPWS_SCRATCH_TOO_SMALL;
+    }
+    for (const Copy& cp : h2d)
+        if (cp.bytes) CUDA_TRY(cudaMemcpyAsync(cp.dst, cp.src, cp.bytes, cudaMemcpyHostToDevice, stream));
+    size_t ws_bytes = 0;                          // the outer-product form sizes its workspace from the device copies
+    if ((st = spws_workspace_size(plan, plan->kind == 2 ? &dA : A, plan->kind == 2 ? &dB : B, &ws_bytes)) != SPWS_OK) return st;
     char* scratch = carve(ws_bytes);
     if (!fits) {
         if (arena_needed) *arena_needed = o;      // lower bound: C's entries are not counted yet
         return SPWS_SCRATCH_TOO_SMALL;
     }
-    for (const Copy& cp : h2d)
-        if (cp.bytes) CUDA_TRY(cudaMemcpyAsync(cp.dst, cp.src, cp.bytes, cudaMemcpyHostToDevice, stream));
     int64_t cap[3] = {C->n[0], C->n[1], C->n[2]};
     int64_t sizes[3];
     if ((st = spws_symbolic(plan, &dA, &dB, &dC, scratch, ws_bytes, sizes)) != SPWS_OK) return st;
-    const int last = plan->kind == 0 ? 1 : 2;
+    const int last = plan->kind == 1 ? 2 : 1;
     const size_t nnz = (size_t)sizes[last];
     dC.crd[last] = (int32_t*)carve(4 * nnz);
     dC.val = carve(V * nnz);
@@ -710,7 +928,7 @@ spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const 
     if ((int64_t)nnz > cap[last]) return SPWS_OUTPUT_TOO_SMALL;
     if (plan->kind == 1 && (sizes[0] > cap[0] || sizes[1] > cap[1])) return SPWS_OUTPUT_TOO_SMALL;
     if ((st = spws_numeric(plan, &dA, &dB, &dC, scratch, ws_bytes)) != SPWS_OK) return st;
-    if (plan->kind == 0) {
+    if (plan->kind != 1) {
         CUDA_TRY(cudaMemcpyAsync(C->pos[1], dC.pos[1], 8 * ((size_t)S.m + 1), cudaMemcpyDeviceToHost, stream));
     } else {
         CUDA_TRY(cudaMemcpyAsync(C->pos[0], dC.pos[0], 16, cudaMemcpyDeviceToHost, stream));

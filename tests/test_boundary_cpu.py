@@ -45,7 +45,10 @@ def test_status_strings(binding):
     ("Z(a,b,c) = T(a,b,x) * M(x,c)", (1, 1, 0), True),
     ("C(i,j)=A(i,k)*B(k,j)", (0, 1, 0), False),        # formats do not fit the order
     ("C(i,j,l)=A(i,j,k)*B(k,l)", (0, 0, 0), False),
-    ("C(i,j)=A(k,i)*B(k,j)", (0, 0, 0), False),        # outer-product order: second-order scatter
+    ("C(i,j)=A(k,i)*B(k,j)", (0, 0, 0), True),         # outer-product order: second-order scatter
+    ("R(u,v) = P(w,u) * Q(w,v)", (0, 0, 0), True),
+    ("C(i,j)=A(k,i)*B(k,j)", (0, 1, 0), False),
+    ("C(i,j)=A(k,j)*B(k,i)", (0, 0, 0), False),        # outer-product order with the output transposed
     ("C(j,i)=A(i,k)*B(k,j)", (0, 0, 0), False),        # transposed output
     ("C(i,j)=A(i,k)*B(j,k)", (0, 0, 0), False),        # B accessed against its storage order
     ("C(i,j)=A(i,j)*B(i,j)", (0, 0, 0), False),        # element-wise: no reduction variable

@@ -449,6 +449,80 @@ def test_full_rmat18_every_entry_streamed(ctx, oracle_mod):
     print(f"rmat18: {entries} entries compared, {second} needed the sum|a*b| clause")
 
 
+# ------------------------------------------------------------------ outer-product form, second-order workspace
+def run_outer(ctx, A, B, policy="auto", **options):
+    """A is the I x K operand; the library takes it by its rows k, i.e. the CSR of its transpose."""
+    from paper_2404_04541_b200 import api
+    dAt = api.DeviceCSR.from_host(A.transpose())
+    dB = api.DeviceCSR.from_host(B)
+    C, stats = ctx.spgemm_outer(dAt, dB, policy=policy, **options)
+    return C.pos.cpu().numpy(), C.crd.cpu().numpy(), C.val.cpu().numpy(), stats
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+@pytest.mark.parametrize("m,k,n,dens,seed", [(1, 1, 1, 1.0, 0), (37, 64, 700, 0.08, 1), (200, 150, 1000, 0.05, 2),
+                                             (64, 64, 64, 0.5, 3), (300, 20, 5000, 0.1, 4)])
+def test_outer_product_matches_the_rowwise_oracle(ctx, oracle_mod, policy, m, k, n, dens, seed):
+    A = random_csr(m, k, dens, seed, empty_row_frac=0.1)
+    B = random_csr(k, n, dens, seed + 9, empty_row_frac=0.1)
+    ref = oracle_mod.spgemm(A, B)
+    pos, crd, val, stats = run_outer(ctx, A, B, policy)
+    assert stats["products"] == int(ref.products.sum()) and stats["nnz"] == ref.nnz
+    assert_matches((pos, crd, val), ref, np.float64)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+@pytest.mark.parametrize("cap", [0, 1, 2, 3, 7, 1000, 10 ** 6])
+def test_outer_product_sparse_workspace_reproduces_algorithm1(ctx, oracle_mod, cap, dtype):
+    """The sparse second-order workspace with an accumulation array of `cap` components sums in the
+    order Algorithm 1 fixes (sort and reduce the full array on its own, then all + accumulated), so
+    with separate multiply and add it must equal the oracle's restatement bit for bit (f64) at
+    every capacity; one round (cap 0) equals the plain loop-order sum k -> i -> j."""
+    A = random_csr(60, 50, 0.15, 21, empty_row_frac=0.1)
+    B = random_csr(50, 90, 0.15, 22, empty_row_frac=0.1)
+    A.val = A.val.astype(dtype)
+    B.val = B.val.astype(dtype)
+    P = int(oracle_mod.spgemm(A, B).products.sum())
+    ref = oracle_mod.ism_outer(A, B, cap if cap > 0 else P)
+    pos, crd, val, stats = run_outer(ctx, A, B, "ism", outer_cap=cap)
+    assert np.array_equal(pos, ref.pos) and np.array_equal(crd, ref.crd)
+    if dtype == np.float64:
+        assert np.array_equal(val, ref.val)
+    else:
+        assert np.allclose(val, ref.val, rtol=1e-5, atol=1e-6)
+
+
+def test_outer_product_on_a_power_law_matrix_and_wide_labels(ctx, oracle_mod):
+    A = rmat_csr(11, 8, 5)
+    ref = oracle_mod.spgemm(A, A, threads=4)
+    for policy in POLICIES:
+        pos, crd, val, stats = run_outer(ctx, A, A, policy)
+        assert_matches((pos, crd, val), ref, np.float64)
+    # labels beyond 32 bits: 3000 x 2^22 outputs; the dense workspace cannot be offered here
+    B = uniform_rows_csr(500, 1 << 22, 6, 7)
+    A2 = random_csr(3000, 500, 0.01, 8)
+    ref = oracle_mod.spgemm(A2, B)
+    pos, crd, val, stats = run_outer(ctx, A2, B, "auto")
+    assert stats["rows_per_class"][GLOBAL] == 3000
+    assert_matches((pos, crd, val), ref, np.float64)
+    # the dense workspace forced with a scratch buffer that cannot hold I x J values: refused, like
+    # the paper's dense workspace running out of memory
+    import torch
+    from paper_2404_04541_b200 import api, binding
+    dAt, dB = api.DeviceCSR.from_host(A2.transpose()), api.DeviceCSR.from_host(B)
+    sparse_plan = ctx.plan(api.EXPR_OUTER, (binding.SPWS_CSR,) * 3, np.float64, "ism")
+    nbytes = sparse_plan.workspace_size(dAt.arrays(), dB.arrays())
+    sparse_plan.close()
+    dense_plan = ctx.plan(api.EXPR_OUTER, (binding.SPWS_CSR,) * 3, np.float64, "dense")
+    assert dense_plan.workspace_size(dAt.arrays(), dB.arrays()) > 3000 * (1 << 22) * 8
+    sc = ctx.scratch(nbytes)
+    c = binding.csr_arrays(3000, 1 << 22, torch.empty(3001, dtype=torch.int64, device="cuda"), None, None)
+    with pytest.raises(binding.SpwsError) as e:
+        dense_plan.symbolic(dAt.arrays(), dB.arrays(), c, ctx._aligned_ptr(sc), nbytes)
+    assert e.value.status == binding.SPWS_WORKSPACE_TOO_LARGE
+    dense_plan.close()
+
+
 # ------------------------------------------------------------------ gather-only lower bound
 @pytest.mark.parametrize("name", ["rmat", "stencil", "heavy"])
 def test_gather_ceiling_visits_every_product_once(ctx, name):
@@ -629,7 +703,7 @@ def test_error_statuses(ctx):
     import torch
     from paper_2404_04541_b200 import api, binding
     with pytest.raises(binding.SpwsError) as e:
-        ctx.plan("C(i,j) = A(k,i) * B(k,j)", (0, 0, 0), np.float64)
+        ctx.plan("C(i,j) = A(i,k) * B(j,k)", (0, 0, 0), np.float64)
     assert e.value.status == binding.SPWS_UNSUPPORTED_EXPRESSION
     A = api.DeviceCSR.from_host(random_csr(10, 12, 0.3, 1))
     Bm = api.DeviceCSR.from_host(random_csr(13, 9, 0.3, 2))

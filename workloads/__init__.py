@@ -11,12 +11,13 @@ from .generators import (
     stencil27_csr,
     uniform_csf3,
     random_csr,
+    crossover_operands,
     config_inputs,
     CONFIG_NAMES,
 )
 
 __all__ = [
     "CSR", "CSF3", "csr_is_canonical", "csf3_is_canonical",
-    "uniform_rows_csr", "rmat_csr", "stencil27_csr", "uniform_csf3", "random_csr",
+    "uniform_rows_csr", "rmat_csr", "stencil27_csr", "uniform_csf3", "random_csr", "crossover_operands",
     "config_inputs", "CONFIG_NAMES",
 ]

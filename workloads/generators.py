@@ -139,6 +139,29 @@ def random_csr(nrows: int, ncols: int, density: float, seed: int, lo=-1.0, hi=1.
     return CSR.from_dense(d, dtype=dtype, keep_mask=mask)
 
 
+def crossover_operands(I: int, K: int, J: int, live_k: int, per_k: int, seed: int, dtype=np.float64):
+    """Operands of the dense-versus-sparse workspace sweeps (Sec. 7.2): `live_k` of the K
+    coordinates of the contracted index are non-empty (drawn uniformly, distinct); each of them
+    has `per_k` entries at distinct uniform positions in A (rows i) and in B (columns j).
+    Returns (At, B): At is A by its rows k (K x I, CSR), B is K x J (CSR); values uniform in [-1,1]."""
+    rng = _rng(seed)
+    live = np.sort(rng.choice(K, size=live_k, replace=False))
+
+    def side(width, stream_seed):
+        r = _rng(stream_seed)
+        n = min(per_k, width)
+        crd = np.empty((live_k, n), dtype=np.int32)
+        for x in range(live_k):
+            crd[x] = np.sort(r.choice(width, size=n, replace=False))
+        counts = np.zeros(K, dtype=np.int64)
+        counts[live] = n
+        pos = np.zeros(K + 1, dtype=np.int64)
+        np.cumsum(counts, out=pos[1:])
+        return CSR(K, width, pos, crd.reshape(-1), _values(r, live_k * n, -1.0, 1.0, dtype))
+
+    return side(I, seed * 7919 + 1), side(J, seed * 7919 + 2)
+
+
 def config_inputs(name: str, seed: int = 1, reduced: bool = False) -> dict:
     """Operands of one benchmark configuration.
 
