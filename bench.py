@@ -7,9 +7,10 @@ operand set already resident in HBM.  Default workload: the power-law configurat
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
-N > 1 (under torchrun): every rank runs its own seeded problem of the same shape (output rows
-are independent, so ranks share nothing on the data path); value = all ranks' flops over the
-slowest rank's device time.
+N > 1 (under torchrun): ONE seeded problem; every rank takes a contiguous block of A's rows,
+balanced on the per-row product counts the device computes, with B replicated (output rows are
+independent, so the only exchange is an all-gather of the ranks' output sizes); value = the
+whole problem's flops over the slowest rank's device time ("scaling": "strong").
 """
 from __future__ import annotations
 
@@ -189,14 +190,24 @@ def measure(workload, args, dev, rank, world, dist, e2e=True, cpu_baseline=True)
     from workloads import config_inputs
 
     WORKLOAD_TEXT.setdefault(workload, f"{workload} (same recipe as the named configuration, other size), fp64")
-    cfg = config_inputs(workload, seed=args.seed + rank)
-    is_ttm = cfg["kind"] == "ttm"
+    is_ttm = workload.startswith("ttm")
+    # N > 1, matrix form: ONE seeded problem; every rank takes a block of A's rows, balanced on the
+    # per-row product counts, with B replicated (output rows are independent).  The 3-tensor form
+    # keeps one problem per rank.
+    sharded = world > 1 and not is_ttm
+    cfg = config_inputs(workload, seed=args.seed + (0 if sharded else rank))
     T3 = cfg["A"] if is_ttm else None           # the CSF operand of the 3-tensor form
     # the 3-tensor form works on the (i,j) fibres as rows: sizes, bytes and the oracle sample use that matrix
     A, B = (T3.fibres_as_csr() if is_ttm else cfg["A"]), cfg["B"]
     V = 8 if cfg["dtype"] == np.float64 else 4
     vt = torch.float64 if V == 8 else torch.float32
     ctx = api.Context(dev)
+    row_block = None
+    if sharded:
+        from paper_2404_04541_b200 import dist as spd
+        bounds = spd.partition_rows(spd.row_products_cuda(ctx)(A, B), world)
+        row_block = (int(bounds[rank]), int(bounds[rank + 1]))
+        A = A.row_block(*row_block)
     options = {}
     for kv in args.opt:
         name, value = kv.split("=", 1)
@@ -221,10 +232,14 @@ def measure(workload, args, dev, rank, world, dist, e2e=True, cpu_baseline=True)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)       # > L2 (126 MB)
     result = {}
 
+    nnz_all = torch.zeros(world, dtype=torch.int64, device=dev)
+
     def step():
         cc, st = symbolic(plan, dA, dB)
         result["C"] = numeric(plan, cc, st, crd=crd, val=val)
         result["c"], result["state"] = cc, st
+        if sharded:                                  # the one exchange: every rank's output size, to place its row pointers
+            dist.all_gather_into_tensor(nnz_all, torch.tensor([cc.n[last]], dtype=torch.int64, device=dev))
 
     for _ in range(args.warmup):
         step()
@@ -323,11 +338,13 @@ def measure(workload, args, dev, rank, world, dist, e2e=True, cpu_baseline=True)
                 "ceiling": "same traversal and gathers, workspace stripped (spws_gather_ceiling)"}
 
     out = {"value": value, "ms_per_step": ms_per_step, "ms_min": ms_min, "ms_median": ms_median,
+           "scaling": "strong" if sharded else "weak",
            "dtype": "f64" if V == 8 else "f32",
            "config": {"workload": WORKLOAD_TEXT[workload], "name": workload, "policy": args.policy, "options": options,
                       "seed": args.seed, "rows": int(A.nrows), "nnzA": int(A.nnz), "products": int(products),
                       "nnzC": int(nnzC), "l2": "512 MiB buffer written between timed steps",
-                      "timed": "spws_symbolic + spws_numeric; C buffers preallocated",
+                      "timed": "spws_symbolic + spws_numeric; C buffers preallocated" + ("; all-gather of the ranks' output sizes" if sharded else ""),
+                      **({"sharding": f"rows {row_block[0]}..{row_block[1]} of one problem on rank {rank}; B replicated"} if sharded else {}),
                       **({"rows_are": "the (i,j) fibres of A"} if is_ttm else {})},
            "effective_gbs": eff_gbs, "algorithmic_bytes_per_step": abytes,
            "hbm_frac_nominal_8tbs": eff_gbs / NOMINAL_HBM_GBS, "hbm_frac_measured": eff_gbs / peak,
@@ -554,7 +571,7 @@ def main():
 
     m = measure(args.workload, args, dev, rank, world, dist, e2e=not args.no_e2e, cpu_baseline=not args.no_cpu_baseline)
     line = {"metric": METRIC, "value": m.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": m.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": m.pop("ms_per_step"), "higher_is_better": True, "scaling": m.pop("scaling"),
             "vs_baseline": None, "dtype": m.pop("dtype"), "data": "synthetic", "config": m.pop("config")}
     line.update(m)
     # the other configuration with a roofline target, same protocol (default run only)

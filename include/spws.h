@@ -70,9 +70,14 @@ typedef enum { SPWS_CSR = 0, SPWS_CSF3 = 1 } spws_format_t;
 typedef enum { SPWS_F32 = 0, SPWS_F64 = 1 } spws_dtype_t;
 /* Workspace policy.  DENSE: value array + occupancy bitmap along the last index (Gustavson's
  * workspace, Table 2), held in shared memory.  SPARSE_ISM: insert-sort-merge with the
- * coordinate-sort policy (Algorithm 1, Sec. 5.2).  AUTO: chosen per row bin from the product
- * count and the column span.  The policy changes the route, never the result. */
-typedef enum { SPWS_DENSE = 0, SPWS_SPARSE_ISM = 1, SPWS_AUTO = 2 } spws_policy_t;
+ * coordinate-sort policy (Algorithm 1, Sec. 5.2).  HASH: insert-sort-merge with the reduction at
+ * insert time (Sec. 4.3; the Bucket / Hash policies of Sec. 5.2): products are deduplicated into an
+ * open-addressing table in shared memory and only the distinct coordinates are sorted; rows with
+ * more than 4096 products take the global-memory ISM.  AUTO: chosen per row bin from the product
+ * count and the column span.  The policy changes the route, never the result: the structure is
+ * identical under every policy; values agree to rounding (routes that add with atomics sum in an
+ * order that can differ from run to run). */
+typedef enum { SPWS_DENSE = 0, SPWS_SPARSE_ISM = 1, SPWS_AUTO = 2, SPWS_HASH = 3 } spws_policy_t;
 
 /* A tensor stored level by level.  Level l of a CSR matrix: l = 0 is Dense (pos[0], crd[0] unused,
  * n[0] = dims[0]); l = 1 is Compressed: pos[1] has dims[0]+1 entries, crd[1] has n[1] = nnz.
@@ -122,14 +127,14 @@ typedef struct {
     int64_t products;         /* intermediate products = sum of the per-row upper bounds          */
     int64_t nnz;              /* stored entries of C                                              */
     int64_t max_row_products;
-    int64_t rows_per_class[8];/* empty, ISM-register, ISM-shared(small), ISM-shared, dense-warp,
-                                 dense-CTA(hub), dense-CTA, ISM-global                            */
+    int64_t rows_per_class[10];/* empty, ISM-register, ISM-shared(small), ISM-shared, dense-warp,
+                                 dense-CTA(hub), dense-CTA, ISM-global, hash(small), hash         */
     int64_t dense_units;      /* CTA work units (row, share of its A entries) of the dense numeric
                                  pass                                                               */
     int32_t device_status;    /* last status word read back from the device                      */
     int32_t reserved;
-    int64_t products_per_class[8];
-    int64_t nnz_per_class[8];
+    int64_t products_per_class[10];
+    int64_t nnz_per_class[10];
     int32_t launches_symbolic; /* kernels enqueued by the last spws_symbolic / spws_numeric       */
     int32_t launches_numeric;
     int64_t dense_warp_rows;  /* dense rows the warp-per-row numeric kernel takes ...             */
@@ -140,7 +145,7 @@ typedef struct {
 
 /* Kernel groups timed by spws_set_profiling (index into the array spws_get_timings fills). */
 enum {
-    SPWS_T_SYM_BOUNDS = 0,    /* per-row upper bound, span and class                               */
+    SPWS_T_SYM_BOUNDS = 0,    /* per-row upper bound, span and class; word lists of long B rows    */
     SPWS_T_SYM_BIN = 1,       /* binning + dense work units                                        */
     SPWS_T_SYM_ISM_REG = 2,
     SPWS_T_SYM_ISM_SMEM_S = 3,
@@ -148,19 +153,21 @@ enum {
     SPWS_T_SYM_DENSE_WARP = 5,
     SPWS_T_SYM_DENSE_CTA = 6,
     SPWS_T_SYM_ISM_GLOBAL = 7,
-    SPWS_T_SYM_SCAN = 8,      /* exclusive scan, numeric routing of dense rows (+ CSF level
+    SPWS_T_SYM_HASH = 8,
+    SPWS_T_SYM_SCAN = 9,      /* exclusive scan, numeric routing of dense rows (+ CSF level
                                  rebuild for the 3-tensor form)                                    */
-    SPWS_T_NUM_ISM_REG = 9,
-    SPWS_T_NUM_ISM_SMEM_S = 10,
-    SPWS_T_NUM_ISM_SMEM = 11,
-    SPWS_T_NUM_DENSE_WARP = 12,
-    SPWS_T_NUM_DENSE_EMIT = 13, /* coordinates of the CTA dense rows; clears the value segments
+    SPWS_T_NUM_ISM_REG = 10,
+    SPWS_T_NUM_ISM_SMEM_S = 11,
+    SPWS_T_NUM_ISM_SMEM = 12,
+    SPWS_T_NUM_DENSE_WARP = 13,
+    SPWS_T_NUM_DENSE_EMIT = 14, /* coordinates of the CTA dense rows; clears the value segments
                                  that several work units add into                                  */
-    SPWS_T_NUM_DENSE_CTA = 14,
-    SPWS_T_NUM_ISM_GLOBAL = 15,
-    SPWS_T_CEIL_DENSE_WARP = 16, /* spws_gather_ceiling: the warp-per-row dense rows ...             */
-    SPWS_T_CEIL_DENSE_CTA = 17,  /* ... and the CTA-unit dense rows                                   */
-    SPWS_T_COUNT = 18
+    SPWS_T_NUM_DENSE_CTA = 15,
+    SPWS_T_NUM_ISM_GLOBAL = 16,
+    SPWS_T_NUM_HASH = 17,
+    SPWS_T_CEIL_DENSE_WARP = 18, /* spws_gather_ceiling: the warp-per-row dense rows ...             */
+    SPWS_T_CEIL_DENSE_CTA = 19,  /* ... and the CTA-unit dense rows                                   */
+    SPWS_T_COUNT = 20
 };
 
 spws_status_t spws_create(spws_handle_t* handle);
@@ -187,7 +194,8 @@ spws_status_t spws_plan_destroy(spws_plan_t plan);
 spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3], int* kind);
 
 /* Upper bound of the scratch bytes spws_symbolic + spws_numeric need for these operands (reads
- * only dims and n[] of A and B; host-side, launches nothing -- except for the outer-product form,
+ * only dims and n[] of A and B; host-side, launches nothing; spws_workspace_size_exact gives the
+ * size actually used -- except for the outer-product form,
  * whose workspace is sized by the number of products: there the call needs A's and B's pos arrays
  * on the device, counts the products with one kernel on the plan's stream and synchronises).  It always suffices; the largest
  * part is room for one occupancy bitmap per row (rows x min(columns, dense_max_span) / 8 bytes),
@@ -196,6 +204,21 @@ spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3
  * 256-byte alignment is required of the scratch pointer. */
 spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
                                   size_t* bytes);
+
+/* The scratch bytes spws_symbolic + spws_numeric really use for these operands, found by running
+ * the first two steps of the symbolic pass (per-row product bound and span, binning; Sec. 5.4's
+ * "balance workloads" needs them anyway): the fixed tables, the occupancy bitmaps of exactly the
+ * rows routed to the dense workspace over exactly their spans, and one all-array slot per CTA of
+ * the global-memory ISM.  Two steps: with scratch = NULL the call writes to *bytes the size of the
+ * buffer it needs itself (host only, no launch); with such a buffer (DEVICE, 256-byte aligned) it
+ * runs the two kernels on the plan's stream, synchronises and writes the exact size.
+ * `row_products` (DEVICE, int64, one entry per output row / input fibre; may be NULL) receives the
+ * per-row product counts, which a caller that shards rows over devices balances on.  A buffer of
+ * the returned size suffices for both passes; the call overwrites what an earlier symbolic pass
+ * left in `scratch`. */
+spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                                        void* scratch, size_t scratch_bytes, size_t* bytes,
+                                        int64_t* row_products);
 
 /* Symbolic pass.  C->pos[] must be allocated by the caller: CSR: pos[1] with dims[0]+1 entries;
  * CSF3: pos[0] (2), crd[0] (A->n[0]), pos[1] (A->n[0]+1), crd[1] (A->n[1]), pos[2] (A->n[1]+1),

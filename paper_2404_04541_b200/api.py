@@ -81,6 +81,21 @@ class Context:
     def plan(self, expr, fmts, dtype, policy="auto", **options) -> B_.Plan:
         return B_.Plan(self.handle, expr, fmts, dtype, policy, **options)
 
+    def exact_scratch_bytes(self, plan: B_.Plan, a: B_.TensorArrays, b: B_.TensorArrays, row_products: torch.Tensor | None = None) -> int:
+        """Bytes the two passes really use for these operands (one sizing pass on the device; the
+        result is remembered per plan and operand pair).  `row_products` (int64, one per row)
+        receives the per-row product counts when given."""
+        ptrs = lambda t: tuple(x.data_ptr() for x in list(t.pos) + list(t.crd) if x is not None)
+        key = (ptrs(a), ptrs(b), tuple(a.n), tuple(b.n))
+        cache = plan.__dict__.setdefault("_exact_bytes", {})
+        if key in cache and row_products is None:
+            return cache[key]
+        own = plan.workspace_size_exact(a, b)
+        sc = self.scratch(own)
+        cache[key] = plan.workspace_size_exact(a, b, self._aligned_ptr(sc), own,
+                                               row_products.data_ptr() if row_products is not None else None)
+        return cache[key]
+
     def scratch(self, nbytes: int) -> torch.Tensor:
         if self._scratch is None or self._scratch.numel() < nbytes:
             self._scratch = None
@@ -94,7 +109,7 @@ class Context:
     # ------------------------------------------------------------------ SpGEMM
     def spgemm_symbolic(self, plan: B_.Plan, A: DeviceCSR, B: DeviceCSR):
         a, b = A.arrays(), B.arrays()
-        nbytes = plan.workspace_size(a, b)
+        nbytes = self.exact_scratch_bytes(plan, a, b)
         sc = self.scratch(nbytes)
         pos = torch.empty(A.nrows + 1, dtype=torch.int64, device=self.device)
         c = B_.csr_arrays(A.nrows, B.ncols, pos, None, None)
@@ -163,7 +178,7 @@ class Context:
         """Symbolic pass of the 3-tensor form: allocates C's upper levels (bounded by A's) and returns
         (C arrays with sizes filled in, state for ttm_numeric)."""
         a, b = A.arrays(), B.arrays()
-        nbytes = plan.workspace_size(a, b)
+        nbytes = self.exact_scratch_bytes(plan, a, b)
         sc = self.scratch(nbytes)
         n_i, n_ij = a.n[0], a.n[1]
         i64, i32, dev = torch.int64, torch.int32, self.device

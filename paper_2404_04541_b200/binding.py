@@ -28,19 +28,20 @@ SPWS_BAD_SEQUENCE = 10
 # enums
 SPWS_CSR, SPWS_CSF3 = 0, 1
 SPWS_F32, SPWS_F64 = 0, 1
-SPWS_DENSE, SPWS_SPARSE_ISM, SPWS_AUTO = 0, 1, 2
-POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPARSE_ISM, "auto": SPWS_AUTO}
+SPWS_DENSE, SPWS_SPARSE_ISM, SPWS_AUTO, SPWS_HASH = 0, 1, 2, 3
+POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPARSE_ISM, "auto": SPWS_AUTO, "hash": SPWS_HASH}
 
 EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create", "spws_plan_destroy",
-           "spws_check_expression", "spws_workspace_size", "spws_symbolic", "spws_numeric",
+           "spws_check_expression", "spws_workspace_size", "spws_workspace_size_exact", "spws_symbolic", "spws_numeric",
            "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host", "spws_gather_ceiling",
            "spws_row_pointer_static", "spws_status_string")
 STATIC_MAX_ROWS = 16777216
 TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense_warp",
-                 "sym_dense_cta", "sym_ism_global", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem",
-                 "num_dense_warp", "num_dense_emit", "num_dense_cta", "num_ism_global", "ceil_dense_warp", "ceil_dense_cta")
+                 "sym_dense_cta", "sym_ism_global", "sym_hash", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem",
+                 "num_dense_warp", "num_dense_emit", "num_dense_cta", "num_ism_global", "num_hash", "ceil_dense_warp",
+                 "ceil_dense_cta")
 # class index of each per-class kernel group (rows_per_class / products_per_class / nnz_per_class)
-CLASS_NAMES = ("empty", "ism_reg", "ism_smem_s", "ism_smem", "dense_warp", "dense_hub", "dense_cta", "ism_global")
+CLASS_NAMES = ("empty", "ism_reg", "ism_smem_s", "ism_smem", "dense_warp", "dense_hub", "dense_cta", "ism_global", "hash_s", "hash")
 
 
 class spws_tensor_t(ctypes.Structure):
@@ -58,9 +59,9 @@ class spws_options_t(ctypes.Structure):
 
 class spws_stats_t(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int64), ("products", ctypes.c_int64), ("nnz", ctypes.c_int64),
-                ("max_row_products", ctypes.c_int64), ("rows_per_class", ctypes.c_int64 * 8),
+                ("max_row_products", ctypes.c_int64), ("rows_per_class", ctypes.c_int64 * 10),
                 ("dense_units", ctypes.c_int64), ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32),
-                ("products_per_class", ctypes.c_int64 * 8), ("nnz_per_class", ctypes.c_int64 * 8),
+                ("products_per_class", ctypes.c_int64 * 10), ("nnz_per_class", ctypes.c_int64 * 10),
                 ("launches_symbolic", ctypes.c_int32), ("launches_numeric", ctypes.c_int32),
                 ("dense_warp_rows", ctypes.c_int64), ("dense_warp_products", ctypes.c_int64),
                 ("dense_warp_nnz", ctypes.c_int64), ("bitmap_bytes", ctypes.c_int64)]
@@ -92,6 +93,7 @@ def lib():
         L.spws_plan_destroy.argtypes = [vp]
         L.spws_check_expression.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.spws_workspace_size.argtypes = [vp, T, T, ctypes.POINTER(sz)]
+        L.spws_workspace_size_exact.argtypes = [vp, T, T, vp, sz, ctypes.POINTER(sz), vp]
         L.spws_symbolic.argtypes = [vp, T, T, T, vp, sz, ctypes.POINTER(ctypes.c_int64)]
         L.spws_numeric.argtypes = [vp, T, T, T, vp, sz]
         L.spws_gather_ceiling.argtypes = [vp, T, T, T, vp, sz, vp, vp]
@@ -221,6 +223,16 @@ class Plan:
         a, b = A.c_struct(), B.c_struct()
         _check(lib().spws_workspace_size(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(out)),
                "spws_workspace_size")
+        return int(out.value)
+
+    def workspace_size_exact(self, A: TensorArrays, B: TensorArrays, scratch_ptr: int | None = None, scratch_bytes: int = 0,
+                             row_products_ptr: int | None = None) -> int:
+        """spws_workspace_size_exact: without a scratch pointer, the bytes the sizing call itself
+        needs; with one, the bytes both passes really use (runs two kernels, synchronises)."""
+        out = ctypes.c_size_t(0)
+        a, b = A.c_struct(), B.c_struct()
+        _check(lib().spws_workspace_size_exact(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(scratch_ptr), scratch_bytes,
+                                               ctypes.byref(out), ctypes.c_void_p(row_products_ptr)), "spws_workspace_size_exact")
         return int(out.value)
 
     def symbolic(self, A, B, C, scratch_ptr: int, scratch_bytes: int):

@@ -8,7 +8,7 @@ namespace spws {
 typedef long long i64;
 typedef unsigned long long u64;
 
-constexpr int NCLASS = 10;
+constexpr int NCLASS = 12;
 // Row classes = the workspace a row (or (i,j) fibre) is routed to in the symbolic pass.
 enum RowClass : int {
     CLS_EMPTY = 0,      // no intermediate product
@@ -20,14 +20,20 @@ enum RowClass : int {
     CLS_DENSE_WARP = 6, // dense workspace (occupancy bitmap), one warp per row
     CLS_DENSE_HUB = 7,  // dense workspace, one CTA per row, heaviest rows (scheduled first)
     CLS_DENSE_CTA = 8,  // dense workspace, one CTA per row
-    CLS_ISM_GLOBAL = 9  // accumulation array in shared memory, all array in global memory
+    CLS_ISM_GLOBAL = 9, // accumulation array in shared memory, all array in global memory
+    CLS_HASH_S = 10,    // hash table in shared memory (reduction at insert time), small CTA
+    CLS_HASH = 11       // hash table in shared memory, full CTA
 };
 constexpr int NUM_SLOT = 16;   // work_counter[cls] in the symbolic pass, work_counter[NUM_SLOT + cls] in the numeric pass
-constexpr int CEIL_SLOT = 20;  // work_counter[CEIL_SLOT + cls] in the gather-only (iteration-only) kernels
-constexpr int EMIT_SLOT = 30;  // work_counter slot of the coordinate emission of the CTA dense route
-constexpr int BW_SLOT = 31;    // work_counter slot of the word-list build
+constexpr int CEIL_SLOT = 32;  // work_counter[CEIL_SLOT + cls] in the gather-only (iteration-only) kernels
+constexpr int EMIT_SLOT = 48;  // work_counter slot of the coordinate emission of the CTA dense route
+constexpr int BW_SLOT = 49;    // work_counter slot of the word-list build
+constexpr int N_WORK_COUNTERS = 64;
 // index of a class in the public statistics (the three register classes are reported as one)
 __host__ __device__ inline int public_class(int cls) { return cls == 0 ? 0 : (cls <= 3 ? 1 : cls - 2); }
+constexpr int N_PUBLIC_CLASS = 10;
+constexpr int HASH_SMALL_CAP = 1024;       // products of a row the small / the full hash workspace takes
+constexpr int HASH_CAP = 4096;
 
 // Capacities fixed at compile time.
 constexpr int DENSE_WARP_BM_WORDS = 1024;  // bitmap words a warp-per-row workspace may span (32768 columns)
@@ -65,7 +71,7 @@ struct DevCtl {
     int n_long;             // B rows with at least BW_MIN_LEN entries (candidates for a word list)
     int class_count[NCLASS];
     int class_cursor[NCLASS];
-    int work_counter[32];   // dynamic work distribution; cleared before each pass
+    int work_counter[N_WORK_COUNTERS];   // dynamic work distribution; cleared before each pass
     i64 class_products[NCLASS];
     i64 class_nnz[NCLASS];
     i64 dense_warp_products, dense_warp_nnz;   // share of the dense rows the warp numeric kernel takes
@@ -218,6 +224,8 @@ cudaError_t launch_dense_num_cta(const LaunchCtx& c, int phase, int n_units_host
                                  u64* chk_idx = nullptr, double* chk_val = nullptr);
 cudaError_t launch_ism_global(const LaunchCtx& c, bool numeric, int n_host, const Csr& A, const Csr& B,
                               const i64* rowptr, int* Ccrd, void* Cval);
+cudaError_t launch_hash(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B, const i64* rowptr,
+                        int* Ccrd, void* Cval);
 
 // outer.cu: second-order workspaces of the outer-product form
 cudaError_t launch_outer_counts(const LaunchCtx& c, const Csr& At, const Csr& B, int* cnt);

@@ -62,6 +62,11 @@ __device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const Cl
         if (ub <= prm.smem_cap) return CLS_ISM_SMEM;
         return CLS_ISM_GLOBAL;
     }
+    if (prm.policy == 3) {                       // hash forced
+        if (ub <= HASH_SMALL_CAP) return CLS_HASH_S;
+        if (ub <= HASH_CAP) return CLS_HASH;
+        return CLS_ISM_GLOBAL;
+    }
     // auto: few products -> sort them in registers; a bitmap that is small next to the work ->
     // dense; mid-size rows -> shared-memory ISM; long rows -> dense; otherwise global ISM.
     if (reg_ok) return reg_cls;

@@ -170,7 +170,7 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, 
     }
     // word lists of long B rows (dense routes): one 8-byte slot per entry of B, used only at the
     // positions of rows with at least BW_MIN_LEN entries
-    if (p->policy != SPWS_SPARSE_ISM && nnzB >= BW_MIN_LEN && nnzB <= BW_MAX_NNZ) {
+    if (p->policy != SPWS_SPARSE_ISM && p->policy != SPWS_HASH && nnzB >= BW_MIN_LEN && nnzB <= BW_MAX_NNZ) {
         L.bw_long_cap = (int)(nnzB / BW_MIN_LEN + 1);
         L.bw_long = take(4 * (size_t)L.bw_long_cap);
         L.bw = take(8 * (size_t)nnzB);
@@ -184,15 +184,19 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, 
 // for a few slots of min(ncols, 2^22) components for the global-memory ISM
 size_t rest_reserve(const spws_plan_s* p, int64_t m, int64_t ncols) {
     size_t bytes = 0;
-    if (p->policy != SPWS_SPARSE_ISM) {
+    if (p->policy != SPWS_SPARSE_ISM && p->policy != SPWS_HASH) {
         const int64_t span_cap = ncols < p->opt.dense_max_span ? ncols : p->opt.dense_max_span;
         const size_t nw = (size_t)((span_cap + 31) / 32 + 1);
         bytes += align256((size_t)m * ((nw + (nw + 31) / 32 + 3) & ~(size_t)3) * 4);
     }
     if (p->policy != SPWS_DENSE) {
+        // global-memory ISM: eight slots of min(ncols, 2^22) components, and never less than the one
+        // slot a row over all ncols columns needs in the numeric pass
         const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
         const size_t comp = 4 + (p->is_f64 ? 8 : 4);
-        bytes += align256(2 * (size_t)((elems + 63) & ~63ll) * comp) * 8;
+        const size_t eight = align256(2 * (size_t)((elems + 63) & ~63ll) * comp) * 8;
+        const size_t one_full = align256(2 * (size_t)((ncols + 63) & ~63ll) * comp);
+        bytes += eight > one_full ? eight : one_full;
     }
     return bytes;
 }
@@ -266,7 +270,7 @@ LaunchCtx make_ctx(const spws_plan_s* p, char* scratch, size_t scratch_bytes, co
     c.prm.unit_cap = L.unit_cap;
     c.rest = scratch + L.rest;
     c.rest_bytes = scratch_bytes > L.rest ? scratch_bytes - L.rest : 0;
-    c.prm.bm_arena_words = p->policy == SPWS_SPARSE_ISM ? 0 : c.rest_bytes / 4;
+    c.prm.bm_arena_words = (p->policy == SPWS_SPARSE_ISM || p->policy == SPWS_HASH) ? 0 : c.rest_bytes / 4;
     c.dense_smem_words = L.dense_smem_words;
     c.tab.ub = reinterpret_cast<i64*>(scratch + L.ub);
     c.tab.cnt = reinterpret_cast<int*>(scratch + L.cnt);
@@ -384,7 +388,7 @@ bool outer_wants_dense(const spws_plan_s* p, int64_t I, int64_t J, int64_t P, si
         if (!fits) *st = SPWS_WORKSPACE_TOO_LARGE;
         return true;
     }
-    if (p->policy == SPWS_SPARSE_ISM) return false;
+    if (p->policy == SPWS_SPARSE_ISM || p->policy == SPWS_HASH) return false;
     return fits && (double)P * 16.0 >= (double)I * (double)J;
 }
 
@@ -544,7 +548,7 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
                                spws_plan_t* plan) {
     if (!handle || !expr || !fmts || !plan) return SPWS_INVALID_ARGUMENT;
     if (value_type != SPWS_F32 && value_type != SPWS_F64) return SPWS_INVALID_ARGUMENT;
-    if (policy != SPWS_DENSE && policy != SPWS_SPARSE_ISM && policy != SPWS_AUTO) return SPWS_INVALID_ARGUMENT;
+    if (policy != SPWS_DENSE && policy != SPWS_SPARSE_ISM && policy != SPWS_AUTO && policy != SPWS_HASH) return SPWS_INVALID_ARGUMENT;
     for (int f = 0; f < 3; ++f)
         if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3) return SPWS_INVALID_ARGUMENT;
     const int kind = classify_expression(expr, fmts);
@@ -632,13 +636,53 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
         if ((st = outer_count_products(plan, S, &P)) != SPWS_OK) return st;
         const OuterLayout OL = make_outer_layout(plan, S.m, S.k, S.ncols, P);
         const size_t dense_ok = (double)S.m * (double)S.ncols <= 2.0e9 ? OL.dense_end : 0;     // a dense workspace beyond 2^31 cells is never offered
-        *bytes = plan->policy == SPWS_SPARSE_ISM ? OL.ism_end
+        *bytes = (plan->policy == SPWS_SPARSE_ISM || plan->policy == SPWS_HASH) ? OL.ism_end
                  : plan->policy == SPWS_DENSE ? OL.dense_end
                  : std::max(OL.ism_end, (double)P * 16.0 >= (double)S.m * (double)S.ncols ? dense_ok : (size_t)0);
         return SPWS_OK;
     }
     const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
     *bytes = L.fixed_end + rest_reserve(plan, S.m, S.ncols);
+    return SPWS_OK;
+}
+
+spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, void* scratch,
+                                        size_t scratch_bytes, size_t* bytes, int64_t* row_products) {
+    if (!plan || !bytes) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind == 2) return spws_workspace_size(plan, A, B, bytes);      // already sized from the product count
+    Shapes S{};
+    spws_status_t st = check_operands(plan, A, B, S, scratch != nullptr);
+    if (st != SPWS_OK) return st;
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    if (!scratch) {                             // first step of the protocol: what this call itself needs
+        *bytes = L.fixed_end;
+        return SPWS_OK;
+    }
+    if (reinterpret_cast<uintptr_t>(scratch) & 255) return SPWS_INVALID_ARGUMENT;
+    if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
+    plan->symbolic_ok = false;                  // the tables of an earlier symbolic pass are overwritten
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
+    c.prm.bm_arena_words = ~0ull >> 3;          // reserve without a limit: only the total is wanted
+    CUDA_TRY(cudaMemsetAsync(c.ctl, 0, sizeof(DevCtl), c.stream));
+    CUDA_TRY(launch_row_bounds(c, S.A, S.B, S.nnzA));
+    CUDA_TRY(launch_bin_rows(c, (int)S.m));
+    if (row_products && S.m > 0)
+        CUDA_TRY(cudaMemcpyAsync(row_products, c.tab.ub, 8 * (size_t)S.m, cudaMemcpyDeviceToDevice, c.stream));
+    CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, c.stream));
+    CUDA_TRY(cudaStreamSynchronize(c.stream));
+    const DevCtl& hc = *plan->host_ctl;
+    if (hc.status != 0 && hc.status != DEV_SCRATCH_TOO_SMALL) return from_dev_status(hc.status);
+    size_t need = L.fixed_end + align256((size_t)hc.bm_words_used * 4);
+    const int64_t n_global = hc.class_count[CLS_ISM_GLOBAL];
+    if (n_global > 0) {                         // one numeric slot per CTA the global-memory ISM launches
+        int64_t elems = hc.max_ub_global < S.ncols ? hc.max_ub_global : S.ncols;
+        elems = (elems + 63) & ~63ll;
+        const size_t comp = 4 + (plan->is_f64 ? 8 : 4);
+        const int64_t ctas = n_global < 2 * (int64_t)plan->h->sm_count ? n_global : 2 * (int64_t)plan->h->sm_count;
+        need += align256(2 * (size_t)elems * comp) * (size_t)ctas;
+    }
+    *bytes = need;
     return SPWS_OK;
 }
 
@@ -675,7 +719,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     // a3: exact count per row through the workspace of its class
     i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<i64*>(sc + L.rowptr_raw);
     if (S.m > 0) {
-        if (plan->policy != SPWS_DENSE) {
+        if (plan->policy != SPWS_DENSE && plan->policy != SPWS_HASH) {
             CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG8, -1, S.A, S.B, rowptr, nullptr, nullptr));
             CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG16, -1, S.A, S.B, rowptr, nullptr, nullptr));
             CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG, -1, S.A, S.B, rowptr, nullptr, nullptr));
@@ -685,7 +729,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
             CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, -1, S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_SMEM);
         }
-        if (plan->policy != SPWS_SPARSE_ISM) {
+        if (plan->policy != SPWS_SPARSE_ISM && plan->policy != SPWS_HASH) {
             CUDA_TRY(launch_dense_sym_warp(c, S.A, S.B));
             mark(plan, SPWS_T_SYM_DENSE_WARP);
             CUDA_TRY(launch_dense_sym_cta(c, S.A, S.B));
@@ -694,6 +738,11 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
         if (plan->policy != SPWS_DENSE) {
             CUDA_TRY(launch_ism_global(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_GLOBAL);
+        }
+        if (plan->policy == SPWS_HASH) {
+            CUDA_TRY(launch_hash(c, false, CLS_HASH_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            CUDA_TRY(launch_hash(c, false, CLS_HASH, -1, S.A, S.B, rowptr, nullptr, nullptr));
+            mark(plan, SPWS_T_SYM_HASH);
         }
     }
     // a4: exclusive scan into the row pointer
@@ -704,7 +753,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
                                     reinterpret_cast<int*>(sc + L.sflags), reinterpret_cast<i64*>(sc + L.spos),
                                     reinterpret_cast<i64*>(sc + L.block_sums), LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
     }
-    if (plan->policy != SPWS_SPARSE_ISM) CUDA_TRY(launch_dense_rebin(c, (int)S.m, rowptr));
+    if (plan->policy != SPWS_SPARSE_ISM && plan->policy != SPWS_HASH) CUDA_TRY(launch_dense_rebin(c, (int)S.m, rowptr));
     CUDA_TRY(launch_class_nnz(c, (int)S.m));
     mark(plan, SPWS_T_SYM_SCAN);
     CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
@@ -797,6 +846,11 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
         CUDA_TRY(launch_ism_global(c, true, (int)bins[CLS_ISM_GLOBAL], S.A, S.B, rowptr, crd, C->val));
         mark(plan, SPWS_T_NUM_ISM_GLOBAL);
     }
+    for (int cls = CLS_HASH_S; cls <= CLS_HASH; ++cls)
+        if (bins[cls] > 0) {
+            CUDA_TRY(launch_hash(c, true, cls, (int)bins[cls], S.A, S.B, rowptr, crd, C->val));
+            mark(plan, SPWS_T_NUM_HASH);
+        }
     plan->stats.launches_numeric = c.launches;
     return SPWS_OK;
 }

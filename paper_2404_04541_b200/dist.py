@@ -5,8 +5,9 @@ rows), so A is cut into contiguous row blocks, B is replicated, every rank runs 
 single-GPU path on its block, and the only exchange is an all-gather of each rank's output size
 to place its row-pointer slice.  No collective touches the data path.
 
-The local product is passed in as a callable so that the same code drives the CUDA path
-(`local_spgemm_cuda`) and, in CPU tests, a stand-in.
+The local product and the per-row product counts the partition balances on are passed in as
+callables, so that the same code drives the CUDA path (`local_spgemm_cuda`, `row_products_cuda`:
+the counts come from the symbolic pass's first kernel on the device) and, in CPU tests, stand-ins.
 """
 from __future__ import annotations
 
@@ -16,13 +17,6 @@ from typing import Callable
 import numpy as np
 import torch
 import torch.distributed as dist
-
-
-def row_weights(A_pos: np.ndarray, A_crd: np.ndarray, B_pos: np.ndarray) -> np.ndarray:
-    """Per-row product upper bound (the symbolic pass's first quantity), on the host."""
-    blen = np.diff(B_pos)
-    rows = np.repeat(np.arange(A_pos.shape[0] - 1), np.diff(A_pos))
-    return np.bincount(rows, weights=blen[A_crd], minlength=A_pos.shape[0] - 1).astype(np.int64)
 
 
 def partition_rows(weights: np.ndarray, world: int) -> np.ndarray:
@@ -46,15 +40,17 @@ class ShardResult:
     nnz_per_rank: np.ndarray
 
 
-def spgemm_sharded(A, B, local_spgemm: Callable, group=None) -> ShardResult:
+def spgemm_sharded(A, B, local_spgemm: Callable, row_products: Callable, group=None) -> ShardResult:
     """Each rank multiplies its row block of A by the replicated B.
 
     `A`, `B` are host CSR containers (attributes nrows, ncols, pos, crd, val and row_block);
-    `local_spgemm(A_block, B)` returns (pos, crd, val) numpy arrays of the block's product.
+    `local_spgemm(A_block, B)` returns (pos, crd, val) numpy arrays of the block's product;
+    `row_products(A, B)` returns the int64 product count of every row of A (every rank computes
+    the same partition from it).
     """
     world = dist.get_world_size(group)
     rank = dist.get_rank(group)
-    bounds = partition_rows(row_weights(A.pos, A.crd, B.pos), world)
+    bounds = partition_rows(np.asarray(row_products(A, B), dtype=np.int64), world)
     r0, r1 = int(bounds[rank]), int(bounds[rank + 1])
     pos, crd, val = local_spgemm(A.row_block(r0, r1), B)
     mine = torch.tensor([int(pos[-1])], dtype=torch.int64)
@@ -88,5 +84,26 @@ def local_spgemm_cuda(ctx, policy: str = "auto", **options) -> Callable:
         dB = api.DeviceCSR.from_host(B, device=ctx.device)
         C, _ = ctx.spgemm(dA, dB, policy=policy, **options)
         return C.pos.cpu().numpy(), C.crd.cpu().numpy(), C.val.cpu().numpy()
+
+    return run
+
+
+def row_products_cuda(ctx) -> Callable:
+    """Per-row product counts from the device: the upper-bound kernel of the symbolic pass, run by
+    the exact-sizing entry point."""
+    from . import api
+    from . import binding as B_
+
+    def run(A, B):
+        dA = api.DeviceCSR.from_host(A, device=ctx.device)
+        dB = api.DeviceCSR.from_host(B, device=ctx.device)
+        dt = np.float64 if dA.val.dtype == torch.float64 else np.float32
+        plan = ctx.plan(api.EXPR_SPGEMM, (B_.SPWS_CSR,) * 3, dt, "auto")
+        try:
+            ub = torch.empty(max(A.nrows, 1), dtype=torch.int64, device=ctx.device)
+            ctx.exact_scratch_bytes(plan, dA.arrays(), dB.arrays(), row_products=ub)
+            return ub[:A.nrows].cpu().numpy()
+        finally:
+            plan.close()
 
     return run

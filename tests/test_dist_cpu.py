@@ -30,7 +30,10 @@ def _worker(rank, world, port, out_dir):
         r = oracle.spgemm(Ab, B)
         return r.pos, r.crd, r.val
 
-    res = spd.spgemm_sharded(A, A, local)
+    def products(Am, Bm):                       # stand-in for the device's per-row product counts
+        return oracle.spgemm(Am, Bm).products
+
+    res = spd.spgemm_sharded(A, A, local, products)
     pos, crd, val = spd.gather_full(res, A.nrows)
     np.savez(os.path.join(out_dir, f"rank{rank}.npz"), pos=pos, crd=crd, val=val, r0=res.row_begin, r1=res.row_end,
              nnz=res.nnz_per_rank, first=res.pos[0])

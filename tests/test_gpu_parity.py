@@ -12,7 +12,7 @@ from workloads import (CSR, CSF3, config_inputs, random_csr, rmat_csr, stencil27
 
 pytestmark = pytest.mark.gpu
 
-POLICIES = ("dense", "ism", "auto")
+POLICIES = ("dense", "ism", "auto", "hash")
 # thresholds that force every route on small inputs
 SMALL_ROUTES = dict(ism_warp_cap=8, ism_cta_cap=64, dense_unit_outputs=64, fallback_cap=16)
 GLOBAL, DENSE = 7, slice(4, 7)          # indices into stats["rows_per_class"]
@@ -108,13 +108,15 @@ def _rows_with_products(targets, ncols, seed, dtype=np.float64):
 
 @pytest.mark.parametrize("policy", POLICIES)
 def test_capacity_boundaries(ctx, oracle_mod, policy):
-    targets = [1, 2, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 255, 256, 257, 1023, 1024, 1025,
+    targets = [1, 2, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025,
                4095, 4096, 4097, 8191, 8192, 8193, 20000]
     A, B = _rows_with_products(targets, 40000, 11)
     stats = check_spgemm(ctx, oracle_mod, A, B, policy)
     assert stats["max_row_products"] == 20000
-    if policy == "ism":
+    if policy in ("ism", "hash"):
         assert stats["rows_per_class"][GLOBAL] == 5                  # rows above the shared-memory capacity
+    if policy == "hash":                                             # the two table sizes split at 1024 products
+        assert stats["rows_per_class"][8] == 22 and stats["rows_per_class"][9] == 3
     A, B = _rows_with_products(targets[:17], 3000, 12)
     check_spgemm(ctx, oracle_mod, A, B, policy, **SMALL_ROUTES)
 
@@ -254,8 +256,8 @@ def test_randomized_shapes_policies_and_thresholds(ctx, oracle_mod, seed):
             A = random_csr(int(rng.integers(2, 30)), k, float(rng.uniform(0.2, 1.0)), s)
         A.val = A.val.astype(dtype)
         B.val = B.val.astype(dtype)
-        policy = POLICIES[int(rng.integers(0, 3))]
-        if policy == "ism" and kind in (1, 4):
+        policy = POLICIES[int(rng.integers(0, 4))]
+        if policy in ("ism", "hash") and kind in (1, 4):
             policy = "auto"                         # the global-memory ISM on very heavy rows is slow
         opts = {}
         if rng.random() < 0.5:
@@ -270,6 +272,29 @@ def test_randomized_shapes_policies_and_thresholds(ctx, oracle_mod, seed):
                 assert e.status == binding.SPWS_WORKSPACE_TOO_LARGE
         else:
             check_spgemm(ctx, oracle_mod, A, B, policy, **opts)
+
+
+def test_hash_workspace_load_factor_and_duplicates(ctx, oracle_mod):
+    """Rows at the hash workspace's limits: as many DISTINCT columns as a table may take (1024 and
+    4096 products, no two colliding: half-full tables), one product more (next table / next route),
+    and rows whose products nearly all fall on a few columns (long probe-free chains of adds)."""
+    rng = np.random.default_rng(17)
+    ncols = 1 << 20
+    rows, cols, arow, acol = [], [], [], []
+    for r, P in enumerate([1023, 1024, 1025, 4095, 4096, 4097]):
+        c = np.sort(rng.choice(ncols, size=P, replace=False))       # one B row per output row: all distinct
+        rows.append(np.full(P, r)); cols.append(c); arow.append(r); acol.append(r)
+    # rows 6..9: 64 B rows that all hold the same 50 columns -> 3200 products on 50 outputs
+    same = np.sort(rng.choice(ncols, size=50, replace=False))
+    for b in range(6, 70):
+        rows.append(np.full(50, b)); cols.append(same)
+    for r in range(6, 10):
+        arow += [r] * 64; acol += list(range(6, 70))
+    B = CSR.from_coo(70, ncols, np.concatenate(rows), np.concatenate(cols), rng.uniform(-1, 1, sum(len(c) for c in cols)))
+    A = CSR.from_coo(10, 70, arow, acol, rng.uniform(-1, 1, len(arow)))
+    stats = check_spgemm(ctx, oracle_mod, A, B, "hash")
+    assert stats["rows_per_class"][8] == 2 and stats["rows_per_class"][9] == 7 and stats["rows_per_class"][GLOBAL] == 1
+    assert stats["nnz"] == 1023 + 1024 + 1025 + 4095 + 4096 + 4097 + 4 * 50
 
 
 # ------------------------------------------------------------------ benchmark configurations
@@ -569,7 +594,7 @@ def _sharded_worker(rank, world, port, out_dir):
     dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
     A = rmat_csr(11, 12, 9)
     ctx = api.Context("cuda:0")
-    res = spd.spgemm_sharded(A, A, spd.local_spgemm_cuda(ctx))
+    res = spd.spgemm_sharded(A, A, spd.local_spgemm_cuda(ctx), spd.row_products_cuda(ctx))
     pos, crd, val = spd.gather_full(res, A.nrows)
     np.savez(os.path.join(out_dir, f"rank{rank}.npz"), pos=pos, crd=crd, val=val, r0=res.row_begin, r1=res.row_end)
     dist.destroy_process_group()
@@ -695,6 +720,51 @@ def test_execute_host_ttm_and_distinct_operands(ctx, oracle_mod):
     assert np.array_equal(cpos, mref.pos) and np.array_equal(ccrd, mref.crd)
     ok, _ = values_close(cval, mref.val_ref, mref.abs, 1e-12)
     assert ok.all()
+    plan.close()
+
+
+# ------------------------------------------------------------------ exact scratch sizing
+@pytest.mark.parametrize("policy", ["auto", "dense", "ism"])
+def test_exact_workspace_size_suffices_and_is_tight(ctx, oracle_mod, policy):
+    """spws_workspace_size_exact returns what both passes use: the result is right with exactly
+    that much scratch, a buffer 256 bytes shorter is refused, and the figure is far below the
+    host-side upper bound when rows are narrower than the matrix."""
+    import torch
+    from paper_2404_04541_b200 import api, binding
+    A = rmat_csr(12, 16, 9)
+    dA = api.DeviceCSR.from_host(A)
+    a = dA.arrays()
+    plan = ctx.plan(api.EXPR_SPGEMM, (binding.SPWS_CSR,) * 3, np.float64, policy, ism_cta_cap=256, fallback_cap=64)
+    upper = plan.workspace_size(a, a)
+    own = plan.workspace_size_exact(a, a)
+    assert 0 < own <= upper
+    buf = torch.empty(upper + 256, dtype=torch.uint8, device="cuda")
+    ptr = ctx._aligned_ptr(buf)
+    ub_dev = torch.empty(A.nrows, dtype=torch.int64, device="cuda")
+    exact = plan.workspace_size_exact(a, a, ptr, own, ub_dev.data_ptr())
+    assert own <= exact <= upper
+    lens = np.diff(A.pos)
+    ub = np.bincount(rows_of(A.pos), weights=lens[A.crd], minlength=A.nrows).astype(np.int64)
+    assert np.array_equal(ub_dev.cpu().numpy(), ub)
+    if policy != "ism":
+        assert exact < upper // 2
+    pos = torch.empty(A.nrows + 1, dtype=torch.int64, device="cuda")
+    c = binding.csr_arrays(A.nrows, A.ncols, pos, None, None)
+    plan.symbolic(a, a, c, ptr, exact)
+    ref = oracle_mod.spgemm(A, A, threads=4)
+    nnz = c.n[1]
+    assert nnz == ref.nnz
+    c.crd[1] = torch.empty(nnz, dtype=torch.int32, device="cuda")
+    c.val = torch.empty(nnz, dtype=torch.float64, device="cuda")
+    plan.numeric(a, a, c, ptr, exact)
+    stats = plan.get_stats()                                         # reports a device-side failure, if any
+    assert_matches((pos.cpu().numpy(), c.crd[1].cpu().numpy(), c.val.cpu().numpy()), ref, np.float64)
+    if policy != "ism" and exact > own:                              # bitmaps in use: a shorter arena cannot hold them
+        with pytest.raises(binding.SpwsError) as e:
+            plan.symbolic(a, a, c, ptr, exact - 256)
+            plan.numeric(a, a, c, ptr, exact - 256)
+            plan.get_stats()
+        assert e.value.status == binding.SPWS_SCRATCH_TOO_SMALL
     plan.close()
 
 
