@@ -5,6 +5,7 @@ this package.  It does not import the CUDA binding and the binding does not impo
 """
 from .oracle import (build, spgemm, ttm, ism_rowwise, ism_outer, hardware_threads,
                      SpgemmResult, TtmResult)
+from .higher import spttm, spttm_i, spmttkrp, CooResult
 
 __all__ = ["build", "spgemm", "ttm", "ism_rowwise", "ism_outer", "hardware_threads",
-           "SpgemmResult", "TtmResult"]
+           "SpgemmResult", "TtmResult", "spttm", "spttm_i", "spmttkrp", "CooResult"]

@@ -319,3 +319,70 @@ def test_generators_are_canonical_and_seeded():
     deg = np.diff(r.pos)
     assert deg.max() > 20 * np.median(deg[deg > 0])     # skewed degrees
     assert r.val.min() >= -1 and r.val.max() <= 1
+
+
+# ---------------------------------------------------------------- higher-order scatters (Sec. 7.3)
+def _dense_coo(d):
+    idx = np.argwhere(d != 0)
+    return idx, d[tuple(idx.T)]
+
+
+@pytest.mark.parametrize("dims,nnz,seed", [((4, 5, 6), 30, 1), ((7, 3, 8), 60, 2), ((9, 9, 9), 200, 3)])
+def test_higher_order_scatters_against_dense_einsum(oracle_mod, dims, nnz, seed):
+    """Each of the three expressions against numpy's einsum on dense copies: structure = where the
+    boolean einsum of the patterns is true, values within rounding of the dense result."""
+    from workloads import uniform_csf3
+    B = uniform_csf3(dims, nnz, seed)
+    Bd = B.to_dense()
+    L = 7
+    cases = [
+        ("spttm", oracle_mod.spttm, "kij,kl->ijl", [random_csr(dims[0], L, 0.4, seed + 10, empty_row_frac=0.2)]),
+        ("spttm_i", oracle_mod.spttm_i, "kij,il->kjl", [random_csr(dims[1], L, 0.4, seed + 11, empty_row_frac=0.2)]),
+        ("spmttkrp", oracle_mod.spmttkrp, "kli,kj,lj->ij", [random_csr(dims[0], L, 0.5, seed + 12), random_csr(dims[1], L, 0.5, seed + 13)]),
+    ]
+    for name, fn, spec, mats in cases:
+        res = fn(B, *mats)
+        dense = [m.to_dense() for m in mats]
+        want = np.einsum(spec, Bd, *dense)
+        pat = np.einsum(spec, (Bd != 0).astype(np.int64), *[(m.pattern_dense()).astype(np.int64) for m in mats]) > 0
+        got_pat = np.zeros(want.shape, dtype=bool)
+        got_pat[tuple(res.crd.T)] = True
+        assert np.array_equal(got_pat, pat), name
+        assert res.nnz == pat.sum(), name
+        # sorted lexicographically and unique
+        order = np.lexsort(tuple(res.crd.T[::-1]))
+        assert np.array_equal(order, np.arange(res.nnz)), name
+        scale = np.einsum(spec, np.abs(Bd), *[np.abs(x) for x in dense])
+        for v in (res.val, res.val_ref):
+            d = np.zeros(want.shape)
+            d[tuple(res.crd.T)] = v
+            assert (np.abs(d - want) <= 1e-13 * scale + 1e-300).all(), name
+        dab = np.zeros(want.shape)
+        dab[tuple(res.crd.T)] = res.abs
+        assert np.allclose(dab, scale * pat, rtol=1e-12, atol=0), name
+        assert res.products == int(np.einsum(spec, (Bd != 0).astype(np.int64), *[(m.pattern_dense()).astype(np.int64) for m in mats]).sum()), name
+
+
+def test_higher_order_hand_case(oracle_mod):
+    """B(k,i,j) with three entries, worked by hand.
+    SpTTM  A(i,j,l) = B(k,i,j) C(k,l):   B(0,1,2)=2, B(1,1,2)=3, B(1,0,0)=5; C(0,1)=10, C(1,1)=100, C(1,3)=7
+        -> A(0,0,1)=500, A(0,0,3)=35, A(1,2,1)=2*10+3*100=320, A(1,2,3)=21
+    SpTTM-I A(k,j,l) = B(k,i,j) C(i,l) with the same C read as C(i,l):
+        -> k=0: B(0,1,2)*C(1,:) -> A(0,2,1)=200, A(0,2,3)=14; k=1: B(1,0,0)*C(0,:) -> A(1,0,1)=50; B(1,1,2)*C(1,:) -> A(1,2,1)=300, A(1,2,3)=21
+    SpMTTKRP A(i,j) = B(k,l,i) C(k,j) D(l,j) with B read as B(k,l,i), D = C:
+        B(0,1,2): C(0,:)={1:10}, D(1,:)={1:100,3:7} -> A(2,1)=2*10*100=2000
+        B(1,0,0): C(1,:)={1:100,3:7}, D(0,:)={1:10} -> A(0,1)=5*100*10=5000
+        B(1,1,2): C(1,:), D(1,:) -> A(2,1)+=3*100*100=30000, A(2,3)=3*7*7=147
+    """
+    from workloads import CSF3
+    B = CSF3.from_coo((2, 2, 3), [0, 1, 1], [1, 1, 0], [2, 2, 0], [2.0, 3.0, 5.0])
+    C = CSR.from_coo(2, 4, [0, 1, 1], [1, 1, 3], [10.0, 100.0, 7.0])
+    r = oracle_mod.spttm(B, C)
+    assert r.crd.tolist() == [[0, 0, 1], [0, 0, 3], [1, 2, 1], [1, 2, 3]] and r.val.tolist() == [500.0, 35.0, 320.0, 21.0]
+    assert r.products == 5
+    r = oracle_mod.spttm_i(B, C)
+    assert r.crd.tolist() == [[0, 2, 1], [0, 2, 3], [1, 0, 1], [1, 2, 1], [1, 2, 3]]
+    assert r.val.tolist() == [200.0, 14.0, 50.0, 300.0, 21.0]
+    r = oracle_mod.spmttkrp(B, C, C)
+    assert r.crd.tolist() == [[0, 1], [2, 1], [2, 3]] and r.val.tolist() == [5000.0, 32000.0, 147.0]
+    assert r.products == 4
