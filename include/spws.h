@@ -8,6 +8,10 @@
  *   tensor-times-matrix      C(i,j,l) = sum_k A(i,j,k) * B(k,l)    A, C in CSF, B in CSR
  *   outer-product SpGEMM     C(i,j)   = sum_k A(k,i)   * B(k,j)    A, B, C in CSR, A stored by
  *                                                                  its rows k (dims = {K, I})
+ *   SpTTM (outer mode)       A(i,j,l) = sum_k B(k,i,j) * C(k,l)    B in CSF, C in CSR, A in COO
+ *   SpTTM-I                  A(k,j,l) = sum_i B(k,i,j) * C(i,l)    B in CSF, C in CSR, A in COO
+ *   SpMTTKRP                 A(i,j)   = sum_kl B(k,l,i) * C(k,j) * D(l,j)
+ *                                                                  B in CSF, C, D in CSR, A in COO
  *
  * following the paper's statement of the problem: an expression over named index variables
  * (Sec. 3), a level format per operand (Sec. 2.1, Fig. 4) and a workspace policy (Sec. 6.1:
@@ -21,7 +25,10 @@
  * and the all array in the scratch buffer) under SPWS_SPARSE_ISM, an I x J value array with
  * flags under SPWS_DENSE (SPWS_WORKSPACE_TOO_LARGE when the scratch given cannot hold it: the
  * paper's dense workspace running out of memory, Sec. 7.2), and under SPWS_AUTO the dense one
- * when it fits and the products number at least I*J/16.
+ * when it fits and the products number at least I*J/16.  The last three are the higher-order
+ * scatters of Sec. 7.3 (sparse output in coordinate form): their workspace is the sparse one on
+ * integer labels over all scattered output indices (third order for SpTTM); no dense workspace
+ * is offered for them (SPWS_DENSE: SPWS_WORKSPACE_TOO_LARGE at plan creation).
  *
  * Work is split in two device passes (Sec. 5.4: a symbolic phase that precomputes the output
  * structure removes the all array):
@@ -65,8 +72,11 @@ enum {
 typedef struct spws_handle_s* spws_handle_t;
 typedef struct spws_plan_s* spws_plan_t;
 
-/* Level formats (Sec. 2.1, Fig. 4).  CSR = {Dense, Compressed}; CSF3 = three Compressed levels. */
-typedef enum { SPWS_CSR = 0, SPWS_CSF3 = 1 } spws_format_t;
+/* Level formats (Sec. 2.1, Fig. 4).  CSR = {Dense, Compressed}; CSF3 = three Compressed levels;
+ * COO = coordinate form, the output format of the higher-order scatters (Sec. 7.3): one coordinate
+ * array per index (crd[0 .. order-1], each with n[0] entries, sorted lexicographically, no
+ * duplicates) and val; pos[] is not used. */
+typedef enum { SPWS_CSR = 0, SPWS_CSF3 = 1, SPWS_COO = 2 } spws_format_t;
 typedef enum { SPWS_F32 = 0, SPWS_F64 = 1 } spws_dtype_t;
 /* Workspace policy.  DENSE: value array + occupancy bitmap along the last index (Gustavson's
  * workspace, Table 2), held in shared memory.  SPARSE_ISM: insert-sort-merge with the
@@ -175,8 +185,9 @@ spws_status_t spws_destroy(spws_handle_t handle);
 /* `cuda_stream` is a cudaStream_t (NULL = the default stream). */
 spws_status_t spws_set_stream(spws_handle_t handle, void* cuda_stream);
 
-/* Parses `expr` -- "C(i,j)=A(i,k)*B(k,j)", "C(i,j,l)=A(i,j,k)*B(k,l)" or "C(i,j)=A(k,i)*B(k,j)" with
- * any tensor and index names and optional blanks -- and checks it against the formats: fmts[0] is the result's,
+/* Parses `expr` -- "C(i,j)=A(i,k)*B(k,j)", "C(i,j,l)=A(i,j,k)*B(k,l)", "C(i,j)=A(k,i)*B(k,j)",
+ * "A(i,j,l)=B(k,i,j)*C(k,l)" or "A(k,j,l)=B(k,i,j)*C(i,l)" with any tensor and index names and
+ * optional blanks -- and checks it against the formats: fmts[0] is the result's,
  * fmts[1], fmts[2] the operands' in the order written.  The expression is accepted when it has
  * exactly one reduction variable, the second operand is a CSR matrix indexed (reduction, last
  * output index), and the first operand's and result's level orders match the loop order
@@ -187,6 +198,21 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
                                spws_dtype_t value_type, spws_policy_t policy,
                                const spws_options_t* options /* may be NULL */, spws_plan_t* plan);
 spws_status_t spws_plan_destroy(spws_plan_t plan);
+
+/* Three operands: "A(i,j) = B(k,l,i) * C(k,j) * D(l,j)" (SpMTTKRP with a sparse result, Sec. 7.3);
+ * fmts[0] is the result's format (SPWS_COO), fmts[1..3] the operands' (SPWS_CSF3, SPWS_CSR,
+ * SPWS_CSR).  Plans made here run through spws_workspace_size3 / spws_symbolic3 / spws_numeric3,
+ * which are the two-operand calls with the third operand added. */
+spws_status_t spws_plan_create3(spws_handle_t handle, const char* expr, const spws_format_t fmts[4],
+                                spws_dtype_t value_type, spws_policy_t policy,
+                                const spws_options_t* options /* may be NULL */, spws_plan_t* plan);
+spws_status_t spws_workspace_size3(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                                   const spws_tensor_t* D, size_t* bytes);
+spws_status_t spws_symbolic3(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                             const spws_tensor_t* D, spws_tensor_t* C, void* scratch, size_t scratch_bytes,
+                             int64_t* sizes_out);
+spws_status_t spws_numeric3(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
+                            const spws_tensor_t* D, spws_tensor_t* C, void* scratch, size_t scratch_bytes);
 
 /* The expression check of spws_plan_create on its own (host only, needs no device): the
  * classification of Sec. 2.2 applied to `expr` and `fmts`.  `kind` (may be NULL) receives 0 for
@@ -208,8 +234,8 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
 /* The scratch bytes spws_symbolic + spws_numeric really use for these operands, found by running
  * the first two steps of the symbolic pass (per-row product bound and span, binning; Sec. 5.4's
  * "balance workloads" needs them anyway): the fixed tables, the occupancy bitmaps of exactly the
- * rows routed to the dense workspace over exactly their spans, and one all-array slot per CTA of
- * the global-memory ISM.  Two steps: with scratch = NULL the call writes to *bytes the size of the
+ * rows routed to the dense workspace over exactly their spans, and up to eight all-array slots of
+ * the global-memory ISM sized for its largest row.  Two steps: with scratch = NULL the call writes to *bytes the size of the
  * buffer it needs itself (host only, no launch); with such a buffer (DEVICE, 256-byte aligned) it
  * runs the two kernels on the plan's stream, synchronises and writes the exact size.
  * `row_products` (DEVICE, int64, one entry per output row / input fibre; may be NULL) receives the
@@ -220,7 +246,10 @@ spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A
                                         void* scratch, size_t scratch_bytes, size_t* bytes,
                                         int64_t* row_products);
 
-/* Symbolic pass.  C->pos[] must be allocated by the caller: CSR: pos[1] with dims[0]+1 entries;
+/* Symbolic pass.  (For a COO result nothing needs to be allocated yet: sizes_out[0] / C->n[0]
+ * receive the number of entries; like the outer-product form, these forms size their workspace
+ * from the product count, which spws_workspace_size counts on the device.)
+ * C->pos[] must be allocated by the caller: CSR: pos[1] with dims[0]+1 entries;
  * CSF3: pos[0] (2), crd[0] (A->n[0]), pos[1] (A->n[0]+1), crd[1] (A->n[1]), pos[2] (A->n[1]+1),
  * i.e. the sizes of A's upper levels, which bound C's.  On return C->n[] holds the result sizes
  * and `sizes_out` (host, 3 entries, may be NULL) a copy.  Synchronises the stream once, to read

@@ -14,6 +14,9 @@ from . import binding as B_
 EXPR_SPGEMM = "C(i,j) = A(i,k) * B(k,j)"
 EXPR_TTM = "C(i,j,l) = A(i,j,k) * B(k,l)"
 EXPR_OUTER = "C(i,j) = A(k,i) * B(k,j)"
+EXPR_SPTTM = "A(i,j,l) = B(k,i,j) * C(k,l)"
+EXPR_SPTTM_I = "A(k,j,l) = B(k,i,j) * C(i,l)"
+EXPR_SPMTTKRP = "A(i,j) = B(k,l,i) * C(k,j) * D(l,j)"
 
 
 def _dev(a, dtype, device):
@@ -172,6 +175,36 @@ class Context:
         finally:
             if own:
                 plan.close()
+
+    # ------------------------------------------------------------------ higher-order scatters, COO result
+    def scatter_coo(self, expr: str, T: DeviceCSF3, C: DeviceCSR, D: DeviceCSR | None = None, policy="auto", **options):
+        """One of the higher-order scatters (EXPR_SPTTM, EXPR_SPTTM_I, EXPR_SPMTTKRP): CSF tensor
+        times one or two CSR matrices, sparse result in coordinate form.  Returns
+        (crd [nnz, order] int32, val [nnz], stats)."""
+        dt = np.float64 if T.val.dtype == torch.float64 else np.float32
+        fmts = (B_.SPWS_COO, B_.SPWS_CSF3, B_.SPWS_CSR) + ((B_.SPWS_CSR,) if D is not None else ())
+        plan = self.plan(expr, fmts, dt, policy, **options)
+        try:
+            t, c = T.arrays(), C.arrays()
+            d = D.arrays() if D is not None else None
+            nbytes = plan.workspace_size(t, c, d)
+            sc = self.scratch(nbytes)
+            if expr == EXPR_SPMTTKRP:
+                order, dims = 2, (T.dims[2], C.ncols, 0)
+            elif expr == EXPR_SPTTM:
+                order, dims = 3, (T.dims[1], T.dims[2], C.ncols)
+            else:
+                order, dims = 3, (T.dims[0], T.dims[2], C.ncols)
+            out = B_.TensorArrays(order, dims, [None, None, None], [None, None, None], None, [0, 0, 0])
+            nnz = plan.symbolic(t, c, out, self._aligned_ptr(sc), nbytes, D=d)[0]
+            crd = [torch.empty(nnz, dtype=torch.int32, device=self.device) for _ in range(order)]
+            out.crd = crd + [None] * (3 - order)
+            out.val = torch.empty(nnz, dtype=T.val.dtype, device=self.device)
+            out.n = [nnz, 0, 0]
+            plan.numeric(t, c, out, self._aligned_ptr(sc), nbytes, D=d)
+            return torch.stack(crd, dim=1) if nnz else torch.empty((0, order), dtype=torch.int32, device=self.device), out.val, plan.get_stats()
+        finally:
+            plan.close()
 
     # ------------------------------------------------------------------ TTM
     def ttm_symbolic(self, plan: B_.Plan, A: DeviceCSF3, B: DeviceCSR):

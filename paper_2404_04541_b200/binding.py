@@ -26,7 +26,7 @@ SPWS_INTERNAL_OVERFLOW = 8
 SPWS_OUTPUT_TOO_SMALL = 9
 SPWS_BAD_SEQUENCE = 10
 # enums
-SPWS_CSR, SPWS_CSF3 = 0, 1
+SPWS_CSR, SPWS_CSF3, SPWS_COO = 0, 1, 2
 SPWS_F32, SPWS_F64 = 0, 1
 SPWS_DENSE, SPWS_SPARSE_ISM, SPWS_AUTO, SPWS_HASH = 0, 1, 2, 3
 POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPARSE_ISM, "auto": SPWS_AUTO, "hash": SPWS_HASH}
@@ -34,7 +34,8 @@ POLICIES = {"dense": SPWS_DENSE, "ism": SPWS_SPARSE_ISM, "sparse_ism": SPWS_SPAR
 EXPORTS = ("spws_create", "spws_destroy", "spws_set_stream", "spws_plan_create", "spws_plan_destroy",
            "spws_check_expression", "spws_workspace_size", "spws_workspace_size_exact", "spws_symbolic", "spws_numeric",
            "spws_get_stats", "spws_set_profiling", "spws_get_timings", "spws_execute_host", "spws_gather_ceiling",
-           "spws_row_pointer_static", "spws_status_string")
+           "spws_row_pointer_static", "spws_status_string", "spws_plan_create3", "spws_workspace_size3", "spws_symbolic3",
+           "spws_numeric3")
 STATIC_MAX_ROWS = 16777216
 TIMING_GROUPS = ("sym_bounds", "sym_bin", "sym_ism_reg", "sym_ism_smem_s", "sym_ism_smem", "sym_dense_warp",
                  "sym_dense_cta", "sym_ism_global", "sym_hash", "sym_scan", "num_ism_reg", "num_ism_smem_s", "num_ism_smem",
@@ -90,6 +91,10 @@ def lib():
         L.spws_set_stream.argtypes = [vp, vp]
         L.spws_plan_create.argtypes = [vp, ctypes.c_char_p, ctypes.POINTER(i32), i32, i32,
                                        ctypes.POINTER(spws_options_t), ctypes.POINTER(vp)]
+        L.spws_plan_create3.argtypes = L.spws_plan_create.argtypes
+        L.spws_workspace_size3.argtypes = [vp, T, T, T, ctypes.POINTER(sz)]
+        L.spws_symbolic3.argtypes = [vp, T, T, T, T, vp, sz, ctypes.POINTER(ctypes.c_int64)]
+        L.spws_numeric3.argtypes = [vp, T, T, T, T, vp, sz]
         L.spws_plan_destroy.argtypes = [vp]
         L.spws_check_expression.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.spws_workspace_size.argtypes = [vp, T, T, ctypes.POINTER(sz)]
@@ -213,16 +218,21 @@ class Plan:
             if not hasattr(opt, k):
                 raise SpwsError(SPWS_INVALID_ARGUMENT, f"Plan: unknown option {k}")
             setattr(opt, k, v)
-        arr = (ctypes.c_int * 3)(*fmts)
+        arr = (ctypes.c_int * len(fmts))(*fmts)
         pol = POLICIES[policy] if isinstance(policy, str) else int(policy)
-        _check(lib().spws_plan_create(handle._h, expr.encode(), arr, vt, pol, ctypes.byref(opt),
-                                      ctypes.byref(self._p)), "spws_plan_create")
+        create = lib().spws_plan_create3 if len(fmts) == 4 else lib().spws_plan_create
+        _check(create(handle._h, expr.encode(), arr, vt, pol, ctypes.byref(opt), ctypes.byref(self._p)), "spws_plan_create")
 
-    def workspace_size(self, A: TensorArrays, B: TensorArrays) -> int:
+    def workspace_size(self, A: TensorArrays, B: TensorArrays, D: TensorArrays | None = None) -> int:
         out = ctypes.c_size_t(0)
         a, b = A.c_struct(), B.c_struct()
-        _check(lib().spws_workspace_size(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(out)),
-               "spws_workspace_size")
+        if D is None:
+            _check(lib().spws_workspace_size(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(out)),
+                   "spws_workspace_size")
+        else:
+            d = D.c_struct()
+            _check(lib().spws_workspace_size3(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(d), ctypes.byref(out)),
+                   "spws_workspace_size3")
         return int(out.value)
 
     def workspace_size_exact(self, A: TensorArrays, B: TensorArrays, scratch_ptr: int | None = None, scratch_bytes: int = 0,
@@ -235,18 +245,28 @@ class Plan:
                                                ctypes.byref(out), ctypes.c_void_p(row_products_ptr)), "spws_workspace_size_exact")
         return int(out.value)
 
-    def symbolic(self, A, B, C, scratch_ptr: int, scratch_bytes: int):
+    def symbolic(self, A, B, C, scratch_ptr: int, scratch_bytes: int, D=None):
         a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
         sizes = (ctypes.c_int64 * 3)()
-        _check(lib().spws_symbolic(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
-                                   ctypes.c_void_p(scratch_ptr), scratch_bytes, sizes), "spws_symbolic")
+        if D is None:
+            _check(lib().spws_symbolic(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                       ctypes.c_void_p(scratch_ptr), scratch_bytes, sizes), "spws_symbolic")
+        else:
+            d = D.c_struct()
+            _check(lib().spws_symbolic3(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(d), ctypes.byref(c),
+                                        ctypes.c_void_p(scratch_ptr), scratch_bytes, sizes), "spws_symbolic3")
         C.n = [int(sizes[0]), int(sizes[1]), int(sizes[2])]
         return C.n
 
-    def numeric(self, A, B, C, scratch_ptr: int, scratch_bytes: int):
+    def numeric(self, A, B, C, scratch_ptr: int, scratch_bytes: int, D=None):
         a, b, c = A.c_struct(), B.c_struct(), C.c_struct()
-        _check(lib().spws_numeric(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
-                                  ctypes.c_void_p(scratch_ptr), scratch_bytes), "spws_numeric")
+        if D is None:
+            _check(lib().spws_numeric(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                      ctypes.c_void_p(scratch_ptr), scratch_bytes), "spws_numeric")
+        else:
+            d = D.c_struct()
+            _check(lib().spws_numeric3(self._p, ctypes.byref(a), ctypes.byref(b), ctypes.byref(d), ctypes.byref(c),
+                                       ctypes.c_void_p(scratch_ptr), scratch_bytes), "spws_numeric3")
 
     def gather_ceiling(self, A, B, C, scratch_ptr: int, scratch_bytes: int, index_sum_ptr: int, value_sum_ptr: int):
         """spws_gather_ceiling: the dense numeric kernels' traversal with the workspace stripped;

@@ -10,8 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libspws.so")
-SOURCES = ["spws_api.cu", "setup.cu", "ism_reg.cu", "ism_smem.cu", "dense.cu", "ism_global.cu", "outer.cu", "hash.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(HERE, "..", "include", "spws.h")]
+SOURCES = ["spws_api.cu", "setup.cu", "ism_reg.cu", "ism_smem.cu", "dense.cu", "ism_global.cu", "outer.cu", "hash.cu", "higher.cu"]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "sortmerge.cuh"), os.path.join(HERE, "..", "include", "spws.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -97,6 +97,18 @@ struct Csr {
     int ncols;
 };
 
+// A CSF 3-tensor on the device (three compressed levels).
+struct Csf3Dev {
+    const i64* pos1;    // n0 + 1
+    const i64* pos2;    // n1 + 1
+    const int* crd0;
+    const int* crd1;
+    const int* crd2;
+    const void* val;
+    int n0, n1;
+    i64 nnz;
+};
+
 // Per-row tables in scratch.
 struct RowTables {
     i64* ub;
@@ -238,5 +250,14 @@ cudaError_t launch_coo_out(const LaunchCtx& c, const u64* ukeys, const void* uva
 cudaError_t launch_outer_dense(const LaunchCtx& c, bool numeric, const Csr& At, const Csr& B, const i64* koff, i64 P, i64 m, i64 J,
                                unsigned* dbits, void* dvals, int* cnt, const i64* pos, int* Ccrd, void* Cval);
 cudaError_t launch_outer_total(const LaunchCtx& c, const Csr& At, const Csr& B, u64* total_mapped_host);
+// higher.cu: the higher-order scatters with coordinate-form output
+cudaError_t launch_higher_total(const LaunchCtx& c, int form, const Csf3Dev& B, const Csr& C, u64* total_mapped_host);
+cudaError_t launch_higher_setup(const LaunchCtx& c, int form, const Csf3Dev& B, const Csr& C, int* fib_of, int* slice_of, int* cnt);
+cudaError_t launch_higher_ism(const LaunchCtx& c, bool numeric, int form, const Csf3Dev& B, const Csr& C, const Csr& D, const int* fib_of,
+                              const int* slice_of, const i64* eoff, i64 P, i64 cap, u64 d1, u64 d2, int label_bits, u64* kA, void* vA,
+                              u64* kB, void* vB, int* head, i64* at, char* sort_tmp, i64* block_sums, i64* nnz_dev,
+                              i64* nnz_host_pinned, bool* result_first);
+cudaError_t launch_higher_unpack(const LaunchCtx& c, int order, const u64* ukeys, const void* uvals, i64 nnz, u64 d1, u64 d2, int* o0,
+                                 int* o1, int* o2, void* oval);
 
 }  // namespace spws

@@ -28,7 +28,7 @@ constexpr int RS_WARPS = RS_THREADS / 32;
 constexpr int RS_STEPS = 8;                             // 32-element steps per warp
 constexpr int RS_TILE = RS_WARPS * RS_STEPS * 32;       // 2048
 
-__global__ void __launch_bounds__(RS_THREADS) radix_hist_kernel(const u64* __restrict__ keys, i64 n, int shift, int nblocks,
+static __global__ void __launch_bounds__(RS_THREADS) radix_hist_kernel(const u64* __restrict__ keys, i64 n, int shift, int nblocks,
                                                                int* __restrict__ hist) {
     __shared__ int s_h[256];
     s_h[threadIdx.x] = 0;
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(RS_THREADS) radix_scatter_kernel(const u64* __
 }
 
 // ---- Merge (reduce runs of equal labels) and Compress ----------------------------------------
-__global__ void __launch_bounds__(OT) heads_kernel(const u64* __restrict__ keys, i64 n, int* __restrict__ head) {
+static __global__ void __launch_bounds__(OT) heads_kernel(const u64* __restrict__ keys, i64 n, int* __restrict__ head) {
     for (i64 t = (i64)blockIdx.x * OT + threadIdx.x; t < n; t += (i64)gridDim.x * OT)
         head[t] = (t == 0 || keys[t] != keys[t - 1]) ? 1 : 0;
 }
@@ -139,7 +139,7 @@ static cudaError_t radix_sort_t(const LaunchCtx& c, i64 n, int bits, u64* k0, T*
     return cudaGetLastError();
 }
 
-__global__ void drop_absent_kernel(const u64* __restrict__ ukeys, i64* cnt) {
+static __global__ void drop_absent_kernel(const u64* __restrict__ ukeys, i64* cnt) {
     if (*cnt > 0 && ukeys[*cnt - 1] == ABSENT_LABEL) --*cnt;
 }
 

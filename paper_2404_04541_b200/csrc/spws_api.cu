@@ -84,37 +84,61 @@ bool distinct(const std::vector<std::string>& v) {
     return true;
 }
 
-// Accepts
-//   out(o_1..o_N) = x(o_1..o_{N-1}, r) * y(r, o_N), N = 2 or 3, with formats (CSR, CSR, CSR) or
-//     (CSF3, CSF3, CSR): loop order o_1 -> .. -> r -> o_N, output order o_1 -> .. -> o_N; they
-//     mismatch only by the reduction variable sitting one position from the innermost index: a
-//     first-order scatter (kinds 0 and 1);
-//   out(o_1, o_2) = x(r, o_1) * y(r, o_2) with formats (CSR, CSR, CSR): loop order r -> o_1 -> o_2,
-//     the reduction variable outermost, so both output indices scatter: a second-order scatter
-//     (kind 2, the outer-product form).
-// Returns the kind or -1.
-int classify_expression(const char* expr, const spws_format_t fmts[3]) {
+// Accepts (kind in brackets)
+//   [0, 1] out(o_1..o_N) = x(o_1..o_{N-1}, r) * y(r, o_N), N = 2 or 3, formats (CSR, CSR, CSR) or
+//     (CSF3, CSF3, CSR): loop order o_1 -> .. -> r -> o_N against output order o_1 -> .. -> o_N: the
+//     reduction variable sits one position from the innermost index: a first-order scatter;
+//   [2] out(o_1, o_2) = x(r, o_1) * y(r, o_2), formats (CSR, CSR, CSR): loop order r -> o_1 -> o_2, both
+//     output indices scatter: a second-order scatter (the outer-product form);
+//   [3] out(o_1, o_2, o_3) = x(r, o_1, o_2) * y(r, o_3), formats (COO, CSF3, CSR): third-order scatter;
+//   [4] out(o_1, o_2, o_3) = x(o_1, r, o_2) * y(r, o_3), formats (COO, CSF3, CSR): o_1 is shared by the
+//     loop nest and the output, the other two indices scatter;
+//   [5] out(o_1, o_2) = x(r_1, r_2, o_1) * y(r_1, o_2) * z(r_2, o_2), formats (COO, CSF3, CSR, CSR): two
+//     reduction variables outermost, a second-order scatter.
+// Returns the kind or -1; `n_fmts` is 3 (two operands) or 4 (three operands).
+int classify_expression(const char* expr, const spws_format_t* fmts, int n_fmts) {
     const char* s = expr;
-    Access out, x, y;
+    Access out, x, y, z;
     if (!parse_access(s, out)) return -1;
     if (*s == '+' && s[1] == '=') s += 2; else if (*s == '=') s += 1; else return -1;
     if (!parse_access(s, x)) return -1;
     if (*s != '*') return -1;
     ++s;
     if (!parse_access(s, y)) return -1;
+    int n_ops = 2;
+    if (*s == '*') {
+        ++s;
+        if (!parse_access(s, z)) return -1;
+        n_ops = 3;
+    }
     if (*s != '\0') return -1;
+    if (n_ops + 1 != n_fmts) return -1;
     const size_t N = out.idx.size();
     if (N != 2 && N != 3) return -1;
-    if (x.idx.size() != N || y.idx.size() != 2) return -1;
-    if (!distinct(out.idx) || !distinct(x.idx) || !distinct(y.idx)) return -1;
-    if (out.name == x.name || out.name == y.name) return -1;
-    if (N == 2 && x.idx[0] == y.idx[0] && x.idx[1] == out.idx[0] && y.idx[1] == out.idx[1] && x.idx[0] != out.idx[0] &&
-        x.idx[0] != out.idx[1]) {
+    if (!distinct(out.idx) || !distinct(x.idx) || !distinct(y.idx) || y.idx.size() != 2) return -1;
+    if (out.name == x.name || out.name == y.name || (n_ops == 3 && (out.name == z.name || !distinct(z.idx) || z.idx.size() != 2))) return -1;
+    auto is_output = [&](const std::string& v) { for (const auto& o : out.idx) if (o == v) return true; return false; };
+    if (n_ops == 3) {
+        if (N != 2 || x.idx.size() != 3) return -1;
+        const std::string &r1 = x.idx[0], &r2 = x.idx[1];
+        if (is_output(r1) || is_output(r2) || r1 == r2) return -1;
+        if (x.idx[2] != out.idx[0] || y.idx[0] != r1 || y.idx[1] != out.idx[1] || z.idx[0] != r2 || z.idx[1] != out.idx[1]) return -1;
+        if (fmts[0] != SPWS_COO || fmts[1] != SPWS_CSF3 || fmts[2] != SPWS_CSR || fmts[3] != SPWS_CSR) return -1;
+        return 5;
+    }
+    if (x.idx.size() != N) return -1;
+    if (fmts[0] == SPWS_COO) {
+        if (N != 3 || fmts[1] != SPWS_CSF3 || fmts[2] != SPWS_CSR) return -1;
+        if (!is_output(x.idx[0]) && x.idx[1] == out.idx[0] && x.idx[2] == out.idx[1] && y.idx[0] == x.idx[0] && y.idx[1] == out.idx[2]) return 3;
+        if (!is_output(x.idx[1]) && x.idx[0] == out.idx[0] && x.idx[2] == out.idx[1] && y.idx[0] == x.idx[1] && y.idx[1] == out.idx[2]) return 4;
+        return -1;
+    }
+    if (N == 2 && x.idx[0] == y.idx[0] && x.idx[1] == out.idx[0] && y.idx[1] == out.idx[1] && !is_output(x.idx[0])) {
         if (fmts[0] != SPWS_CSR || fmts[1] != SPWS_CSR || fmts[2] != SPWS_CSR) return -1;
         return 2;
     }
     const std::string& r = x.idx[N - 1];
-    for (size_t a = 0; a < N; ++a) if (out.idx[a] == r) return -1;           // r must be a reduction variable
+    if (is_output(r)) return -1;                                             // r must be a reduction variable
     for (size_t a = 0; a + 1 < N; ++a) if (x.idx[a] != out.idx[a]) return -1;
     if (y.idx[0] != r || y.idx[1] != out.idx[N - 1]) return -1;
     if (N == 2) {
@@ -503,6 +527,219 @@ spws_status_t outer_numeric(spws_plan_s* plan, const Shapes& S, spws_tensor_t* C
     return SPWS_OK;
 }
 
+// ---- higher-order scatters with coordinate-form output (kinds 3, 4, 5) -------------------------
+struct HShapes {
+    int form;                   // 0 SpTTM, 1 SpTTM-I, 2 SpMTTKRP
+    Csf3Dev B;
+    Csr C, D;
+    int order;                  // of the output
+    int64_t odims[3];
+    u64 d1, d2;                 // label = (c_a * d1 + c_b) * d2 + c_c, or c_a * d2 + c_b
+    int label_bits;
+};
+
+spws_status_t check_higher(const spws_plan_s* p, const spws_tensor_t* B, const spws_tensor_t* C, const spws_tensor_t* D, HShapes& H,
+                           bool need_pointers) {
+    if (!B || !C) return SPWS_INVALID_ARGUMENT;
+    H.form = p->kind - 3;
+    if ((H.form == 2) != (D != nullptr)) return SPWS_INVALID_ARGUMENT;
+    if (B->order != 3 || C->order != 2 || (D && D->order != 2)) return SPWS_INVALID_ARGUMENT;
+    for (int a = 0; a < 3; ++a)
+        if (B->dims[a] < 0 || B->dims[a] > 0x7ffffff0ll || B->n[a] < 0) return SPWS_INVALID_ARGUMENT;
+    if (B->n[0] > B->dims[0] || B->n[1] < B->n[0] || B->n[2] < B->n[1]) return SPWS_INVALID_ARGUMENT;
+    if (C->dims[0] < 0 || C->dims[1] < 0 || C->dims[1] > 0x7ffffff0ll || C->n[1] < 0) return SPWS_INVALID_ARGUMENT;
+    H.B = Csf3Dev{LL(B->pos[1]), LL(B->pos[2]), B->crd[0], B->crd[1], B->crd[2], B->val, (int)B->n[0], (int)B->n[1], B->n[2]};
+    H.C = Csr{LL(C->pos[1]), C->crd[1], C->val, (int)C->dims[0], (int)C->dims[1]};
+    H.D = Csr{};
+    if (H.form == 0) {          // B(k,i,j), C(k,l) -> (i,j,l)
+        if (C->dims[0] != B->dims[0]) return SPWS_DIM_MISMATCH;
+        H.order = 3; H.odims[0] = B->dims[1]; H.odims[1] = B->dims[2]; H.odims[2] = C->dims[1];
+    } else if (H.form == 1) {   // B(k,i,j), C(i,l) -> (k,j,l)
+        if (C->dims[0] != B->dims[1]) return SPWS_DIM_MISMATCH;
+        H.order = 3; H.odims[0] = B->dims[0]; H.odims[1] = B->dims[2]; H.odims[2] = C->dims[1];
+    } else {                    // B(k,l,i), C(k,j), D(l,j) -> (i,j)
+        if (C->dims[0] != B->dims[0] || D->dims[0] != B->dims[1] || D->dims[1] != C->dims[1]) return SPWS_DIM_MISMATCH;
+        if (D->n[1] < 0) return SPWS_INVALID_ARGUMENT;
+        H.D = Csr{LL(D->pos[1]), D->crd[1], D->val, (int)D->dims[0], (int)D->dims[1]};
+        H.order = 2; H.odims[0] = B->dims[2]; H.odims[1] = C->dims[1]; H.odims[2] = 1;
+    }
+    // the label must fit 63 bits (one more is kept for the absent label)
+    long double cells = 1.0L;
+    for (int a = 0; a < H.order; ++a) cells *= (long double)(H.odims[a] > 0 ? H.odims[a] : 1);
+    if (cells >= 4.0e18L) return SPWS_WORKSPACE_TOO_LARGE;
+    H.d1 = H.order == 3 ? (u64)H.odims[1] : 1;
+    H.d2 = (u64)H.odims[H.order - 1];
+    u64 top = 1;
+    for (int a = 0; a < H.order; ++a) top *= (u64)(H.odims[a] > 0 ? H.odims[a] : 1);
+    H.label_bits = 1;
+    while (H.label_bits < 63 && (top >> H.label_bits) != 0) ++H.label_bits;
+    ++H.label_bits;             // the absent label's extra bit
+    if (!need_pointers) return SPWS_OK;
+    if (B->n[2] > 0 && (!H.B.pos1 || !H.B.pos2 || !H.B.crd0 || !H.B.crd1 || !H.B.crd2 || !H.B.val)) return SPWS_INVALID_ARGUMENT;
+    if (C->dims[0] > 0 && !H.C.pos) return SPWS_INVALID_ARGUMENT;
+    if (C->n[1] > 0 && (!H.C.crd || !H.C.val)) return SPWS_INVALID_ARGUMENT;
+    if (D && ((D->dims[0] > 0 && !H.D.pos) || (D->n[1] > 0 && (!H.D.crd || !H.D.val)))) return SPWS_INVALID_ARGUMENT;
+    return SPWS_OK;
+}
+
+struct HLayout {
+    size_t ctl, fib_of, slice_of, cnt, eoff, block_sums, fixed_end, kA, kB, vA, vB, head, at, sort_tmp, end;
+    int64_t N;
+};
+
+HLayout make_hlayout(const spws_plan_s* p, const HShapes& H, int64_t P) {
+    HLayout L{};
+    const size_t V = p->is_f64 ? 8 : 4;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
+    const int64_t cap = p->opt.outer_cap > 0 ? p->opt.outer_cap : P;
+    L.N = P + (cap < P ? cap : 0);
+    const int64_t longest = std::max<int64_t>(H.B.nnz, L.N);
+    L.ctl = take(sizeof(DevCtl));
+    L.fib_of = take(4 * (size_t)H.B.nnz);
+    L.slice_of = take(4 * (size_t)H.B.n1);
+    L.cnt = take(4 * (size_t)H.B.nnz);
+    L.eoff = take(8 * ((size_t)H.B.nnz + 1));
+    L.block_sums = take(8 * ((size_t)longest / 2048 + 2));
+    L.fixed_end = o;
+    L.kA = take(8 * (size_t)L.N);
+    L.kB = take(8 * (size_t)L.N);
+    L.vA = take(V * (size_t)L.N);
+    L.vB = take(V * (size_t)L.N);
+    L.head = take(4 * (size_t)L.N);
+    L.at = take(8 * ((size_t)L.N + 1));
+    L.sort_tmp = take(outer_sort_scratch_bytes(L.N));
+    L.end = o;
+    return L;
+}
+
+spws_status_t higher_count_products(spws_plan_s* p, const HShapes& H, int64_t* P) {
+    LaunchCtx c{};
+    c.stream = p->h->stream;
+    c.sm_count = p->h->sm_count;
+    u64* word = reinterpret_cast<u64*>(&p->host_ctl->products);
+    *word = 0;
+    CUDA_TRY(launch_higher_total(c, H.form, H.B, H.C, word));
+    CUDA_TRY(cudaStreamSynchronize(c.stream));
+    *P = (int64_t)*word;
+    return SPWS_OK;
+}
+
+spws_status_t higher_workspace_size(spws_plan_s* plan, const spws_tensor_t* B, const spws_tensor_t* C, const spws_tensor_t* D, size_t* bytes) {
+    HShapes H{};
+    spws_status_t st = check_higher(plan, B, C, D, H, true);
+    if (st != SPWS_OK) return st;
+    int64_t P = 0;
+    if ((st = higher_count_products(plan, H, &P)) != SPWS_OK) return st;
+    *bytes = make_hlayout(plan, H, P).end;
+    return SPWS_OK;
+}
+
+spws_status_t check_coo_output(const HShapes& H, const spws_tensor_t* Out) {
+    if (!Out || Out->order != H.order) return SPWS_INVALID_ARGUMENT;
+    for (int a = 0; a < H.order; ++a)
+        if (Out->dims[a] != H.odims[a]) return SPWS_DIM_MISMATCH;
+    return SPWS_OK;
+}
+
+spws_status_t higher_symbolic(spws_plan_s* plan, const spws_tensor_t* B, const spws_tensor_t* C, const spws_tensor_t* D, spws_tensor_t* Out,
+                              void* scratch, size_t scratch_bytes, int64_t* sizes_out) {
+    plan->symbolic_ok = false;
+    HShapes H{};
+    spws_status_t st = check_higher(plan, B, C, D, H, true);
+    if (st != SPWS_OK) return st;
+    if ((st = check_coo_output(H, Out)) != SPWS_OK) return st;
+    if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return SPWS_INVALID_ARGUMENT;
+    int64_t P = 0;
+    if ((st = higher_count_products(plan, H, &P)) != SPWS_OK) return st;
+    if (P > 0x7fff0000ll || H.B.nnz > 0x7fff0000ll) return SPWS_INTERNAL_OVERFLOW;       // ordinals and scans are 31-bit here
+    const HLayout L = make_hlayout(plan, H, P);
+    if (scratch_bytes < L.end) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c{};
+    c.stream = plan->h->stream;
+    c.sm_count = plan->h->sm_count;
+    c.ctl = reinterpret_cast<DevCtl*>(sc + L.ctl);
+    c.is_f64 = plan->is_f64;
+    CUDA_TRY(cudaMemsetAsync(c.ctl, 0, sizeof(DevCtl), c.stream));
+    mark_start(plan, 0);
+    int* fib_of = reinterpret_cast<int*>(sc + L.fib_of);
+    int* slice_of = reinterpret_cast<int*>(sc + L.slice_of);
+    int* cnt = reinterpret_cast<int*>(sc + L.cnt);
+    i64* eoff = reinterpret_cast<i64*>(sc + L.eoff);
+    i64* block_sums = reinterpret_cast<i64*>(sc + L.block_sums);
+    CUDA_TRY(launch_higher_setup(c, H.form, H.B, H.C, fib_of, slice_of, cnt));
+    CUDA_TRY(launch_scan_counts(c, cnt, (int)H.B.nnz, eoff, block_sums, &c.ctl->products));
+    mark(plan, SPWS_T_SYM_BOUNDS);
+    bool first = true;
+    i64* nnz_host = reinterpret_cast<i64*>(&plan->host_ctl->nnz);
+    const int64_t cap = plan->opt.outer_cap > 0 ? plan->opt.outer_cap : (P > 0 ? P : 1);
+    CUDA_TRY(launch_higher_ism(c, false, H.form, H.B, H.C, H.D, fib_of, slice_of, eoff, P, cap, H.d1, H.d2, H.label_bits,
+                               reinterpret_cast<u64*>(sc + L.kA), nullptr, reinterpret_cast<u64*>(sc + L.kB), nullptr,
+                               reinterpret_cast<int*>(sc + L.head), reinterpret_cast<i64*>(sc + L.at), sc + L.sort_tmp, block_sums,
+                               &c.ctl->nnz, nnz_host, &first));
+    const int64_t nnz = *nnz_host;
+    mark(plan, SPWS_T_SYM_ISM_GLOBAL);
+    CUDA_TRY(cudaMemcpyAsync(&plan->host_ctl->status, &c.ctl->status, sizeof(int), cudaMemcpyDeviceToHost, c.stream));
+    CUDA_TRY(cudaStreamSynchronize(c.stream));
+    plan->stats = spws_stats_t{};
+    plan->stats.device_status = plan->host_ctl->status;
+    if (plan->host_ctl->status != 0) return from_dev_status(plan->host_ctl->status);
+    plan->stats.rows = H.B.nnz;
+    plan->stats.products = P;
+    plan->stats.nnz = nnz;
+    plan->stats.rows_per_class[public_class(CLS_ISM_GLOBAL)] = H.B.nnz;
+    plan->stats.products_per_class[public_class(CLS_ISM_GLOBAL)] = P;
+    plan->stats.nnz_per_class[public_class(CLS_ISM_GLOBAL)] = nnz;
+    plan->stats.launches_symbolic = c.launches;
+    plan->outer_products = P;
+    Out->n[0] = nnz; Out->n[1] = 0; Out->n[2] = 0;
+    if (sizes_out) { sizes_out[0] = nnz; sizes_out[1] = 0; sizes_out[2] = 0; }
+    plan->symbolic_ok = true;
+    plan->m = H.B.nnz;
+    plan->scratch = scratch;
+    return SPWS_OK;
+}
+
+spws_status_t higher_numeric(spws_plan_s* plan, const spws_tensor_t* B, const spws_tensor_t* C, const spws_tensor_t* D, spws_tensor_t* Out,
+                             void* scratch, size_t scratch_bytes) {
+    if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
+    HShapes H{};
+    spws_status_t st = check_higher(plan, B, C, D, H, true);
+    if (st != SPWS_OK) return st;
+    if ((st = check_coo_output(H, Out)) != SPWS_OK) return st;
+    if (scratch != plan->scratch || H.B.nnz != plan->m) return SPWS_BAD_SEQUENCE;
+    const int64_t P = plan->outer_products, nnz = plan->stats.nnz;
+    if (Out->n[0] < nnz) return SPWS_OUTPUT_TOO_SMALL;
+    if (nnz > 0) {
+        if (!Out->val) return SPWS_INVALID_ARGUMENT;
+        for (int a = 0; a < H.order; ++a) if (!Out->crd[a]) return SPWS_INVALID_ARGUMENT;
+    }
+    const HLayout L = make_hlayout(plan, H, P);
+    if (scratch_bytes < L.end) return SPWS_SCRATCH_TOO_SMALL;
+    char* sc = static_cast<char*>(scratch);
+    LaunchCtx c{};
+    c.stream = plan->h->stream;
+    c.sm_count = plan->h->sm_count;
+    c.ctl = reinterpret_cast<DevCtl*>(sc + L.ctl);
+    c.is_f64 = plan->is_f64;
+    mark_start(plan, 1);
+    bool first = true;
+    i64* nnz_host = reinterpret_cast<i64*>(&plan->host_ctl->nnz);
+    const int64_t cap = plan->opt.outer_cap > 0 ? plan->opt.outer_cap : (P > 0 ? P : 1);
+    CUDA_TRY(launch_higher_ism(c, true, H.form, H.B, H.C, H.D, reinterpret_cast<int*>(sc + L.fib_of), reinterpret_cast<int*>(sc + L.slice_of),
+                               reinterpret_cast<i64*>(sc + L.eoff), P, cap, H.d1, H.d2, H.label_bits, reinterpret_cast<u64*>(sc + L.kA),
+                               sc + L.vA, reinterpret_cast<u64*>(sc + L.kB), sc + L.vB, reinterpret_cast<int*>(sc + L.head),
+                               reinterpret_cast<i64*>(sc + L.at), sc + L.sort_tmp, reinterpret_cast<i64*>(sc + L.block_sums),
+                               &c.ctl->kept[0], nnz_host, &first));
+    if (*nnz_host != nnz) return SPWS_BAD_SEQUENCE;                 // operands differ from the symbolic pass's
+    CUDA_TRY(launch_higher_unpack(c, H.order, reinterpret_cast<u64*>(sc + (first ? L.kA : L.kB)), sc + (first ? L.vA : L.vB), nnz, H.d1, H.d2,
+                                  Out->crd[0], Out->crd[1], Out->crd[2], Out->val));
+    mark(plan, SPWS_T_NUM_ISM_GLOBAL);
+    plan->stats.launches_numeric = c.launches;
+    return SPWS_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -510,8 +747,8 @@ extern "C" {
 spws_status_t spws_check_expression(const char* expr, const spws_format_t fmts[3], int* kind) {
     if (!expr || !fmts) return SPWS_INVALID_ARGUMENT;
     for (int f = 0; f < 3; ++f)
-        if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3) return SPWS_INVALID_ARGUMENT;
-    const int k = classify_expression(expr, fmts);
+        if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3 && fmts[f] != SPWS_COO) return SPWS_INVALID_ARGUMENT;
+    const int k = classify_expression(expr, fmts, 3);
     if (k < 0) return SPWS_UNSUPPORTED_EXPRESSION;
     if (kind) *kind = k;
     return SPWS_OK;
@@ -543,16 +780,17 @@ spws_status_t spws_set_stream(spws_handle_t handle, void* cuda_stream) {
     return SPWS_OK;
 }
 
-spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spws_format_t fmts[3],
-                               spws_dtype_t value_type, spws_policy_t policy, const spws_options_t* options,
-                               spws_plan_t* plan) {
+static spws_status_t plan_create_n(spws_handle_t handle, const char* expr, const spws_format_t* fmts, int n_fmts,
+                                   spws_dtype_t value_type, spws_policy_t policy, const spws_options_t* options,
+                                   spws_plan_t* plan) {
     if (!handle || !expr || !fmts || !plan) return SPWS_INVALID_ARGUMENT;
     if (value_type != SPWS_F32 && value_type != SPWS_F64) return SPWS_INVALID_ARGUMENT;
     if (policy != SPWS_DENSE && policy != SPWS_SPARSE_ISM && policy != SPWS_AUTO && policy != SPWS_HASH) return SPWS_INVALID_ARGUMENT;
-    for (int f = 0; f < 3; ++f)
-        if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3) return SPWS_INVALID_ARGUMENT;
-    const int kind = classify_expression(expr, fmts);
+    for (int f = 0; f < n_fmts; ++f)
+        if (fmts[f] != SPWS_CSR && fmts[f] != SPWS_CSF3 && fmts[f] != SPWS_COO) return SPWS_INVALID_ARGUMENT;
+    const int kind = classify_expression(expr, fmts, n_fmts);
     if (kind < 0) return SPWS_UNSUPPORTED_EXPRESSION;
+    if (kind >= 3 && policy == SPWS_DENSE) return SPWS_WORKSPACE_TOO_LARGE;      // no dense workspace of order three is offered
     spws_options_t o{};
     if (options) o = *options;
     const bool f64 = value_type == SPWS_F64;
@@ -585,6 +823,16 @@ spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spw
     memset(p->host_ctl, 0, sizeof(DevCtl));
     *plan = p;
     return SPWS_OK;
+}
+
+spws_status_t spws_plan_create(spws_handle_t handle, const char* expr, const spws_format_t fmts[3], spws_dtype_t value_type,
+                               spws_policy_t policy, const spws_options_t* options, spws_plan_t* plan) {
+    return plan_create_n(handle, expr, fmts, 3, value_type, policy, options, plan);
+}
+
+spws_status_t spws_plan_create3(spws_handle_t handle, const char* expr, const spws_format_t fmts[4], spws_dtype_t value_type,
+                                spws_policy_t policy, const spws_options_t* options, spws_plan_t* plan) {
+    return plan_create_n(handle, expr, fmts, 4, value_type, policy, options, plan);
 }
 
 spws_status_t spws_set_profiling(spws_plan_t plan, int enabled) {
@@ -628,6 +876,8 @@ spws_status_t spws_plan_destroy(spws_plan_t plan) {
 
 spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, size_t* bytes) {
     if (!plan || !bytes) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind == 5) return SPWS_INVALID_ARGUMENT;           // three operands: spws_workspace_size3
+    if (plan->kind >= 3) return higher_workspace_size(plan, A, B, nullptr, bytes);
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S, plan->kind != 2);   // pointers may still be unset when sizing
     if (st != SPWS_OK) return st;
@@ -649,7 +899,7 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
 spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, void* scratch,
                                         size_t scratch_bytes, size_t* bytes, int64_t* row_products) {
     if (!plan || !bytes) return SPWS_INVALID_ARGUMENT;
-    if (plan->kind == 2) return spws_workspace_size(plan, A, B, bytes);      // already sized from the product count
+    if (plan->kind >= 2) return spws_workspace_size(plan, A, B, bytes);      // already sized from the product count
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S, scratch != nullptr);
     if (st != SPWS_OK) return st;
@@ -675,12 +925,11 @@ spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A
     if (hc.status != 0 && hc.status != DEV_SCRATCH_TOO_SMALL) return from_dev_status(hc.status);
     size_t need = L.fixed_end + align256((size_t)hc.bm_words_used * 4);
     const int64_t n_global = hc.class_count[CLS_ISM_GLOBAL];
-    if (n_global > 0) {                         // one numeric slot per CTA the global-memory ISM launches
+    if (n_global > 0) {                         // numeric slots of the global-memory ISM: one per row, eight at most
         int64_t elems = hc.max_ub_global < S.ncols ? hc.max_ub_global : S.ncols;
         elems = (elems + 63) & ~63ll;
         const size_t comp = 4 + (plan->is_f64 ? 8 : 4);
-        const int64_t ctas = n_global < 2 * (int64_t)plan->h->sm_count ? n_global : 2 * (int64_t)plan->h->sm_count;
-        need += align256(2 * (size_t)elems * comp) * (size_t)ctas;
+        need += align256(2 * (size_t)elems * comp) * (size_t)(n_global < 8 ? n_global : 8);
     }
     *bytes = need;
     return SPWS_OK;
@@ -689,6 +938,8 @@ spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A
 spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, spws_tensor_t* C,
                             void* scratch, size_t scratch_bytes, int64_t* sizes_out) {
     if (!plan) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind == 5) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind >= 3) return higher_symbolic(plan, A, B, nullptr, C, scratch, scratch_bytes, sizes_out);
     plan->symbolic_ok = false;
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S);
@@ -799,6 +1050,8 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
 spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, spws_tensor_t* C,
                            void* scratch, size_t scratch_bytes) {
     if (!plan) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind == 5) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind >= 3) return higher_numeric(plan, A, B, nullptr, C, scratch, scratch_bytes);
     if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S);
@@ -858,7 +1111,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
 spws_status_t spws_gather_ceiling(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* C,
                                   void* scratch, size_t scratch_bytes, uint64_t* index_sum, double* value_sum) {
     if (!plan || !index_sum || !value_sum) return SPWS_INVALID_ARGUMENT;
-    if (plan->kind == 2) return SPWS_UNSUPPORTED_EXPRESSION;    // the first-order dense kernels do not run for the outer form
+    if (plan->kind >= 2) return SPWS_UNSUPPORTED_EXPRESSION;    // the first-order dense kernels run for the row-wise forms only
     if (!plan->symbolic_ok) return SPWS_BAD_SEQUENCE;
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S);
@@ -898,9 +1151,27 @@ spws_status_t spws_get_stats(spws_plan_t plan, spws_stats_t* stats) {
     return from_dev_status(plan->host_ctl->status);
 }
 
+spws_status_t spws_workspace_size3(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* D, size_t* bytes) {
+    if (!plan || !bytes || plan->kind != 5) return SPWS_INVALID_ARGUMENT;
+    return higher_workspace_size(plan, A, B, D, bytes);
+}
+
+spws_status_t spws_symbolic3(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* D, spws_tensor_t* C,
+                             void* scratch, size_t scratch_bytes, int64_t* sizes_out) {
+    if (!plan || plan->kind != 5) return SPWS_INVALID_ARGUMENT;
+    return higher_symbolic(plan, A, B, D, C, scratch, scratch_bytes, sizes_out);
+}
+
+spws_status_t spws_numeric3(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, const spws_tensor_t* D, spws_tensor_t* C,
+                            void* scratch, size_t scratch_bytes) {
+    if (!plan || plan->kind != 5) return SPWS_INVALID_ARGUMENT;
+    return higher_numeric(plan, A, B, D, C, scratch, scratch_bytes);
+}
+
 spws_status_t spws_execute_host(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B, spws_tensor_t* C,
                                 void* arena, size_t arena_bytes, size_t* arena_needed) {
     if (!plan || !A || !B || !C || !arena) return SPWS_INVALID_ARGUMENT;
+    if (plan->kind >= 3) return SPWS_UNSUPPORTED_EXPRESSION;     // host entry: the CSR / CSF result forms only
     if (reinterpret_cast<uintptr_t>(arena) & 255) return SPWS_INVALID_ARGUMENT;
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S);

@@ -19,7 +19,7 @@ def binding():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "spws.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(spws_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(spws_[a-z_0-9]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol(binding):
@@ -52,7 +52,11 @@ def test_status_strings(binding):
     ("C(j,i)=A(i,k)*B(k,j)", (0, 0, 0), False),        # transposed output
     ("C(i,j)=A(i,k)*B(j,k)", (0, 0, 0), False),        # B accessed against its storage order
     ("C(i,j)=A(i,j)*B(i,j)", (0, 0, 0), False),        # element-wise: no reduction variable
-    ("C(i,j,l)=A(k,i,j)*B(k,l)", (1, 1, 0), False),    # contraction of the outermost mode
+    ("C(i,j,l)=A(k,i,j)*B(k,l)", (1, 1, 0), False),    # contraction of the outermost mode needs a COO result
+    ("C(i,j,l)=A(k,i,j)*B(k,l)", (2, 1, 0), True),     # SpTTM, third-order scatter
+    ("C(k,j,l)=A(k,i,j)*B(i,l)", (2, 1, 0), True),     # SpTTM-I
+    ("C(i,j,l)=A(i,j,k)*B(k,l)", (2, 1, 0), False),    # the first-order form has a CSF result
+    ("C(k,j,l)=A(k,i,j)*B(i,l)", (2, 0, 0), False),
     ("C(i,j)=A(i,k)+B(k,j)", (0, 0, 0), False),
     ("C(i,j)=A(i,k)*B(k,j)*D(j,j)", (0, 0, 0), False),
     ("C(i,i)=A(i,k)*B(k,i)", (0, 0, 0), False),

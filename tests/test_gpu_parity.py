@@ -548,6 +548,41 @@ def test_outer_product_on_a_power_law_matrix_and_wide_labels(ctx, oracle_mod):
     dense_plan.close()
 
 
+# ------------------------------------------------------------------ higher-order scatters, COO result
+@pytest.mark.parametrize("dims,nnz,L,seed", [((6, 7, 8), 80, 9, 1), ((40, 30, 50), 3000, 64, 2), ((8, 200, 300), 5000, 1000, 3)])
+def test_higher_order_scatters_match_the_oracle(ctx, oracle_mod, dims, nnz, L, seed):
+    """SpTTM with the outermost mode contracted, SpTTM-I and SpMTTKRP (sparse result in coordinate
+    form) against the map oracle: coordinates exact and in lexicographic order, values under the
+    two-clause rule, in one round and with accumulation arrays that fill several times."""
+    from paper_2404_04541_b200 import api
+    B = uniform_csf3(dims, nnz, seed)
+    dB = api.DeviceCSF3.from_host(B)
+    cases = [
+        (api.EXPR_SPTTM, oracle_mod.spttm, [random_csr(dims[0], L, 0.3, seed + 10, empty_row_frac=0.2)]),
+        (api.EXPR_SPTTM_I, oracle_mod.spttm_i, [random_csr(dims[1], L, 0.05 if L > 500 else 0.3, seed + 11, empty_row_frac=0.2)]),
+        (api.EXPR_SPMTTKRP, oracle_mod.spmttkrp, [random_csr(dims[0], L, 0.3, seed + 12), random_csr(dims[1], L, 0.05 if L > 500 else 0.3, seed + 13)]),
+    ]
+    for expr, fn, mats in cases:
+        ref = fn(B, *mats)
+        dm = [api.DeviceCSR.from_host(m) for m in mats]
+        caps = [0, max(7, ref.products // 3 + 1)] + ([5] if nnz < 100 else [])
+        for cap in caps:
+            crd, val, stats = ctx.scatter_coo(expr, dB, *dm, policy="ism", outer_cap=cap)
+            assert stats["nnz"] == ref.nnz, expr
+            if expr != api.EXPR_SPMTTKRP:
+                assert stats["products"] == ref.products, expr     # (SpMTTKRP numbers the C-row elements; some are absent)
+            assert np.array_equal(crd.cpu().numpy().astype(np.int64), ref.crd), expr
+            ok, _ = values_close(val.cpu().numpy(), ref.val_ref, ref.abs, 1e-12)
+            assert ok.all(), expr
+
+
+def test_higher_order_scatters_refuse_a_dense_workspace(ctx):
+    from paper_2404_04541_b200 import api, binding
+    with pytest.raises(binding.SpwsError) as e:
+        ctx.plan(api.EXPR_SPTTM, (binding.SPWS_COO, binding.SPWS_CSF3, binding.SPWS_CSR), np.float64, "dense")
+    assert e.value.status == binding.SPWS_WORKSPACE_TOO_LARGE
+
+
 # ------------------------------------------------------------------ gather-only lower bound
 @pytest.mark.parametrize("name", ["rmat", "stencil", "heavy"])
 def test_gather_ceiling_visits_every_product_once(ctx, name):
