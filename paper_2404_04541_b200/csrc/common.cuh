@@ -8,7 +8,7 @@ namespace spws {
 typedef long long i64;
 typedef unsigned long long u64;
 
-constexpr int NCLASS = 12;
+constexpr int NCLASS = 13;
 // Row classes = the workspace a row (or (i,j) fibre) is routed to in the symbolic pass.
 enum RowClass : int {
     CLS_EMPTY = 0,      // no intermediate product
@@ -22,7 +22,8 @@ enum RowClass : int {
     CLS_DENSE_CTA = 8,  // dense workspace, one CTA per row
     CLS_ISM_GLOBAL = 9, // accumulation array in shared memory, all array in global memory
     CLS_HASH_S = 10,    // hash table in shared memory (reduction at insert time), small CTA
-    CLS_HASH = 11       // hash table in shared memory, full CTA
+    CLS_HASH = 11,      // hash table in shared memory, full CTA
+    CLS_COPY8 = 12      // one A entry picking a B row of at most 8 entries: the result is that row, scaled
 };
 constexpr int NUM_SLOT = 16;   // work_counter[cls] in the symbolic pass, work_counter[NUM_SLOT + cls] in the numeric pass
 constexpr int CEIL_SLOT = 32;  // work_counter[CEIL_SLOT + cls] in the gather-only (iteration-only) kernels
@@ -30,7 +31,7 @@ constexpr int EMIT_SLOT = 48;  // work_counter slot of the coordinate emission o
 constexpr int BW_SLOT = 49;    // work_counter slot of the word-list build
 constexpr int N_WORK_COUNTERS = 64;
 // index of a class in the public statistics (the three register classes are reported as one)
-__host__ __device__ inline int public_class(int cls) { return cls == 0 ? 0 : (cls <= 3 ? 1 : cls - 2); }
+__host__ __device__ inline int public_class(int cls) { return cls == 0 ? 0 : ((cls <= 3 || cls == 12) ? 1 : cls - 2); }
 constexpr int N_PUBLIC_CLASS = 10;
 constexpr int HASH_SMALL_CAP = 1024;       // products of a row the small / the full hash workspace takes
 constexpr int HASH_CAP = 4096;

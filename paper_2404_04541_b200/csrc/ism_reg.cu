@@ -170,11 +170,11 @@ static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int cls, int n_hos
 cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                            const i64* rowptr, int* Ccrd, void* Cval) {
     if (c.is_f64) {
-        if (cls == CLS_ISM_REG8) return launch_g<double, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
+        if (cls == CLS_ISM_REG8 || cls == CLS_COPY8) return launch_g<double, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
         if (cls == CLS_ISM_REG16) return launch_g<double, 16>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
         return launch_g<double, 32>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
     }
-    if (cls == CLS_ISM_REG8) return launch_g<float, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
+    if (cls == CLS_ISM_REG8 || cls == CLS_COPY8) return launch_g<float, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
     if (cls == CLS_ISM_REG16) return launch_g<float, 16>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
     return launch_g<float, 32>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
 }

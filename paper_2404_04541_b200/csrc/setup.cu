@@ -45,7 +45,7 @@ __device__ __forceinline__ int dense_class(i64 ub, i64 span_words) {
     return ub >= DENSE_HUB_UB ? CLS_DENSE_HUB : CLS_DENSE_CTA;
 }
 
-__device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const ClassParams& prm, DevCtl* ctl) {
+__device__ __forceinline__ int classify_row(i64 ub, i64 entries, int jmin, int jmax, const ClassParams& prm, DevCtl* ctl) {
     if (ub == 0) return CLS_EMPTY;
     const i64 span = (i64)jmax - jmin + 1;
     const i64 span_words = (span + 31) >> 5;
@@ -55,7 +55,9 @@ __device__ __forceinline__ int classify_row(i64 ub, int jmin, int jmax, const Cl
         if (!dense_ok) { raise_status(ctl, DEV_WORKSPACE_TOO_LARGE); return CLS_EMPTY; }
         return dense_class(ub, span_words);
     }
-    const int reg_cls = ub <= 8 ? CLS_ISM_REG8 : (ub <= 16 ? CLS_ISM_REG16 : CLS_ISM_REG);
+    // a single entry picking a short B row: Insert, Sort and Merge are the identity and the
+    // output count is the B row's length, known right here
+    const int reg_cls = ub <= 8 ? (entries == 1 ? CLS_COPY8 : CLS_ISM_REG8) : (ub <= 16 ? CLS_ISM_REG16 : CLS_ISM_REG);
     if (prm.policy == 1) {                       // sparse ISM forced
         if (reg_ok) return reg_cls;
         if (ub <= prm.smem_small_cap) return CLS_ISM_SMEM_S;
@@ -153,11 +155,11 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         if (gl == 0) {
             if (lo < 0 || hi >= B.ncols) { raise_status(ctl, DEV_NONCANONICAL); u = 0; }
             if (u > 0) lo &= ~31;               // bitmap words of every row start at a multiple of 32 columns
-            const int cls = classify_row(u, lo, hi, prm, ctl);
+            const int cls = classify_row(u, pe - ps, lo, hi, prm, ctl);
             tab.ub[row] = u;
             tab.jmin[row] = lo;
             tab.jmax[row] = hi;
-            tab.cnt[row] = 0;
+            tab.cnt[row] = cls == CLS_COPY8 ? (int)u : 0;
             tab.cls[row] = (unsigned char)cls;
             if (cls != run_cls) {
                 if (run_rows) {

@@ -967,34 +967,44 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     mark(plan, SPWS_T_SYM_BOUNDS);
     CUDA_TRY(launch_bin_rows(c, (int)S.m));
     mark(plan, SPWS_T_SYM_BIN);
+    // the class sizes come back now, so that only the workspaces that have rows are launched, with
+    // grids sized for them (a launch for an empty class costs as much as a small class's work)
+    int* hcount = plan->host_ctl->class_count;
+    CUDA_TRY(cudaMemcpyAsync(hcount, c.ctl->class_count, sizeof(int) * NCLASS, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
     // a3: exact count per row through the workspace of its class
     i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<i64*>(sc + L.rowptr_raw);
     if (S.m > 0) {
-        if (plan->policy != SPWS_DENSE && plan->policy != SPWS_HASH) {
-            CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG8, -1, S.A, S.B, rowptr, nullptr, nullptr));
-            CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG16, -1, S.A, S.B, rowptr, nullptr, nullptr));
-            CUDA_TRY(launch_ism_reg(c, false, CLS_ISM_REG, -1, S.A, S.B, rowptr, nullptr, nullptr));
-            mark(plan, SPWS_T_SYM_ISM_REG);
-            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        for (int cls = CLS_ISM_REG8; cls <= CLS_ISM_REG; ++cls)
+            if (hcount[cls] > 0) {
+                CUDA_TRY(launch_ism_reg(c, false, cls, hcount[cls], S.A, S.B, rowptr, nullptr, nullptr));
+                mark(plan, SPWS_T_SYM_ISM_REG);
+            }
+        if (hcount[CLS_ISM_SMEM_S] > 0) {
+            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, hcount[CLS_ISM_SMEM_S], S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_SMEM_S);
-            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        }
+        if (hcount[CLS_ISM_SMEM] > 0) {
+            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, hcount[CLS_ISM_SMEM], S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_SMEM);
         }
-        if (plan->policy != SPWS_SPARSE_ISM && plan->policy != SPWS_HASH) {
+        if (hcount[CLS_DENSE_WARP] > 0) {
             CUDA_TRY(launch_dense_sym_warp(c, S.A, S.B));
             mark(plan, SPWS_T_SYM_DENSE_WARP);
+        }
+        if (hcount[CLS_DENSE_HUB] + hcount[CLS_DENSE_CTA] > 0) {
             CUDA_TRY(launch_dense_sym_cta(c, S.A, S.B));
             mark(plan, SPWS_T_SYM_DENSE_CTA);
         }
-        if (plan->policy != SPWS_DENSE) {
-            CUDA_TRY(launch_ism_global(c, false, -1, S.A, S.B, rowptr, nullptr, nullptr));
+        if (hcount[CLS_ISM_GLOBAL] > 0) {
+            CUDA_TRY(launch_ism_global(c, false, hcount[CLS_ISM_GLOBAL], S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_GLOBAL);
         }
-        if (plan->policy == SPWS_HASH) {
-            CUDA_TRY(launch_hash(c, false, CLS_HASH_S, -1, S.A, S.B, rowptr, nullptr, nullptr));
-            CUDA_TRY(launch_hash(c, false, CLS_HASH, -1, S.A, S.B, rowptr, nullptr, nullptr));
-            mark(plan, SPWS_T_SYM_HASH);
-        }
+        for (int cls = CLS_HASH_S; cls <= CLS_HASH; ++cls)
+            if (hcount[cls] > 0) {
+                CUDA_TRY(launch_hash(c, false, cls, hcount[cls], S.A, S.B, rowptr, nullptr, nullptr));
+                mark(plan, SPWS_T_SYM_HASH);
+            }
     }
     // a4: exclusive scan into the row pointer
     CUDA_TRY(launch_scan_counts(c, c.tab.cnt, (int)S.m, rowptr, reinterpret_cast<i64*>(sc + L.block_sums), &c.ctl->nnz));
@@ -1004,7 +1014,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
                                     reinterpret_cast<int*>(sc + L.sflags), reinterpret_cast<i64*>(sc + L.spos),
                                     reinterpret_cast<i64*>(sc + L.block_sums), LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
     }
-    if (plan->policy != SPWS_SPARSE_ISM && plan->policy != SPWS_HASH) CUDA_TRY(launch_dense_rebin(c, (int)S.m, rowptr));
+    if (hcount[CLS_DENSE_WARP] + hcount[CLS_DENSE_HUB] + hcount[CLS_DENSE_CTA] > 0) CUDA_TRY(launch_dense_rebin(c, (int)S.m, rowptr));
     CUDA_TRY(launch_class_nnz(c, (int)S.m));
     mark(plan, SPWS_T_SYM_SCAN);
     CUDA_TRY(cudaMemcpyAsync(plan->host_ctl, c.ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost, stream));
@@ -1072,7 +1082,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     const spws_stats_t& s = plan->stats;
     int* crd = C->crd[last];
     const int64_t* bins = plan->bin_rows;
-    for (int cls = CLS_ISM_REG8; cls <= CLS_ISM_REG; ++cls)
+    for (int cls : {(int)CLS_COPY8, (int)CLS_ISM_REG8, (int)CLS_ISM_REG16, (int)CLS_ISM_REG})
         if (bins[cls] > 0) {
             CUDA_TRY(launch_ism_reg(c, true, cls, (int)bins[cls], S.A, S.B, rowptr, crd, C->val));
             mark(plan, SPWS_T_NUM_ISM_REG);
