@@ -62,6 +62,7 @@ struct DevCtl {
     i64 products;
     i64 max_ub;
     i64 max_ub_global;      // largest product count among CLS_ISM_GLOBAL rows
+    i64 max_ub_smem;        // largest product count among CLS_ISM_SMEM rows (sizes that kernel's launch)
     i64 kept[2];            // TTM: surviving slices (level 0) and fibres (level 1)
     u64 bm_words_used;      // words handed out of the bitmap arena
     int status;
@@ -204,6 +205,7 @@ struct LaunchCtx {
     char* rest;              // scratch after the fixed tables: bitmap arena, then the ISM-global arena
     size_t rest_bytes;
     int global_cap;          // accumulation-array capacity of CLS_ISM_GLOBAL
+    i64 max_ub_smem;         // largest product count of a CLS_ISM_SMEM row when known (0: unknown)
     uint2* bw;               // word lists of long B rows, indexed like B's entries (null: not built)
     int* bw_long;            // the long B rows, in arrival order
     int bw_long_cap;

@@ -182,7 +182,10 @@ static cudaError_t launch_cap(const LaunchCtx& c, bool numeric, int cls, int n_h
 template <typename T>
 static cudaError_t launch_t(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                             const i64* rowptr, int* Ccrd, void* Cval) {
-    const int cap = (cls == CLS_ISM_SMEM_S) ? c.prm.smem_small_cap : c.prm.smem_cap;
+    // the full class is launched for the largest row it actually holds when that is known: a
+    // smaller accumulation array means more CTAs per SM and cheaper barriers
+    int cap = (cls == CLS_ISM_SMEM_S) ? c.prm.smem_small_cap : c.prm.smem_cap;
+    if (cls == CLS_ISM_SMEM && c.max_ub_smem > 0 && c.max_ub_smem < cap) cap = (int)c.max_ub_smem;
     if (cap <= 64) return launch_cap<T, 64, 64>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
     if (cap <= 256) return launch_cap<T, 256, 64>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
     if (cap <= 1024) return launch_cap<T, 1024, 128>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);

@@ -83,17 +83,17 @@ template <int G>
 __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl) {
     __shared__ int s_hist[NCLASS];
     __shared__ i64 s_cprod[NCLASS];
-    __shared__ i64 s_products, s_max_ub, s_max_ub_global;
+    __shared__ i64 s_products, s_max_ub, s_max_ub_global, s_max_ub_smem;
     __shared__ int s_max_span_words;
     if (threadIdx.x < NCLASS) { s_hist[threadIdx.x] = 0; s_cprod[threadIdx.x] = 0; }
-    if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; s_max_span_words = 0; }
+    if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; s_max_ub_smem = 0; s_max_span_words = 0; }
     __syncthreads();
     const int gl = threadIdx.x % G;
     const unsigned lane = threadIdx.x & 31;
     const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane - gl));
     const i64 group = ((i64)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const i64 ngroups = ((i64)gridDim.x * blockDim.x) / G;
-    i64 my_products = 0, my_max = 0, my_max_global = 0;
+    i64 my_products = 0, my_max = 0, my_max_global = 0, my_max_smem = 0;
     // rows and products of the class of this group's last rows: neighbouring rows mostly share a
     // class, so the shared-memory histogram is touched only when the class changes
     int run_cls = -1, run_rows = 0, my_span_words = 0;
@@ -175,6 +175,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             my_products += u;
             my_max = max(my_max, u);
             if (cls == CLS_ISM_GLOBAL) my_max_global = max(my_max_global, u);
+            if (cls == CLS_ISM_SMEM) my_max_smem = max(my_max_smem, u);
             if (cls == CLS_DENSE_HUB || cls == CLS_DENSE_CTA || cls == CLS_DENSE_WARP)
                 my_span_words = max(my_span_words, (hi - lo) / 32 + 1);
         }
@@ -187,6 +188,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
     if (gl == 0 && my_products) atomicAdd((u64*)&s_products, (u64)my_products);
     if (gl == 0 && my_max) atomicMax(&s_max_ub, my_max);
     if (gl == 0 && my_max_global) atomicMax(&s_max_ub_global, my_max_global);
+    if (gl == 0 && my_max_smem) atomicMax(&s_max_ub_smem, my_max_smem);
     __syncthreads();
     if (threadIdx.x < NCLASS && s_hist[threadIdx.x]) {
         atomicAdd(&ctl->class_count[threadIdx.x], s_hist[threadIdx.x]);
@@ -196,6 +198,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         if (s_products) atomicAdd((u64*)&ctl->products, (u64)s_products);
         if (s_max_ub) atomicMax(&ctl->max_ub, s_max_ub);
         if (s_max_ub_global) atomicMax(&ctl->max_ub_global, s_max_ub_global);
+        if (s_max_ub_smem) atomicMax(&ctl->max_ub_smem, s_max_ub_smem);
         if (s_max_span_words) atomicMax(&ctl->max_span_words, s_max_span_words);
     }
 }

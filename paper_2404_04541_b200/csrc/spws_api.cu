@@ -33,6 +33,7 @@ struct spws_plan_s {
     void* scratch = nullptr;
     int max_span_words = 0;     // widest dense bitmap of the last symbolic pass
     int max_warp_cnt = 0;       // most outputs of a warp-numeric row
+    int64_t max_ub_smem = 0;    // most products of a shared-memory ISM row
     int64_t bin_rows[NCLASS] = {};  // rows per internal class of the last symbolic pass
     // outer-product form: what the last symbolic pass decided
     int64_t outer_products = 0;
@@ -971,7 +972,10 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     // grids sized for them (a launch for an empty class costs as much as a small class's work)
     int* hcount = plan->host_ctl->class_count;
     CUDA_TRY(cudaMemcpyAsync(hcount, c.ctl->class_count, sizeof(int) * NCLASS, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaMemcpyAsync(&plan->host_ctl->max_ub_smem, &c.ctl->max_ub_smem, sizeof(i64), cudaMemcpyDeviceToHost, stream));
     CUDA_TRY(cudaStreamSynchronize(stream));
+    plan->max_ub_smem = plan->host_ctl->max_ub_smem;
+    c.max_ub_smem = plan->max_ub_smem;
     // a3: exact count per row through the workspace of its class
     i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<i64*>(sc + L.rowptr_raw);
     if (S.m > 0) {
@@ -1079,6 +1083,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     const i64* rowptr = (plan->kind == 0) ? LL(C->pos[1]) : reinterpret_cast<const i64*>(sc + L.rowptr_raw);
     CUDA_TRY(cudaMemsetAsync(c.ctl->work_counter, 0, sizeof(c.ctl->work_counter), c.stream));
     mark_start(plan, 1);
+    c.max_ub_smem = plan->max_ub_smem;
     const spws_stats_t& s = plan->stats;
     int* crd = C->crd[last];
     const int64_t* bins = plan->bin_rows;
