@@ -219,7 +219,8 @@ cudaError_t launch_bw_build(const LaunchCtx& c, const Csr& B);
 cudaError_t launch_bin_rows(const LaunchCtx& c, int m);
 cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr);
 cudaError_t launch_class_nnz(const LaunchCtx& c, int m);
-cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out);
+// as_flags: scan (cnt[i] > 0) instead of cnt[i]
+cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out, bool as_flags = false);
 cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
                                const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
                                i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2);

@@ -148,6 +148,53 @@ __global__ void __launch_bounds__(256) ism_reg_kernel(const int* __restrict__ pe
     }
 }
 
+// Rows with ONE A entry that picks a B row of at most 8 entries (the commonest fibre of a
+// hyper-sparse 3-tensor): the products are the picked B row itself, already sorted and free of
+// duplicates, so Insert, Sort and Merge are the identity and the row is copied out scaled.  Every
+// lane first walks one row's chain of dependent loads (row id, A range, A entry, B range, output
+// offset), 32 chains per warp in flight; then the warp copies the 32 rows together, eight lanes per
+// row and four rows per step.
+template <typename T>
+__global__ void __launch_bounds__(256) copy_rows_kernel(const int* __restrict__ perm, const DevCtl* __restrict__ ctl, Csr A, Csr B,
+                                                        const i64* __restrict__ rowptr, int* __restrict__ Ccrd, T* __restrict__ Cval) {
+    if (ctl->status != 0) return;
+    int off, n;
+    class_range(ctl, CLS_COPY8, off, n);
+    const int* __restrict__ rows = perm + off;
+    const int lane = threadIdx.x & 31;
+    const T* __restrict__ Aval = (const T*)A.val;
+    const T* __restrict__ Bval = (const T*)B.val;
+    const i64 stride = (i64)gridDim.x * blockDim.x;
+    for (i64 r0 = ((i64)blockIdx.x * blockDim.x + threadIdx.x) - lane; r0 < n; r0 += stride) {
+        const i64 r = r0 + lane;
+        i64 qs = 0, out = 0;
+        int len = 0;
+        T a = 0;
+        if (r < n) {
+            const int row = __ldg(rows + r);
+            const i64 p = __ldg(A.pos + row);
+            const int k = __ldg(A.crd + p);
+            a = __ldg(Aval + p);
+            out = __ldg(rowptr + row);
+            if ((unsigned)k < (unsigned)B.nrows) {
+                qs = __ldg(B.pos + k);
+                len = min((int)(__ldg(B.pos + k + 1) - qs), 8);
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            const int src = 4 * s + (lane >> 3), e = lane & 7;
+            const i64 q = __shfl_sync(0xffffffffu, qs, src), o = __shfl_sync(0xffffffffu, out, src);
+            const int l = __shfl_sync(0xffffffffu, len, src);
+            const T av = __shfl_sync(0xffffffffu, a, src);
+            if (e < l) {
+                Ccrd[o + e] = __ldg(B.crd + q + e);
+                Cval[o + e] = mul_rn(av, __ldg(Bval + q + e));
+            }
+        }
+    }
+}
+
 template <typename T, int G>
 static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                             const i64* rowptr, int* Ccrd, void* Cval) {
@@ -169,6 +216,15 @@ static cudaError_t launch_g(const LaunchCtx& c, bool numeric, int cls, int n_hos
 
 cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                            const i64* rowptr, int* Ccrd, void* Cval) {
+    if (cls == CLS_COPY8 && numeric) {
+        const i64 rows = n_host >= 0 ? n_host : A.nrows;
+        i64 want = (rows + 255) / 256, cap = (i64)c.sm_count * 16;
+        const int grid = (int)(want < 1 ? 1 : (want < cap ? want : cap));
+        if (c.is_f64) copy_rows_kernel<double><<<grid, 256, 0, c.stream>>>(c.tab.perm, c.ctl, A, B, rowptr, Ccrd, (double*)Cval);
+        else copy_rows_kernel<float><<<grid, 256, 0, c.stream>>>(c.tab.perm, c.ctl, A, B, rowptr, Ccrd, (float*)Cval);
+        ++c.launches;
+        return cudaGetLastError();
+    }
     if (c.is_f64) {
         if (cls == CLS_ISM_REG8 || cls == CLS_COPY8) return launch_g<double, 8>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);
         if (cls == CLS_ISM_REG16) return launch_g<double, 16>(c, numeric, cls, n_host, A, B, rowptr, Ccrd, Cval);

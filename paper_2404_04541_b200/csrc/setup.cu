@@ -212,6 +212,8 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
         i64 cap = (i64)c.sm_count * 16;
         return (int)(want < cap ? want : cap);
     };
+    // (one and two lanes per row were measured on the fibre matrix of the 3-tensor workload, 1.06
+    // entries per row: slower than four)
     if (avg <= 6.0) row_bounds_kernel<4><<<grid_for(4), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
     else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
     else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
@@ -485,13 +487,15 @@ constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_ITEMS = 8;
 constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
 
+// FLAG: scan (in[i] > 0) instead of in[i] (compaction positions without a flag array).
+template <bool FLAG>
 __global__ void __launch_bounds__(SCAN_THREADS) scan_reduce_kernel(const int* __restrict__ in, int n, i64* block_sums) {
     __shared__ i64 s_part[SCAN_THREADS / 32];
     const i64 base = (i64)blockIdx.x * SCAN_TILE;
     i64 s = 0;
     for (int x = 0; x < SCAN_ITEMS; ++x) {
         const i64 i = base + x * SCAN_THREADS + threadIdx.x;
-        if (i < n) s += in[i];
+        if (i < n) s += FLAG ? (in[i] > 0) : in[i];
     }
     for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
     if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = s;
@@ -542,6 +546,7 @@ __global__ void __launch_bounds__(1024) scan_block_sums_kernel(i64* block_sums, 
 }
 
 // The in-tile prefix is carried in 64 bits: a tile of 2048 counts may total 2^31 or more.
+template <bool FLAG>
 __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int* __restrict__ in, int n, const i64* __restrict__ block_sums, i64* __restrict__ out) {
     __shared__ i64 s_warp[SCAN_THREADS / 32];
     const i64 base = (i64)blockIdx.x * SCAN_TILE + (i64)threadIdx.x * SCAN_ITEMS;
@@ -550,7 +555,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int* __r
     i64 s = 0;
 #pragma unroll
     for (int x = 0; x < SCAN_ITEMS; ++x) {
-        v[x] = (base + x < n) ? in[base + x] : 0;
+        v[x] = (base + x < n) ? (FLAG ? (in[base + x] > 0) : in[base + x]) : 0;
         s += v[x];
     }
     i64 incl = s;
@@ -572,11 +577,17 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int* __r
     }
 }
 
-cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out) {
+cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out, bool as_flags) {
     const int nblocks = (int)(((i64)n + SCAN_TILE - 1) / SCAN_TILE);
-    if (nblocks > 0) scan_reduce_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums);
+    if (nblocks > 0) {
+        if (as_flags) scan_reduce_kernel<true><<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums);
+        else scan_reduce_kernel<false><<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums);
+    }
     scan_block_sums_kernel<<<1, 1024, 0, c.stream>>>(block_sums, nblocks, out + n, total_out);
-    if (nblocks > 0) scan_apply_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums, out);
+    if (nblocks > 0) {
+        if (as_flags) scan_apply_kernel<true><<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums, out);
+        else scan_apply_kernel<false><<<nblocks, SCAN_THREADS, 0, c.stream>>>(cnt, n, block_sums, out);
+    }
     c.launches += nblocks > 0 ? 3 : 1;
     return cudaGetLastError();
 }
@@ -585,17 +596,12 @@ cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* o
 // TTM: rebuild C's two upper CSF levels.  A fibre (i,j) survives when it produced at least
 // one output; a slice i survives when one of its fibres does.
 // ---------------------------------------------------------------------------------------
-__global__ void ttm_fibre_flags_kernel(int n_ij, const int* __restrict__ cnt, int* flags) {
-    for (i64 f = (i64)blockIdx.x * blockDim.x + threadIdx.x; f < n_ij; f += (i64)gridDim.x * blockDim.x)
-        flags[f] = cnt[f] > 0;
-}
-
-__global__ void ttm_fibre_compact_kernel(int n_ij, const int* __restrict__ flags, const i64* __restrict__ fpos,
+__global__ void ttm_fibre_compact_kernel(int n_ij, const int* __restrict__ cnt, const i64* __restrict__ fpos,
                                          const int* __restrict__ Acrd1, const i64* __restrict__ rowptr_raw,
                                          int* Ccrd1, i64* Cpos2) {
     for (i64 f = (i64)blockIdx.x * blockDim.x + threadIdx.x; f <= n_ij; f += (i64)gridDim.x * blockDim.x) {
         if (f == n_ij) { Cpos2[fpos[n_ij]] = rowptr_raw[n_ij]; continue; }
-        if (flags[f]) {
+        if (cnt[f] > 0) {
             Ccrd1[fpos[f]] = Acrd1[f];
             Cpos2[fpos[f]] = rowptr_raw[f];
         }
@@ -626,19 +632,58 @@ __global__ void ttm_slice_compact_kernel(int n_i, int n_ij, const int* __restric
     }
 }
 
+// The slice level in ONE launch when it is small: a single block flags, scans and compacts the
+// slices 1024 at a time with a running count.
+__global__ void __launch_bounds__(1024) ttm_slices_small_kernel(int n_i, int n_ij, const i64* __restrict__ Apos1, const i64* __restrict__ fpos,
+                                                                const int* __restrict__ Acrd0, int* Ccrd0, i64* Cpos1, i64* Cpos0,
+                                                                DevCtl* ctl) {
+    __shared__ int ws[33];
+    int kept = 0;
+    for (int s0 = 0; s0 < n_i; s0 += 1024) {
+        const int s = s0 + threadIdx.x;
+        i64 first = 0;
+        int flag = 0;
+        if (s < n_i) {
+            first = fpos[Apos1[s]];
+            flag = fpos[Apos1[s + 1]] > first;
+        }
+        int total;
+        const int at = kept + block_excl_scan<1024>(flag, ws, total);
+        if (flag) {
+            Ccrd0[at] = Acrd0[s];
+            Cpos1[at] = first;
+        }
+        kept += total;
+    }
+    if (threadIdx.x == 0) {
+        Cpos1[kept] = fpos[n_ij];
+        Cpos0[0] = 0;
+        Cpos0[1] = kept;
+        ctl->kept[0] = kept;
+        ctl->kept[1] = fpos[n_ij];
+    }
+}
+
 cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
                                const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
                                i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2) {
+    (void)flags;
     const int grid = c.sm_count * 8;
-    if (n_ij > 0) ttm_fibre_flags_kernel<<<grid, 256, 0, c.stream>>>(n_ij, c.tab.cnt, flags);
-    cudaError_t e = launch_scan_counts(c, flags, n_ij, fpos, block_sums, nullptr);
+    // fibres that produced an output keep their place among the survivors: positions by a scan of (cnt > 0)
+    cudaError_t e = launch_scan_counts(c, c.tab.cnt, n_ij, fpos, block_sums, nullptr, true);
     if (e != cudaSuccess) return e;
-    ttm_fibre_compact_kernel<<<grid, 256, 0, c.stream>>>(n_ij, flags, fpos, Acrd1, rowptr_raw, Ccrd1, Cpos2);
-    if (n_i > 0) ttm_slice_flags_kernel<<<grid, 256, 0, c.stream>>>(n_i, Apos1, fpos, sflags);
+    ttm_fibre_compact_kernel<<<grid, 256, 0, c.stream>>>(n_ij, c.tab.cnt, fpos, Acrd1, rowptr_raw, Ccrd1, Cpos2);
+    ++c.launches;
+    if (n_i <= (1 << 16)) {
+        ttm_slices_small_kernel<<<1, 1024, 0, c.stream>>>(n_i, n_ij, Apos1, fpos, Acrd0, Ccrd0, Cpos1, Cpos0, c.ctl);
+        ++c.launches;
+        return cudaGetLastError();
+    }
+    ttm_slice_flags_kernel<<<grid, 256, 0, c.stream>>>(n_i, Apos1, fpos, sflags);
     e = launch_scan_counts(c, sflags, n_i, spos, block_sums, nullptr);
     if (e != cudaSuccess) return e;
     ttm_slice_compact_kernel<<<grid, 256, 0, c.stream>>>(n_i, n_ij, sflags, spos, Apos1, fpos, Acrd0, Ccrd0, Cpos1, Cpos0, c.ctl);
-    c.launches += 2 + (n_ij > 0) + (n_i > 0);
+    c.launches += 2;
     return cudaGetLastError();
 }
 
