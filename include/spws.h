@@ -25,7 +25,7 @@
  * and the all array in the scratch buffer) under SPWS_SPARSE_ISM, an I x J value array with
  * flags under SPWS_DENSE (SPWS_WORKSPACE_TOO_LARGE when the scratch given cannot hold it: the
  * paper's dense workspace running out of memory, Sec. 7.2), and under SPWS_AUTO the dense one
- * when it fits and the products number at least I*J/16.  The last three are the higher-order
+ * when it fits and either I*J <= 2^27 or the products number at least I*J/16.  The last three are the higher-order
  * scatters of Sec. 7.3 (sparse output in coordinate form): their workspace is the sparse one on
  * integer labels over all scattered output indices (third order for SpTTM); no dense workspace
  * is offered for them (SPWS_DENSE: SPWS_WORKSPACE_TOO_LARGE at plan creation).
@@ -252,7 +252,8 @@ spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A
  * C->pos[] must be allocated by the caller: CSR: pos[1] with dims[0]+1 entries;
  * CSF3: pos[0] (2), crd[0] (A->n[0]), pos[1] (A->n[0]+1), crd[1] (A->n[1]), pos[2] (A->n[1]+1),
  * i.e. the sizes of A's upper levels, which bound C's.  On return C->n[] holds the result sizes
- * and `sizes_out` (host, 3 entries, may be NULL) a copy.  Synchronises the stream once, to read
+ * and `sizes_out` (host, 3 entries, may be NULL) a copy.  Synchronises the stream twice: after
+ * binning, to learn which workspaces have rows (only those are launched), and at the end, to read
  * the sizes back. */
 spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws_tensor_t* B,
                             spws_tensor_t* C, void* scratch, size_t scratch_bytes,

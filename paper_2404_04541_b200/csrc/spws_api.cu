@@ -414,7 +414,9 @@ bool outer_wants_dense(const spws_plan_s* p, int64_t I, int64_t J, int64_t P, si
         return true;
     }
     if (p->policy == SPWS_SPARSE_ISM || p->policy == SPWS_HASH) return false;
-    return fits && (double)P * 16.0 >= (double)I * (double)J;
+    // measured on B200 (I = J = 10^4): the dense workspace wins from the smallest product count on,
+    // so it is taken whenever it is small in absolute terms or next to the work
+    return fits && ((double)I * (double)J <= 134217728.0 || (double)P * 16.0 >= (double)I * (double)J);
 }
 
 spws_status_t outer_symbolic(spws_plan_s* plan, const Shapes& S, spws_tensor_t* C, void* scratch, size_t scratch_bytes, int64_t* sizes_out) {
@@ -889,7 +891,7 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
         const size_t dense_ok = (double)S.m * (double)S.ncols <= 2.0e9 ? OL.dense_end : 0;     // a dense workspace beyond 2^31 cells is never offered
         *bytes = (plan->policy == SPWS_SPARSE_ISM || plan->policy == SPWS_HASH) ? OL.ism_end
                  : plan->policy == SPWS_DENSE ? OL.dense_end
-                 : std::max(OL.ism_end, (double)P * 16.0 >= (double)S.m * (double)S.ncols ? dense_ok : (size_t)0);
+                 : std::max(OL.ism_end, ((double)S.m * (double)S.ncols <= 134217728.0 || (double)P * 16.0 >= (double)S.m * (double)S.ncols) ? dense_ok : (size_t)0);
         return SPWS_OK;
     }
     const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
