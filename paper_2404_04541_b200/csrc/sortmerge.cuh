@@ -22,7 +22,8 @@ static int grid_for(const LaunchCtx& c, i64 work_items, int per_block) {
 // A block owns a tile of RS_TILE consecutive elements; warp w of the block owns the w-th
 // contiguous slice of the tile and walks it 32 elements at a time, so "block, warp, step, lane"
 // is the input order.  Pass = histogram per (digit, block) -> exclusive scan over (digit major,
-// block minor) -> scatter with the element's rank among equal digits before it.
+// block minor) -> scatter with the element's rank among equal digits before it; the tile is put in
+// digit order in shared memory first, so every digit's elements leave as one contiguous run.
 constexpr int RS_THREADS = 256;
 constexpr int RS_WARPS = RS_THREADS / 32;
 constexpr int RS_STEPS = 8;                             // 32-element steps per warp
@@ -44,7 +45,12 @@ template <typename T, bool VALUES>
 __global__ void __launch_bounds__(RS_THREADS) radix_scatter_kernel(const u64* __restrict__ keys, const T* __restrict__ vals, i64 n,
                                                                   int shift, int nblocks, const i64* __restrict__ offs,
                                                                   u64* __restrict__ keys_out, T* __restrict__ vals_out) {
-    __shared__ int s_cnt[RS_WARPS][256];        // elements with the digit in this warp's slice, then their start inside the tile
+    __shared__ int s_cnt[RS_WARPS][256];        // elements with the digit in this warp's slice, then their start inside the digit's part
+    __shared__ int s_start[256];                // start of the digit's part inside the tile
+    __shared__ i64 s_goff[256];
+    __shared__ int s_ws[33];
+    __shared__ u64 s_key[RS_TILE];
+    __shared__ T s_val[VALUES ? RS_TILE : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int d = lane; d < 256; d += 32) s_cnt[warp][d] = 0;
     __syncwarp();
@@ -70,11 +76,17 @@ __global__ void __launch_bounds__(RS_THREADS) radix_scatter_kernel(const u64* __
         __syncwarp();
     }
     __syncthreads();
-    // start of each warp's share of a digit = global start of (digit, block) + earlier warps' counts
+    // start of each warp's share of a digit inside the digit's part of the tile, and the start of
+    // every digit's part inside the tile (the tile is first put in digit order in shared memory,
+    // so that each digit's elements leave as one contiguous run)
+    int tile_total;
     {
         const int d = threadIdx.x;                       // RS_THREADS == 256 digits
         int run = 0;
         for (int w = 0; w < RS_WARPS; ++w) { const int c = s_cnt[w][d]; s_cnt[w][d] = run; run += c; }
+        const int start = block_excl_scan<RS_THREADS>(run, s_ws, tile_total);
+        s_start[d] = start;
+        s_goff[d] = offs[(i64)d * nblocks + blockIdx.x] - start;     // global position of staged slot i of digit d = s_goff[d] + i
     }
     __syncthreads();
 #pragma unroll
@@ -82,10 +94,17 @@ __global__ void __launch_bounds__(RS_THREADS) radix_scatter_kernel(const u64* __
         const i64 t = base + st * 32 + lane;
         if (t < n) {
             const unsigned d = (unsigned)(key[st] >> shift) & 255u;
-            const i64 at = offs[(i64)d * nblocks + blockIdx.x] + s_cnt[warp][d] + rank[st];
-            keys_out[at] = key[st];
-            if (VALUES) vals_out[at] = vals[t];
+            const int at = s_start[d] + s_cnt[warp][d] + rank[st];
+            s_key[at] = key[st];
+            if (VALUES) s_val[at] = vals[t];
         }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < tile_total; i += RS_THREADS) {
+        const u64 k = s_key[i];
+        const i64 at = s_goff[(unsigned)(k >> shift) & 255u] + i;
+        keys_out[at] = k;
+        if (VALUES) vals_out[at] = s_val[i];
     }
 }
 
