@@ -234,8 +234,8 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
 /* The scratch bytes spws_symbolic + spws_numeric really use for these operands, found by running
  * the first two steps of the symbolic pass (per-row product bound and span, binning; Sec. 5.4's
  * "balance workloads" needs them anyway): the fixed tables, the occupancy bitmaps of exactly the
- * rows routed to the dense workspace over exactly their spans, and up to eight all-array slots of
- * the global-memory ISM sized for its largest row.  Two steps: with scratch = NULL the call writes to *bytes the size of the
+ * rows routed to the dense workspace over exactly their spans, and the all-array slots of the
+ * global-memory ISM (one per CTA it keeps busy, sized for its largest row, 2 GiB at most).  Two steps: with scratch = NULL the call writes to *bytes the size of the
  * buffer it needs itself (host only, no launch); with such a buffer (DEVICE, 256-byte aligned) it
  * runs the two kernels on the plan's stream, synchronises and writes the exact size.
  * `row_products` (DEVICE, int64, one entry per output row / input fibre; may be NULL) receives the

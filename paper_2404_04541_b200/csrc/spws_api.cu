@@ -205,8 +205,19 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, 
     return L;
 }
 
+// All-array slots the global-memory ISM is given: one per CTA it can keep busy (two per SM), but
+// no more than rows of that class and no more than fit 2 GiB; eight at least.
+size_t global_ism_slots(const spws_plan_s* p, size_t slot_bytes, int64_t rows) {
+    size_t slots = 2 * (size_t)p->h->sm_count;
+    const size_t fit = slot_bytes ? ((size_t)2 << 30) / slot_bytes : slots;
+    if (slots > fit) slots = fit;
+    if (slots < 8) slots = 8;
+    if ((int64_t)slots > rows) slots = (size_t)(rows > 0 ? rows : 1);
+    return slots;
+}
+
 // what follows the fixed tables: one bitmap per row in the worst case (dense routes), and room
-// for a few slots of min(ncols, 2^22) components for the global-memory ISM
+// for the all-array slots of the global-memory ISM at min(ncols, 2^22) components each
 size_t rest_reserve(const spws_plan_s* p, int64_t m, int64_t ncols) {
     size_t bytes = 0;
     if (p->policy != SPWS_SPARSE_ISM && p->policy != SPWS_HASH) {
@@ -219,9 +230,10 @@ size_t rest_reserve(const spws_plan_s* p, int64_t m, int64_t ncols) {
         // slot a row over all ncols columns needs in the numeric pass
         const int64_t elems = ncols < (1ll << 22) ? ncols : (1ll << 22);
         const size_t comp = 4 + (p->is_f64 ? 8 : 4);
-        const size_t eight = align256(2 * (size_t)((elems + 63) & ~63ll) * comp) * 8;
+        const size_t slot = align256(2 * (size_t)((elems + 63) & ~63ll) * comp);
         const size_t one_full = align256(2 * (size_t)((ncols + 63) & ~63ll) * comp);
-        bytes += eight > one_full ? eight : one_full;
+        const size_t many = slot * global_ism_slots(p, slot, 0x7fffffff);
+        bytes += many > one_full ? many : one_full;
     }
     return bytes;
 }
@@ -928,11 +940,12 @@ spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A
     if (hc.status != 0 && hc.status != DEV_SCRATCH_TOO_SMALL) return from_dev_status(hc.status);
     size_t need = L.fixed_end + align256((size_t)hc.bm_words_used * 4);
     const int64_t n_global = hc.class_count[CLS_ISM_GLOBAL];
-    if (n_global > 0) {                         // numeric slots of the global-memory ISM: one per row, eight at most
+    if (n_global > 0) {                         // numeric slots of the global-memory ISM, sized for its largest row
         int64_t elems = hc.max_ub_global < S.ncols ? hc.max_ub_global : S.ncols;
         elems = (elems + 63) & ~63ll;
         const size_t comp = 4 + (plan->is_f64 ? 8 : 4);
-        need += align256(2 * (size_t)elems * comp) * (size_t)(n_global < 8 ? n_global : 8);
+        const size_t slot = align256(2 * (size_t)elems * comp);
+        need += slot * global_ism_slots(plan, slot, n_global);
     }
     *bytes = need;
     return SPWS_OK;
