@@ -15,8 +15,8 @@
  *
  * following the paper's statement of the problem: an expression over named index variables
  * (Sec. 3), a level format per operand (Sec. 2.1, Fig. 4) and a workspace policy (Sec. 6.1:
- * the workspace tensor's format and policy; Sec. 6.2: dense-workspace optimisation).  Both
- * expressions are first-order scatters (Sec. 2.2): the loop order i -> k -> j differs from the
+ * the workspace tensor's format and policy; Sec. 6.2: dense-workspace optimisation).  The first
+ * two expressions are first-order scatters (Sec. 2.2): the loop order i -> k -> j differs from the
  * output order i -> j only by the reduction variable, so every output row (every (i,j) fibre,
  * after hoisting the shared outer loops, Sec. 6.2) owns a first-order workspace along the last
  * index.  The third expression is the paper's running example (Sec. 2.1): the reduction variable is
@@ -25,8 +25,8 @@
  * and the all array in the scratch buffer) under SPWS_SPARSE_ISM, an I x J value array with
  * flags under SPWS_DENSE (SPWS_WORKSPACE_TOO_LARGE when the scratch given cannot hold it: the
  * paper's dense workspace running out of memory, Sec. 7.2), and under SPWS_AUTO the dense one
- * when it fits and either I*J <= 2^27 or the products number at least I*J/16.  The last three are the higher-order
- * scatters of Sec. 7.3 (sparse output in coordinate form): their workspace is the sparse one on
+ * when it fits and either I*J <= 2^27 or the products number at least I*J/16.  The last three are
+ * the higher-order scatters of Sec. 7.3 (sparse output in coordinate form): their workspace is the sparse one on
  * integer labels over all scattered output indices (third order for SpTTM); no dense workspace
  * is offered for them (SPWS_DENSE: SPWS_WORKSPACE_TOO_LARGE at plan creation).
  *
