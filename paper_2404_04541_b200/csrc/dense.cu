@@ -56,12 +56,19 @@ __device__ __forceinline__ int pick_group_size(i64 ub, i64 entries, int parts) {
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __restrict__ ctl, Csr A, Csr B, RowTables tab) {
     __shared__ unsigned s_bm[DW_WARPS][DENSE_WARP_BM_WORDS];
+    // bit w of the summary = bitmap word w is non-empty, so the copy-out walks only those words
+    __shared__ unsigned s_sum[DW_WARPS][DENSE_WARP_BM_WORDS / 32];
+    // descriptors of 32 A entries: (start of the B row << 16) | its length (a warp row has <= 4096 products)
+    __shared__ __align__(16) u64 s_desc[DW_WARPS][32];
     if (ctl->status != 0) return;
     int off, n;
     class_range(ctl, CLS_DENSE_WARP, off, n);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned* bm = s_bm[warp];
+    unsigned* sum = s_sum[warp];
+    u64* desc = s_desc[warp];
     for (int w = lane; w < DENSE_WARP_BM_WORDS; w += 32) bm[w] = 0;     // every row leaves its bitmap clear
+    sum[lane] = 0;
     __syncwarp();
     for (;;) {
         int r = 0;
@@ -74,37 +81,53 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
         const unsigned span = (unsigned)nw * 32u;
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         const int gs = pick_group_size(tab.ub[row], pe - ps, 1);
+        // the lane that sets a bit first counts the output; the lane that touches a word first
+        // counts the word and flags it in the summary
+        int cnt = 0, nzw = 0;
+        auto mark = [&](unsigned rel) {
+            if (rel < span) {
+                const unsigned w = rel >> 5, bit = 1u << (rel & 31);
+                const unsigned old = atomicOr(&bm[w], bit);
+                if (!(old & bit)) {
+                    ++cnt;
+                    if (old == 0u) { ++nzw; atomicOr(&sum[w >> 5], 1u << (w & 31)); }
+                }
+            }
+        };
         if (gs == 32) {
-            // descriptors of 32 A entries at a time (one per lane), then the first 32 elements of
-            // four B rows are loaded before any is consumed, to keep loads in flight
+            // descriptors of 32 A entries at a time (one per lane, passed through shared memory), then
+            // the first 32 elements of four B rows are loaded before any is consumed, to keep loads
+            // in flight
             for (i64 p0 = ps; p0 < pe; p0 += 32) {
-                i64 my_qs = 0;
-                int my_len = 0;
+                u64 mine = 0;
                 if (p0 + lane < pe) {
                     const int k = __ldg(A.crd + p0 + lane);
                     if ((unsigned)k < (unsigned)B.nrows) {
-                        my_qs = __ldg(B.pos + k);
-                        my_len = (int)(__ldg(B.pos + k + 1) - my_qs);
+                        const i64 qs = __ldg(B.pos + k);
+                        mine = ((u64)qs << 16) | (u64)(__ldg(B.pos + k + 1) - qs);
                     }
                 }
+                __syncwarp();
+                desc[lane] = mine;
+                __syncwarp();
                 const int nE = (int)min((i64)32, pe - p0);
                 for (int e = 0; e < nE; e += 4) {
+                    const ulonglong2 d01 = *reinterpret_cast<const ulonglong2*>(desc + e);
+                    const ulonglong2 d23 = *reinterpret_cast<const ulonglong2*>(desc + e + 2);
+                    const u64 d[4] = {d01.x, d01.y, d23.x, d23.y};
                     i64 qs[4];
                     int len[4];
                     unsigned rel[4];
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
-                        qs[x] = __shfl_sync(0xffffffffu, my_qs, (e + x) & 31);
-                        len[x] = (e + x < nE) ? __shfl_sync(0xffffffffu, my_len, (e + x) & 31) : 0;
+                        qs[x] = (i64)(d[x] >> 16);
+                        len[x] = (int)(d[x] & 0xffffu);                  // 0 past the last entry
                         rel[x] = (lane < len[x]) ? (unsigned)(__ldg(B.crd + qs[x] + lane) - base) : 0xffffffffu;
                     }
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
-                        if (rel[x] < span) atomicOr(&bm[rel[x] >> 5], 1u << (rel[x] & 31));
-                        for (int t = lane + 32; t < len[x]; t += 32) {
-                            const unsigned r2 = (unsigned)(__ldg(B.crd + qs[x] + t) - base);
-                            if (r2 < span) atomicOr(&bm[r2 >> 5], 1u << (r2 & 31));
-                        }
+                        mark(rel[x]);
+                        for (int t = lane + 32; t < len[x]; t += 32) mark((unsigned)(__ldg(B.crd + qs[x] + t) - base));
                     }
                 }
             }
@@ -116,41 +139,34 @@ __global__ void __launch_bounds__(DW_THREADS) dense_sym_warp_kernel(DevCtl* __re
                 const i64 qs = __ldg(B.pos + k);
                 const int len = (int)(__ldg(B.pos + k + 1) - qs);
                 const int* __restrict__ ck = B.crd + qs;
-                for (int t = gl; t < len; t += gs) {
-                    const unsigned rel = (unsigned)(__ldg(ck + t) - base);
-                    if (rel < span) atomicOr(&bm[rel >> 5], 1u << (rel & 31));
-                }
+                for (int t = gl; t < len; t += gs) mark((unsigned)(__ldg(ck + t) - base));
             }
         }
-        __syncwarp();
-        // outputs and non-empty words of the row
-        int cnt = 0, nzw = 0;
-        for (int w0 = 0; w0 < nw; w0 += 32) {
-            const int w = w0 + lane;
-            const unsigned word = (w < nw) ? bm[w] : 0u;
-            cnt += __popc(word);
-            nzw += __popc(__ballot_sync(0xffffffffu, word != 0u));
+        for (int d = 16; d > 0; d >>= 1) {
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+            nzw += __shfl_xor_sync(0xffffffffu, nzw, d);
         }
-        for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+        __syncwarp();
         const i64 slot = tab.bm_off[row];
         unsigned* out = tab.bm_arena + slot;
         if (cnt <= DENSE_WARP_ACC && 2 * nzw <= nw + chunks_of(nw)) {
-            // compact form for the warp numeric kernel: only the non-empty words, as (bits, word index)
+            // compact form for the warp numeric kernel: only the non-empty words, as (bits, word
+            // index) in column order; lane l owns the words its summary word flags
             uint2* out2 = reinterpret_cast<uint2*>(out);
-            int at = 0;
-            for (int w0 = 0; w0 < nw; w0 += 32) {
-                const int w = w0 + lane;
-                const unsigned word = (w < nw) ? bm[w] : 0u;
-                const unsigned ball = __ballot_sync(0xffffffffu, word != 0u);
-                if (word != 0u) {
-                    out2[at + __popc(ball & ((1u << lane) - 1u))] = make_uint2(word, (unsigned)w);
-                    bm[w] = 0;
-                }
-                at += __popc(ball);
+            unsigned s = sum[lane];
+            sum[lane] = 0;
+            const int c = __popc(s);
+            int at = warp_incl_scan(c) - c;
+            while (s) {
+                const int w = (lane << 5) + __ffs(s) - 1;
+                s &= s - 1;
+                out2[at++] = make_uint2(bm[w], (unsigned)w);
+                bm[w] = 0;
             }
             if (lane == 0) tab.bm_off[row] = slot | ((i64)nzw << BM_NZW_SHIFT) | BM_COMPACT;
         } else {
             // full form: every word, then the rank at every 32-word chunk start
+            sum[lane] = 0;
             int carry = 0;
             for (int w0 = 0; w0 < nw; w0 += 32) {
                 const int w = w0 + lane;
