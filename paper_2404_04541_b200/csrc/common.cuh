@@ -209,6 +209,7 @@ struct LaunchCtx {
     uint2* bw;               // word lists of long B rows, indexed like B's entries (null: not built)
     int* bw_long;            // the long B rows, in arrival order
     int bw_long_cap;
+    int4* brow;                 // per B row: first column, last column, length (null: not kept)
     mutable int launches;    // kernels enqueued through this context
 };
 
@@ -221,9 +222,9 @@ cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr);
 cudaError_t launch_class_nnz(const LaunchCtx& c, int m);
 // as_flags: scan (cnt[i] > 0) instead of cnt[i]
 cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* out, i64* block_sums, i64* total_out, bool as_flags = false);
-cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
-                               const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
-                               i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2);
+cudaError_t launch_ttm_scan_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0, const int* Acrd1,
+                                    i64* rowptr_raw, i64* fpos, int* sflags, i64* spos, i64* block_sums, i64* nnz_out,
+                                    i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2);
 // class kernels: n_host < 0 means "size the grid for any count"
 cudaError_t launch_ism_reg(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B,
                            const i64* rowptr, int* Ccrd, void* Cval);

@@ -79,21 +79,42 @@ __device__ __forceinline__ int classify_row(i64 ub, i64 entries, int jmin, int j
     return CLS_ISM_GLOBAL;
 }
 
+// First column, last column and length of every B row, in one 16-byte record: when A has several
+// times more entries than B has rows, the bounds kernel reads the record of the row an entry picks
+// (one load, neighbouring rows share sectors) instead of two offsets and two coordinates.
+__global__ void __launch_bounds__(256) brow_summary_kernel(Csr B, int4* __restrict__ brow) {
+    for (i64 k = (i64)blockIdx.x * blockDim.x + threadIdx.x; k < B.nrows; k += (i64)gridDim.x * blockDim.x) {
+        const i64 qs = B.pos[k], qe = B.pos[k + 1];
+        int4 s = make_int4(0x7fffffff, -1, 0, 0);
+        if (qe > qs) {
+            s.x = __ldg(B.crd + qs);
+            s.y = __ldg(B.crd + qe - 1);
+            s.z = (int)min(qe - qs, (i64)0x7fffffff);
+        }
+        brow[k] = s;
+    }
+}
+
 template <int G>
-__global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl) {
-    __shared__ int s_hist[NCLASS];
-    __shared__ i64 s_cprod[NCLASS];
+__global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl,
+                                                         const int4* __restrict__ brow) {
+    // rows and products per class, one histogram per warp: 64-bit shared-memory adds are
+    // compare-and-swap loops, which many threads on one address turn into a queue
+    __shared__ int s_hist[8][NCLASS];
+    __shared__ i64 s_cprod[8][NCLASS];
     __shared__ i64 s_products, s_max_ub, s_max_ub_global, s_max_ub_smem;
     __shared__ int s_max_span_words;
-    if (threadIdx.x < NCLASS) { s_hist[threadIdx.x] = 0; s_cprod[threadIdx.x] = 0; }
+    for (int x = threadIdx.x; x < 8 * NCLASS; x += blockDim.x) { (&s_hist[0][0])[x] = 0; (&s_cprod[0][0])[x] = 0; }
     if (threadIdx.x == 0) { s_products = 0; s_max_ub = 0; s_max_ub_global = 0; s_max_ub_smem = 0; s_max_span_words = 0; }
     __syncthreads();
+    int* const w_hist = s_hist[threadIdx.x >> 5];
+    i64* const w_cprod = s_cprod[threadIdx.x >> 5];
     const int gl = threadIdx.x % G;
     const unsigned lane = threadIdx.x & 31;
     const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane - gl));
     const i64 group = ((i64)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const i64 ngroups = ((i64)gridDim.x * blockDim.x) / G;
-    i64 my_products = 0, my_max = 0, my_max_global = 0, my_max_smem = 0;
+    i64 my_products = 0, my_max = 0;
     // rows and products of the class of this group's last rows: neighbouring rows mostly share a
     // class, so the shared-memory histogram is touched only when the class changes
     int run_cls = -1, run_rows = 0, my_span_words = 0;
@@ -110,11 +131,18 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             if (p0 < pe) {
                 const int k = __ldg(A.crd + p0);
                 if ((unsigned)k < (unsigned)B.nrows) {
-                    const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
-                    if (qe > qs) {
-                        u = qe - qs;
-                        lo = __ldg(B.crd + qs);
-                        hi = __ldg(B.crd + qe - 1);
+                    if (brow) {
+                        const int4 s = __ldg(brow + k);
+                        u = s.z;
+                        lo = s.x;
+                        hi = s.y;
+                    } else {
+                        const i64 qs = __ldg(B.pos + k), qe = __ldg(B.pos + k + 1);
+                        if (qe > qs) {
+                            u = qe - qs;
+                            lo = __ldg(B.crd + qs);
+                            hi = __ldg(B.crd + qe - 1);
+                        }
                     }
                 } else {
                     bad = true;
@@ -130,6 +158,17 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
                 const i64 p = p0 + (i64)x * G;
                 k[x] = p < pe ? __ldg(A.crd + p) : -1;
                 if (p < pe && (unsigned)k[x] >= (unsigned)B.nrows) bad = true;
+            }
+            if (brow) {
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+                    if ((unsigned)k[x] < (unsigned)B.nrows) {
+                        const int4 s = __ldg(brow + k[x]);
+                        u += s.z;
+                        lo = min(lo, s.x);
+                        hi = max(hi, s.y);
+                    }
+                continue;
             }
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
@@ -163,8 +202,8 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             tab.cls[row] = (unsigned char)cls;
             if (cls != run_cls) {
                 if (run_rows) {
-                    atomicAdd(&s_hist[run_cls], run_rows);
-                    if (run_products) atomicAdd((u64*)&s_cprod[run_cls], (u64)run_products);
+                    atomicAdd(&w_hist[run_cls], run_rows);
+                    if (run_products) atomicAdd((u64*)&w_cprod[run_cls], (u64)run_products);
                 }
                 run_cls = cls;
                 run_rows = 0;
@@ -174,25 +213,35 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             run_products += u;
             my_products += u;
             my_max = max(my_max, u);
-            if (cls == CLS_ISM_GLOBAL) my_max_global = max(my_max_global, u);
-            if (cls == CLS_ISM_SMEM) my_max_smem = max(my_max_smem, u);
+            // (rare classes: straight to shared memory, and only when the maximum would move)
+            if (cls == CLS_ISM_GLOBAL && u > s_max_ub_global) atomicMax(&s_max_ub_global, u);
+            if (cls == CLS_ISM_SMEM && u > s_max_ub_smem) atomicMax(&s_max_ub_smem, u);
             if (cls == CLS_DENSE_HUB || cls == CLS_DENSE_CTA || cls == CLS_DENSE_WARP)
                 my_span_words = max(my_span_words, (hi - lo) / 32 + 1);
         }
     }
     if (gl == 0 && run_rows) {
-        atomicAdd(&s_hist[run_cls], run_rows);
-        if (run_products) atomicAdd((u64*)&s_cprod[run_cls], (u64)run_products);
+        atomicAdd(&w_hist[run_cls], run_rows);
+        if (run_products) atomicAdd((u64*)&w_cprod[run_cls], (u64)run_products);
     }
-    if (gl == 0 && my_span_words) atomicMax(&s_max_span_words, my_span_words);
-    if (gl == 0 && my_products) atomicAdd((u64*)&s_products, (u64)my_products);
-    if (gl == 0 && my_max) atomicMax(&s_max_ub, my_max);
-    if (gl == 0 && my_max_global) atomicMax(&s_max_ub_global, my_max_global);
-    if (gl == 0 && my_max_smem) atomicMax(&s_max_ub_smem, my_max_smem);
+    // the totals: reduced over the warp first (lanes other than a group's first hold zeros)
+    for (int d = 16; d > 0; d >>= 1) {
+        my_products += __shfl_xor_sync(0xffffffffu, my_products, d);
+        my_max = max(my_max, __shfl_xor_sync(0xffffffffu, my_max, d));
+        my_span_words = max(my_span_words, __shfl_xor_sync(0xffffffffu, my_span_words, d));
+    }
+    if (lane == 0) {
+        if (my_span_words) atomicMax(&s_max_span_words, my_span_words);
+        if (my_products) atomicAdd((u64*)&s_products, (u64)my_products);
+        if (my_max) atomicMax(&s_max_ub, my_max);
+    }
     __syncthreads();
-    if (threadIdx.x < NCLASS && s_hist[threadIdx.x]) {
-        atomicAdd(&ctl->class_count[threadIdx.x], s_hist[threadIdx.x]);
-        if (s_cprod[threadIdx.x]) atomicAdd((u64*)&ctl->class_products[threadIdx.x], (u64)s_cprod[threadIdx.x]);
+    if (threadIdx.x < NCLASS) {
+        int rows = 0;
+        i64 prods = 0;
+        for (int w = 0; w < 8; ++w) { rows += s_hist[w][threadIdx.x]; prods += s_cprod[w][threadIdx.x]; }
+        if (rows) atomicAdd(&ctl->class_count[threadIdx.x], rows);
+        if (prods) atomicAdd((u64*)&ctl->class_products[threadIdx.x], (u64)prods);
     }
     if (threadIdx.x == 0) {
         if (s_products) atomicAdd((u64*)&ctl->products, (u64)s_products);
@@ -214,9 +263,17 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
     };
     // (one and two lanes per row were measured on the fibre matrix of the 3-tensor workload, 1.06
     // entries per row: slower than four)
-    if (avg <= 6.0) row_bounds_kernel<4><<<grid_for(4), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
-    else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
-    else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl);
+    if (c.brow) {
+        i64 want = ((i64)B.nrows + threads - 1) / threads;
+        i64 cap = (i64)c.sm_count * 8;
+        brow_summary_kernel<<<(int)(want < cap ? want : cap), threads, 0, c.stream>>>(B, c.brow);
+        ++c.launches;
+    }
+    if (avg <= 1.5) row_bounds_kernel<1><<<grid_for(1), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+    else if (avg <= 3.0) row_bounds_kernel<2><<<grid_for(2), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+    else if (avg <= 6.0) row_bounds_kernel<4><<<grid_for(4), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+    else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+    else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
     ++c.launches;
     return cudaGetLastError();
 }
@@ -418,9 +475,6 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
             if (to_warp) {
                 tab.warp_rows[s_wbase + wpos] = row;
                 tab.row_unit0[row] = -1;
-                atomicAdd((u64*)&s_wp, (u64)tab.ub[row]);
-                atomicAdd((u64*)&s_wn, (u64)cnt);
-                atomicMax(&s_wmax, cnt);
             } else {
                 const int u0 = s_ubase + upos;
                 if (u0 + nu > prm.unit_cap) {
@@ -430,6 +484,22 @@ __global__ void __launch_bounds__(256) dense_rebin_kernel(int m, RowTables tab, 
                     tab.row_unit0[row] = u0;
                     for (int t = 0; t < nu; ++t) tab.unit_row[u0 + t] = row;
                 }
+            }
+        }
+        {
+            // products, outputs and largest output count of the warp rows: one shared atomic per warp
+            i64 wp = (row >= 0 && to_warp) ? tab.ub[row] : 0;
+            i64 wn = (row >= 0 && to_warp) ? cnt : 0;
+            int wm = (row >= 0 && to_warp) ? cnt : 0;
+            for (int d = 16; d > 0; d >>= 1) {
+                wp += __shfl_xor_sync(0xffffffffu, wp, d);
+                wn += __shfl_xor_sync(0xffffffffu, wn, d);
+                wm = max(wm, __shfl_xor_sync(0xffffffffu, wm, d));
+            }
+            if ((threadIdx.x & 31) == 0 && wp) {
+                atomicAdd((u64*)&s_wp, (u64)wp);
+                atomicAdd((u64*)&s_wn, (u64)wn);
+                atomicMax(&s_wmax, wm);
             }
         }
         __syncthreads();
@@ -452,21 +522,30 @@ cudaError_t launch_dense_rebin(const LaunchCtx& c, int m, const i64* rowptr) {
     return cudaGetLastError();
 }
 
-// Output entries per class (statistics for the per-kernel byte counts).  Rows are grouped by
-// class in perm, so each class is one contiguous range: sum it with a grid-stride loop and one
-// atomic per warp.
+// Output entries per class (statistics for the per-kernel byte counts): one pass over the rows in
+// row order, every thread keeping a sum per class.
 __global__ void __launch_bounds__(256) class_nnz_kernel(int m, RowTables tab, DevCtl* ctl) {
-    int off = 0;
-    for (int c = 0; c < NCLASS; ++c) {
-        const int n = ctl->class_count[c];
-        if (c != CLS_EMPTY && n > 0) {
-            i64 sum = 0;
-            for (i64 r = (i64)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += (i64)gridDim.x * blockDim.x)
-                sum += tab.cnt[tab.perm[off + r]];
-            for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
-            if ((threadIdx.x & 31) == 0 && sum) atomicAdd((u64*)&ctl->class_nnz[c], (u64)sum);
-        }
-        off += n;
+    i64 sum[NCLASS];
+#pragma unroll
+    for (int k = 0; k < NCLASS; ++k) sum[k] = 0;
+    for (i64 row = (i64)blockIdx.x * blockDim.x + threadIdx.x; row < m; row += (i64)gridDim.x * blockDim.x) {
+        const int c = tab.cls[row];
+        const int v = tab.cnt[row];
+#pragma unroll
+        for (int k = 0; k < NCLASS; ++k) sum[k] += (c == k) ? v : 0;
+    }
+    __shared__ i64 s_part[8][NCLASS];
+#pragma unroll
+    for (int k = 0; k < NCLASS; ++k) {
+        i64 t = sum[k];
+        for (int d = 16; d > 0; d >>= 1) t += __shfl_xor_sync(0xffffffffu, t, d);
+        if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5][k] = t;
+    }
+    __syncthreads();
+    if (threadIdx.x < NCLASS && threadIdx.x != CLS_EMPTY) {
+        i64 t = 0;
+        for (int w = 0; w < 8; ++w) t += s_part[w][threadIdx.x];
+        if (t) atomicAdd((u64*)&ctl->class_nnz[threadIdx.x], (u64)t);
     }
 }
 
@@ -596,18 +675,6 @@ cudaError_t launch_scan_counts(const LaunchCtx& c, const int* cnt, int n, i64* o
 // TTM: rebuild C's two upper CSF levels.  A fibre (i,j) survives when it produced at least
 // one output; a slice i survives when one of its fibres does.
 // ---------------------------------------------------------------------------------------
-__global__ void ttm_fibre_compact_kernel(int n_ij, const int* __restrict__ cnt, const i64* __restrict__ fpos,
-                                         const int* __restrict__ Acrd1, const i64* __restrict__ rowptr_raw,
-                                         int* Ccrd1, i64* Cpos2) {
-    for (i64 f = (i64)blockIdx.x * blockDim.x + threadIdx.x; f <= n_ij; f += (i64)gridDim.x * blockDim.x) {
-        if (f == n_ij) { Cpos2[fpos[n_ij]] = rowptr_raw[n_ij]; continue; }
-        if (cnt[f] > 0) {
-            Ccrd1[fpos[f]] = Acrd1[f];
-            Cpos2[fpos[f]] = rowptr_raw[f];
-        }
-    }
-}
-
 __global__ void ttm_slice_flags_kernel(int n_i, const i64* __restrict__ Apos1, const i64* __restrict__ fpos, int* sflags) {
     for (i64 s = (i64)blockIdx.x * blockDim.x + threadIdx.x; s < n_i; s += (i64)gridDim.x * blockDim.x)
         sflags[s] = fpos[Apos1[s + 1]] > fpos[Apos1[s]];
@@ -639,20 +706,31 @@ __global__ void __launch_bounds__(1024) ttm_slices_small_kernel(int n_i, int n_i
                                                                 DevCtl* ctl) {
     __shared__ int ws[33];
     int kept = 0;
-    for (int s0 = 0; s0 < n_i; s0 += 1024) {
-        const int s = s0 + threadIdx.x;
-        i64 first = 0;
-        int flag = 0;
-        if (s < n_i) {
-            first = fpos[Apos1[s]];
-            flag = fpos[Apos1[s + 1]] > first;
+    // four consecutive slices per thread, their loads issued together (this block is alone on the
+    // GPU, so every dependent load costs a full memory latency)
+    for (int s0 = 0; s0 < n_i; s0 += 4096) {
+        const int s = s0 + 4 * threadIdx.x;
+        i64 edge[5], fp[5];
+#pragma unroll
+        for (int x = 0; x < 5; ++x) edge[x] = (s + x <= n_i) ? Apos1[s + x] : -1;
+#pragma unroll
+        for (int x = 0; x < 5; ++x) fp[x] = edge[x] >= 0 ? fpos[edge[x]] : 0;
+        int crd[4], nflag = 0;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const bool flag = s + x < n_i && fp[x + 1] > fp[x];
+            crd[x] = flag ? Acrd0[s + x] : -1;
+            nflag += flag;
         }
         int total;
-        const int at = kept + block_excl_scan<1024>(flag, ws, total);
-        if (flag) {
-            Ccrd0[at] = Acrd0[s];
-            Cpos1[at] = first;
-        }
+        int at = kept + block_excl_scan<1024>(nflag, ws, total);
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+            if (s + x < n_i && fp[x + 1] > fp[x]) {
+                Ccrd0[at] = crd[x];
+                Cpos1[at] = fp[x];
+                ++at;
+            }
         kept += total;
     }
     if (threadIdx.x == 0) {
@@ -664,23 +742,173 @@ __global__ void __launch_bounds__(1024) ttm_slices_small_kernel(int n_i, int n_i
     }
 }
 
-cudaError_t launch_ttm_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0,
-                               const int* Acrd1, const i64* rowptr_raw, int* flags, i64* fpos, int* sflags,
-                               i64* spos, i64* block_sums, i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2) {
-    (void)flags;
-    const int grid = c.sm_count * 8;
-    // fibres that produced an output keep their place among the survivors: positions by a scan of (cnt > 0)
-    cudaError_t e = launch_scan_counts(c, c.tab.cnt, n_ij, fpos, block_sums, nullptr, true);
-    if (e != cudaSuccess) return e;
-    ttm_fibre_compact_kernel<<<grid, 256, 0, c.stream>>>(n_ij, c.tab.cnt, fpos, Acrd1, rowptr_raw, Ccrd1, Cpos2);
-    ++c.launches;
+// The fibre level in three launches: the scan of the counts (C's bottom-level positions) and the
+// scan of (count > 0) (where a surviving fibre goes) share their passes over the counts, and the
+// second pass places the survivors as it goes.
+__global__ void __launch_bounds__(SCAN_THREADS) ttm_dual_reduce_kernel(const int* __restrict__ cnt, int n, i64* sums, i64* kept) {
+    __shared__ i64 s_part[2][SCAN_THREADS / 32];
+    const i64 base = (i64)blockIdx.x * SCAN_TILE;
+    i64 s = 0;
+    int k = 0;
+    for (int x = 0; x < SCAN_ITEMS; ++x) {
+        const i64 i = base + x * SCAN_THREADS + threadIdx.x;
+        if (i < n) { const int v = cnt[i]; s += v; k += v > 0; }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, d);
+        k += __shfl_xor_sync(0xffffffffu, k, d);
+    }
+    if ((threadIdx.x & 31) == 0) { s_part[0][threadIdx.x >> 5] = s; s_part[1][threadIdx.x >> 5] = k; }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        i64 t = 0;
+        for (int w = 0; w < SCAN_THREADS / 32; ++w) t += s_part[threadIdx.x][w];
+        (threadIdx.x == 0 ? sums : kept)[blockIdx.x] = t;
+    }
+}
+
+// exclusive scans of both block-sum arrays by one block; the totals close the three arrays
+__global__ void __launch_bounds__(1024) ttm_dual_block_sums_kernel(i64* sums, i64* kept, int nblocks, int n, i64* rowptr_raw, i64* fpos,
+                                                                   i64* Cpos2, i64* nnz_out) {
+    __shared__ i64 s_warp[2][32];
+    __shared__ i64 s_carry[2];
+    if (threadIdx.x < 2) s_carry[threadIdx.x] = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < nblocks; base += 1024) {
+        const int i = base + threadIdx.x;
+        const i64 v0 = (i < nblocks) ? sums[i] : 0, v1 = (i < nblocks) ? kept[i] : 0;
+        i64 i0 = v0, i1 = v1;
+        for (int d = 1; d < 32; d <<= 1) {
+            const i64 t0 = __shfl_up_sync(0xffffffffu, i0, d), t1 = __shfl_up_sync(0xffffffffu, i1, d);
+            if (lane >= d) { i0 += t0; i1 += t1; }
+        }
+        if (lane == 31) { s_warp[0][warp] = i0; s_warp[1][warp] = i1; }
+        __syncthreads();
+        if (warp < 2) {
+            const i64 w = s_warp[warp][lane];
+            i64 wi = w;
+            for (int d = 1; d < 32; d <<= 1) {
+                const i64 t = __shfl_up_sync(0xffffffffu, wi, d);
+                if (lane >= d) wi += t;
+            }
+            s_warp[warp][lane] = wi - w;
+        }
+        __syncthreads();
+        const i64 c0 = s_carry[0], c1 = s_carry[1];
+        if (i < nblocks) { sums[i] = c0 + s_warp[0][warp] + i0 - v0; kept[i] = c1 + s_warp[1][warp] + i1 - v1; }
+        __syncthreads();
+        if (threadIdx.x == 1023) { s_carry[0] = c0 + s_warp[0][warp] + i0; s_carry[1] = c1 + s_warp[1][warp] + i1; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        rowptr_raw[n] = s_carry[0];
+        fpos[n] = s_carry[1];
+        Cpos2[s_carry[1]] = s_carry[0];
+        *nnz_out = s_carry[0];
+    }
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) ttm_dual_apply_kernel(const int* __restrict__ cnt, int n, const i64* __restrict__ sums,
+                                                                      const i64* __restrict__ kept, const int* __restrict__ Acrd1,
+                                                                      i64* __restrict__ rowptr_raw, i64* __restrict__ fpos,
+                                                                      int* __restrict__ Ccrd1, i64* __restrict__ Cpos2) {
+    // a thread scans SCAN_ITEMS consecutive counts; everything crosses shared memory on the way in
+    // and out so that global loads and stores are contiguous across the block
+    __shared__ i64 s_a[SCAN_TILE];          // counts on the way in (as int), then one output array at a time
+    __shared__ int s_crd[SCAN_TILE];        // the tile's fibre coordinates, then the survivors'
+    __shared__ i64 s_warp[SCAN_THREADS / 32];
+    __shared__ int s_kwarp[SCAN_THREADS / 32];
+    const i64 tile = (i64)blockIdx.x * SCAN_TILE;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int len = (int)min((i64)SCAN_TILE, (i64)n - tile);
+    int* s_cnt = reinterpret_cast<int*>(s_a);
+    for (int i = tid; i < SCAN_TILE; i += SCAN_THREADS) {
+        s_cnt[i] = i < len ? cnt[tile + i] : 0;
+        s_crd[i] = i < len ? Acrd1[tile + i] : 0;
+    }
+    __syncthreads();
+    int v[SCAN_ITEMS], crd[SCAN_ITEMS];
+    i64 s = 0;
+    int k = 0;
+#pragma unroll
+    for (int x = 0; x < SCAN_ITEMS; ++x) {
+        v[x] = s_cnt[tid * SCAN_ITEMS + x];
+        crd[x] = s_crd[tid * SCAN_ITEMS + x];
+        s += v[x];
+        k += v[x] > 0;
+    }
+    i64 incl = s;
+    int kincl = k;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const i64 t = __shfl_up_sync(0xffffffffu, incl, d);
+        const int tk = __shfl_up_sync(0xffffffffu, kincl, d);
+        if (lane >= d) { incl += t; kincl += tk; }
+    }
+    if (lane == 31) { s_warp[warp] = incl; s_kwarp[warp] = kincl; }
+    __syncthreads();                                      // also: every thread has read s_cnt and s_crd
+    i64 before = 0;
+    int kbefore = 0, ktile = 0;
+#pragma unroll
+    for (int w = 0; w < SCAN_THREADS / 32; ++w) {
+        before += (w < warp) ? s_warp[w] : 0;
+        kbefore += (w < warp) ? s_kwarp[w] : 0;
+        ktile += s_kwarp[w];
+    }
+    const i64 run0 = sums[blockIdx.x] + before + incl - s;
+    const i64 kept0 = kept[blockIdx.x];
+    const int at0 = kbefore + kincl - k;                  // survivors of the tile before this thread's
+    // C's bottom-level positions of all fibres
+    i64 run = run0;
+#pragma unroll
+    for (int x = 0; x < SCAN_ITEMS; ++x) { s_a[tid * SCAN_ITEMS + x] = run; run += v[x]; }
+    __syncthreads();
+    for (int i = tid; i < len; i += SCAN_THREADS) rowptr_raw[tile + i] = s_a[i];
+    __syncthreads();
+    // place of every fibre among the survivors
+    int at = at0;
+#pragma unroll
+    for (int x = 0; x < SCAN_ITEMS; ++x) { s_a[tid * SCAN_ITEMS + x] = kept0 + at; at += v[x] > 0; }
+    __syncthreads();
+    for (int i = tid; i < len; i += SCAN_THREADS) fpos[tile + i] = s_a[i];
+    __syncthreads();
+    // the survivors' coordinates and positions, packed
+    run = run0;
+    at = at0;
+#pragma unroll
+    for (int x = 0; x < SCAN_ITEMS; ++x) {
+        if (v[x] > 0) { s_a[at] = run; s_crd[at] = crd[x]; ++at; }
+        run += v[x];
+    }
+    __syncthreads();
+    for (int i = tid; i < ktile; i += SCAN_THREADS) {
+        Cpos2[kept0 + i] = s_a[i];
+        Ccrd1[kept0 + i] = s_crd[i];
+    }
+}
+
+// Scan of the fibre counts, survivors' positions, C's two lower levels' coordinates and positions,
+// then the slice level.  `block_sums` holds two arrays of one entry per scan tile.
+cudaError_t launch_ttm_scan_compact(const LaunchCtx& c, int n_i, int n_ij, const i64* Apos1, const int* Acrd0, const int* Acrd1,
+                                    i64* rowptr_raw, i64* fpos, int* sflags, i64* spos, i64* block_sums, i64* nnz_out,
+                                    i64* Cpos0, int* Ccrd0, i64* Cpos1, int* Ccrd1, i64* Cpos2) {
+    const int nblocks = (int)(((i64)n_ij + SCAN_TILE - 1) / SCAN_TILE);
+    i64* sums = block_sums;
+    i64* kept = block_sums + nblocks + 1;
+    if (nblocks > 0) ttm_dual_reduce_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(c.tab.cnt, n_ij, sums, kept);
+    ttm_dual_block_sums_kernel<<<1, 1024, 0, c.stream>>>(sums, kept, nblocks, n_ij, rowptr_raw, fpos, Cpos2, nnz_out);
+    if (nblocks > 0)
+        ttm_dual_apply_kernel<<<nblocks, SCAN_THREADS, 0, c.stream>>>(c.tab.cnt, n_ij, sums, kept, Acrd1, rowptr_raw, fpos, Ccrd1, Cpos2);
+    c.launches += nblocks > 0 ? 3 : 1;
     if (n_i <= (1 << 16)) {
         ttm_slices_small_kernel<<<1, 1024, 0, c.stream>>>(n_i, n_ij, Apos1, fpos, Acrd0, Ccrd0, Cpos1, Cpos0, c.ctl);
         ++c.launches;
         return cudaGetLastError();
     }
+    const int grid = c.sm_count * 8;
     ttm_slice_flags_kernel<<<grid, 256, 0, c.stream>>>(n_i, Apos1, fpos, sflags);
-    e = launch_scan_counts(c, sflags, n_i, spos, block_sums, nullptr);
+    cudaError_t e = launch_scan_counts(c, sflags, n_i, spos, block_sums, nullptr);
     if (e != cudaSuccess) return e;
     ttm_slice_compact_kernel<<<grid, 256, 0, c.stream>>>(n_i, n_ij, sflags, spos, Apos1, fpos, Acrd0, Ccrd0, Cpos1, Cpos0, c.ctl);
     c.launches += 2;

@@ -155,13 +155,14 @@ bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 // ---- scratch layout ------------------------------------------------------------------------
 struct Layout {
     size_t ctl, ub, rowptr_raw, cnt, jmin, jmax, cls, perm, bm_off, warp_rows, row_unit0, unit_row, block_sums,
-        flags, fpos, sflags, spos, bw_long, bw, rest, fixed_end;
+        fpos, sflags, spos, bw_long, bw, brow, rest, fixed_end;
+    bool has_brow;
     int unit_cap;
     int bw_long_cap;            // 0: no word lists for this B
     int dense_smem_words;
 };
 
-Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, int64_t nnzB) {
+Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, int64_t nnzB, int64_t k, int64_t nnzA) {
     Layout L{};
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
@@ -186,9 +187,8 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, 
     if (words > DENSE_MAX_SPAN_WORDS) words = DENSE_MAX_SPAN_WORDS;
     L.dense_smem_words = (int)((words + 7) & ~7ll);
     const size_t longest = (size_t)(m > n_i ? m : n_i);
-    L.block_sums = take(8 * (longest / 2048 + 2));
+    L.block_sums = take(16 * (longest / 2048 + 2));     // two arrays for the 3-tensor form's paired scan
     if (p->kind == 1) {
-        L.flags = take(4 * (size_t)m);
         L.fpos = take(8 * ((size_t)m + 1));
         L.sflags = take(4 * (size_t)n_i);
         L.spos = take(8 * ((size_t)n_i + 1));
@@ -199,6 +199,12 @@ Layout make_layout(const spws_plan_s* p, int64_t m, int64_t ncols, int64_t n_i, 
         L.bw_long_cap = (int)(nnzB / BW_MIN_LEN + 1);
         L.bw_long = take(4 * (size_t)L.bw_long_cap);
         L.bw = take(8 * (size_t)nnzB);
+    }
+    // first column, last column and length of every B row, for the bounds kernel: kept when A
+    // picks every B row several times over on average
+    if (k > 0 && nnzA >= 4 * k) {
+        L.has_brow = true;
+        L.brow = take(16 * (size_t)k);
     }
     L.fixed_end = o;
     L.rest = o;
@@ -327,6 +333,7 @@ LaunchCtx make_ctx(const spws_plan_s* p, char* scratch, size_t scratch_bytes, co
         c.bw_long = reinterpret_cast<int*>(scratch + L.bw_long);
         c.bw_long_cap = L.bw_long_cap;
     }
+    if (L.has_brow) c.brow = reinterpret_cast<int4*>(scratch + L.brow);
     return c;
 }
 
@@ -906,7 +913,7 @@ spws_status_t spws_workspace_size(spws_plan_t plan, const spws_tensor_t* A, cons
                  : std::max(OL.ism_end, ((double)S.m * (double)S.ncols <= 134217728.0 || (double)P * 16.0 >= (double)S.m * (double)S.ncols) ? dense_ok : (size_t)0);
         return SPWS_OK;
     }
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB, S.k, S.nnzA);
     *bytes = L.fixed_end + rest_reserve(plan, S.m, S.ncols);
     return SPWS_OK;
 }
@@ -918,7 +925,7 @@ spws_status_t spws_workspace_size_exact(spws_plan_t plan, const spws_tensor_t* A
     Shapes S{};
     spws_status_t st = check_operands(plan, A, B, S, scratch != nullptr);
     if (st != SPWS_OK) return st;
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB, S.k, S.nnzA);
     if (!scratch) {                             // first step of the protocol: what this call itself needs
         *bytes = L.fixed_end;
         return SPWS_OK;
@@ -963,7 +970,7 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
     if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
     if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return SPWS_INVALID_ARGUMENT;
     if (plan->kind == 2) return outer_symbolic(plan, S, C, scratch, scratch_bytes, sizes_out);
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB, S.k, S.nnzA);
     if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
     char* sc = static_cast<char*>(scratch);
     LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
@@ -1026,12 +1033,14 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
             }
     }
     // a4: exclusive scan into the row pointer
-    CUDA_TRY(launch_scan_counts(c, c.tab.cnt, (int)S.m, rowptr, reinterpret_cast<i64*>(sc + L.block_sums), &c.ctl->nnz));
     if (plan->kind == 1) {
-        CUDA_TRY(launch_ttm_compact(c, (int)S.n_i, (int)S.m, LL(A->pos[1]), A->crd[0], A->crd[1], rowptr,
-                                    reinterpret_cast<int*>(sc + L.flags), reinterpret_cast<i64*>(sc + L.fpos),
-                                    reinterpret_cast<int*>(sc + L.sflags), reinterpret_cast<i64*>(sc + L.spos),
-                                    reinterpret_cast<i64*>(sc + L.block_sums), LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
+        // with C's fibre and slice levels rebuilt from the fibres that produced an output
+        CUDA_TRY(launch_ttm_scan_compact(c, (int)S.n_i, (int)S.m, LL(A->pos[1]), A->crd[0], A->crd[1], rowptr,
+                                         reinterpret_cast<i64*>(sc + L.fpos), reinterpret_cast<int*>(sc + L.sflags),
+                                         reinterpret_cast<i64*>(sc + L.spos), reinterpret_cast<i64*>(sc + L.block_sums), &c.ctl->nnz,
+                                         LL(C->pos[0]), C->crd[0], LL(C->pos[1]), C->crd[1], LL(C->pos[2])));
+    } else {
+        CUDA_TRY(launch_scan_counts(c, c.tab.cnt, (int)S.m, rowptr, reinterpret_cast<i64*>(sc + L.block_sums), &c.ctl->nnz));
     }
     if (hcount[CLS_DENSE_WARP] + hcount[CLS_DENSE_HUB] + hcount[CLS_DENSE_CTA] > 0) CUDA_TRY(launch_dense_rebin(c, (int)S.m, rowptr));
     CUDA_TRY(launch_class_nnz(c, (int)S.m));
@@ -1091,7 +1100,7 @@ spws_status_t spws_numeric(spws_plan_t plan, const spws_tensor_t* A, const spws_
     const int last = plan->kind == 0 ? 1 : 2;
     if (C->n[last] < plan->stats.nnz) return SPWS_OUTPUT_TOO_SMALL;
     if (plan->stats.nnz > 0 && (!C->crd[last] || !C->val)) return SPWS_INVALID_ARGUMENT;
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB, S.k, S.nnzA);
     if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
     char* sc = static_cast<char*>(scratch);
     LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
@@ -1148,7 +1157,7 @@ spws_status_t spws_gather_ceiling(spws_plan_t plan, const spws_tensor_t* A, cons
     if (st != SPWS_OK) return st;
     if ((st = check_output_dims(plan, A, B, C)) != SPWS_OK) return st;
     if (scratch != plan->scratch || S.m != plan->m) return SPWS_BAD_SEQUENCE;
-    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB);
+    const Layout L = make_layout(plan, S.m, S.ncols, S.n_i, S.nnzB, S.k, S.nnzA);
     if (scratch_bytes < L.fixed_end) return SPWS_SCRATCH_TOO_SMALL;
     char* sc = static_cast<char*>(scratch);
     LaunchCtx c = make_ctx(plan, sc, scratch_bytes, L);
