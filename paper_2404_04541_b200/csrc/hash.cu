@@ -18,8 +18,8 @@ constexpr int HASH_EMPTY = -1;
 
 template <typename T, int CAP, int THREADS, bool NUMERIC>
 __global__ void __launch_bounds__(THREADS) hash_kernel(const int* __restrict__ perm, DevCtl* __restrict__ ctl, int cls, int counter_slot,
-                                                       Csr A, Csr B, int* __restrict__ cnt, const i64* __restrict__ rowptr,
-                                                       int* __restrict__ Ccrd, T* __restrict__ Cval) {
+                                                       Csr A, Csr B, const i64* __restrict__ ub, int* __restrict__ cnt,
+                                                       const i64* __restrict__ rowptr, int* __restrict__ Ccrd, T* __restrict__ Cval) {
     constexpr int SLOTS = 2 * CAP;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* vals = reinterpret_cast<T*>(smem_raw);                             // SLOTS (numeric only)
@@ -48,14 +48,17 @@ __global__ void __launch_bounds__(THREADS) hash_kernel(const int* __restrict__ p
         const int row = rows[r];
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
         // the numeric pass knows the row's distinct columns and sizes the table from them
-        int slots = SLOTS;
+        // (the counting pass sizes it from the row's product count, an upper bound of them)
+        int slots = 16;
         i64 out0 = 0;
         int row_cnt = 0;
         if (NUMERIC) {
             out0 = rowptr[row];
             row_cnt = min((int)(rowptr[row + 1] - out0), CAP);
-            slots = 16;
             while (slots < 2 * row_cnt) slots <<= 1;
+        } else {
+            const int bound = (int)min(ub[row], (i64)CAP);
+            while (slots < 2 * bound) slots <<= 1;
         }
         const unsigned mask = (unsigned)slots - 1u;
         const int shift = 32 - __popc(mask);
@@ -173,7 +176,7 @@ static cudaError_t hash_launch_k(const LaunchCtx& c, int cls, int n_host, const 
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, THREADS, smem)) != cudaSuccess) return e;
     i64 grid = (i64)c.sm_count * (per_sm > 0 ? per_sm : 1);
     if (n_host >= 0 && n_host < grid) grid = n_host > 0 ? n_host : 1;
-    k<<<(int)grid, THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, cls, slot, A, B, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
+    k<<<(int)grid, THREADS, smem, c.stream>>>(c.tab.perm, c.ctl, cls, slot, A, B, c.tab.ub, c.tab.cnt, rowptr, Ccrd, (T*)Cval);
     ++c.launches;
     return cudaGetLastError();
 }
@@ -181,6 +184,10 @@ static cudaError_t hash_launch_k(const LaunchCtx& c, int cls, int n_host, const 
 template <typename T>
 static cudaError_t hash_launch_t(const LaunchCtx& c, bool numeric, int cls, int n_host, const Csr& A, const Csr& B, const i64* rowptr,
                                  int* Ccrd, void* Cval) {
+    // the counting pass also serves the shared-memory insert-sort-merge classes (no sort is needed to
+    // count distinct columns); their rows have at most HASH_CAP products
+    if (!numeric && cls == CLS_ISM_SMEM_S) return hash_launch_k<T, HASH_SMALL_CAP, 128, false>(c, cls, n_host, A, B, rowptr, Ccrd, Cval);
+    if (!numeric && cls == CLS_ISM_SMEM) return hash_launch_k<T, HASH_CAP, 256, false>(c, cls, n_host, A, B, rowptr, Ccrd, Cval);
     if (cls == CLS_HASH_S)
         return numeric ? hash_launch_k<T, HASH_SMALL_CAP, 128, true>(c, cls, n_host, A, B, rowptr, Ccrd, Cval)
                        : hash_launch_k<T, HASH_SMALL_CAP, 128, false>(c, cls, n_host, A, B, rowptr, Ccrd, Cval);

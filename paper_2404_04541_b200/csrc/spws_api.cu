@@ -1006,12 +1006,17 @@ spws_status_t spws_symbolic(spws_plan_t plan, const spws_tensor_t* A, const spws
                 CUDA_TRY(launch_ism_reg(c, false, cls, hcount[cls], S.A, S.B, rowptr, nullptr, nullptr));
                 mark(plan, SPWS_T_SYM_ISM_REG);
             }
+        // under `auto` the rows of the shared-memory insert-sort-merge classes are counted through a
+        // hash set of their columns: the count needs no order
+        const bool count_by_hash = plan->policy == SPWS_AUTO;
         if (hcount[CLS_ISM_SMEM_S] > 0) {
-            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, hcount[CLS_ISM_SMEM_S], S.A, S.B, rowptr, nullptr, nullptr));
+            if (count_by_hash) CUDA_TRY(launch_hash(c, false, CLS_ISM_SMEM_S, hcount[CLS_ISM_SMEM_S], S.A, S.B, rowptr, nullptr, nullptr));
+            else CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM_S, hcount[CLS_ISM_SMEM_S], S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_SMEM_S);
         }
         if (hcount[CLS_ISM_SMEM] > 0) {
-            CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, hcount[CLS_ISM_SMEM], S.A, S.B, rowptr, nullptr, nullptr));
+            if (count_by_hash) CUDA_TRY(launch_hash(c, false, CLS_ISM_SMEM, hcount[CLS_ISM_SMEM], S.A, S.B, rowptr, nullptr, nullptr));
+            else CUDA_TRY(launch_ism_smem(c, false, CLS_ISM_SMEM, hcount[CLS_ISM_SMEM], S.A, S.B, rowptr, nullptr, nullptr));
             mark(plan, SPWS_T_SYM_ISM_SMEM);
         }
         if (hcount[CLS_DENSE_WARP] > 0) {
