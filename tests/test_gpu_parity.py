@@ -227,6 +227,21 @@ def test_warp_dense_route_compact_and_full_bitmaps(ctx, oracle_mod):
     assert 0 < stats["dense_warp_rows"] < 72 and stats["dense_units"] > 0
 
 
+@pytest.mark.parametrize("summaries", [True, False])
+@pytest.mark.parametrize("per_row", [1, 2, 5, 10, 20])
+def test_bounds_kernel_widths_with_and_without_b_row_summaries(ctx, oracle_mod, per_row, summaries):
+    """The bounds kernel gives a row 1, 2, 4, 8 or 32 lanes by A's mean row length, and reads per-B-row
+    summaries (first / last column, length) when A has at least four entries per B row, else B's own
+    arrays: every combination against the oracle, B with empty rows."""
+    m = 3000
+    k = 500 if summaries else 40000
+    assert (m * per_row >= 4 * k) == summaries
+    A = uniform_rows_csr(m, k, per_row, 11 + per_row)
+    B = random_csr(k, 6000, 0.002, 12 + per_row, empty_row_frac=0.25)
+    for policy in ("auto", "dense"):
+        check_spgemm(ctx, oracle_mod, A, B, policy)
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_randomized_shapes_policies_and_thresholds(ctx, oracle_mod, seed):
     """Seeded random sweep: shapes from 1 x 1 to a few thousand rows and up to 2^20 columns, uniform /
@@ -697,6 +712,17 @@ def test_ttm_config(ctx, oracle_mod, reduced, policy):
     c = config_inputs("ttm4096", reduced=reduced)
     stats = check_ttm(ctx, oracle_mod, c["A"], c["B"], policy)
     assert stats["products"] == 8 * c["A"].nnz
+
+
+@pytest.mark.parametrize("slices", [4097, 9001, 70001])
+def test_ttm_many_slices_and_dropped_fibres(ctx, oracle_mod, slices):
+    """Slice levels of one and several 4096-slice rounds with a ragged tail, and beyond 2^16 slices
+    (the multi-launch slice level); half of B's rows are empty, so many fibres and slices produce no
+    output and drop out of C's upper levels; the fibre count spans several scan tiles."""
+    A = uniform_csf3((slices, 50, 64), 3 * slices, 21)
+    B = random_csr(64, 400, 0.05, 22, empty_row_frac=0.5)
+    stats = check_ttm(ctx, oracle_mod, A, B, "auto")
+    assert stats["rows"] > 2048
 
 
 def test_ttm_equals_spgemm_of_the_fibre_matrix(ctx):
