@@ -50,11 +50,18 @@ def uniform_rows_csr(nrows: int, ncols: int, d: int, seed: int, lo=-1.0, hi=1.0,
         e = min(nrows, s + step)
         blk = rng.integers(0, ncols, size=(e - s, d), dtype=np.int32)
         blk.sort(axis=1)
+        rounds = 0
         while d > 1:
             bad = np.nonzero((blk[:, 1:] == blk[:, :-1]).any(axis=1))[0]
             if bad.size == 0:
                 break
-            redo = rng.integers(0, ncols, size=(bad.size, d), dtype=np.int32)
+            rounds += 1
+            if rounds > 64:
+                # d is close to ncols: redrawing would go on for ever; take the first d of a
+                # random permutation of the columns instead
+                redo = np.argsort(rng.random((bad.size, ncols)), axis=1)[:, :d].astype(np.int32)
+            else:
+                redo = rng.integers(0, ncols, size=(bad.size, d), dtype=np.int32)
             redo.sort(axis=1)
             blk[bad] = redo
         crd[s:e] = blk
