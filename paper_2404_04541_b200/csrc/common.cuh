@@ -45,6 +45,7 @@ constexpr int DENSE_MAX_SPAN_WORDS = 16384;// 2^19 columns: the widest bitmap (8
 // Word lists of long B rows (symbolic pass of the CTA dense route): a B row with at least
 // BW_MIN_LEN entries whose entries share bitmap words is also kept as (word index, bits) pairs,
 // so that a row that picks it sets one word per pair instead of one bit per entry.
+constexpr int LONG_A_ROW = 1024;     // entries of an A row beyond which a whole CTA computes its bounds
 constexpr int BW_MIN_LEN = 256;
 constexpr i64 BW_MAX_NNZ = 1ll << 26;      // lists are built only for a B with at most this many entries
 
@@ -71,6 +72,7 @@ struct DevCtl {
     int max_span_words;     // widest bitmap among the dense rows
     int max_warp_cnt;       // most outputs of a row the warp numeric kernel takes
     int n_long;             // B rows with at least BW_MIN_LEN entries (candidates for a word list)
+    int n_long_a;           // rows of A with more than LONG_A_ROW entries, left to the bounds kernel for long rows
     int class_count[NCLASS];
     int class_cursor[NCLASS];
     int work_counter[N_WORK_COUNTERS];   // dynamic work distribution; cleared before each pass

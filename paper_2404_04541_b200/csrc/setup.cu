@@ -95,7 +95,9 @@ __global__ void __launch_bounds__(256) brow_summary_kernel(Csr B, int4* __restri
     }
 }
 
-template <int G>
+// SUMMARY: brow holds the B-row summaries (the instantiation without them carries B's own arrays'
+// two-level gathers and needs more registers).
+template <int G, bool SUMMARY>
 __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl,
                                                          const int4* __restrict__ brow) {
     // rows and products per class, one histogram per warp: 64-bit shared-memory adds are
@@ -121,6 +123,13 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
     i64 run_products = 0;
     for (i64 row = group; row < A.nrows; row += ngroups) {
         const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        if (pe - ps > LONG_A_ROW) {
+            // a very long row would be this group's serial chain and set the kernel's time on power-law
+            // inputs: it is listed for the kernel that gives such rows a CTA each (the list borrows the
+            // table of warp rows, which is not in use before the numeric routing)
+            if (gl == 0) tab.warp_rows[atomicAdd(&ctl->n_long_a, 1)] = (int)row;
+            continue;
+        }
         i64 u = 0;
         int lo = 0x7fffffff, hi = -1;
         bool bad = false;
@@ -131,7 +140,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
             if (p0 < pe) {
                 const int k = __ldg(A.crd + p0);
                 if ((unsigned)k < (unsigned)B.nrows) {
-                    if (brow) {
+                    if (SUMMARY) {
                         const int4 s = __ldg(brow + k);
                         u = s.z;
                         lo = s.x;
@@ -152,14 +161,13 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
         }
         for (; p0 < pe; p0 += 4 * G) {
             int k[4];
-            i64 qs[4], qe[4];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const i64 p = p0 + (i64)x * G;
                 k[x] = p < pe ? __ldg(A.crd + p) : -1;
                 if (p < pe && (unsigned)k[x] >= (unsigned)B.nrows) bad = true;
             }
-            if (brow) {
+            if (SUMMARY) {
 #pragma unroll
                 for (int x = 0; x < 4; ++x)
                     if ((unsigned)k[x] < (unsigned)B.nrows) {
@@ -170,6 +178,7 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
                     }
                 continue;
             }
+            i64 qs[4], qe[4];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 qs[x] = qe[x] = 0;
@@ -252,6 +261,84 @@ __global__ void __launch_bounds__(256) row_bounds_kernel(Csr A, Csr B, RowTables
     }
 }
 
+// Bounds and class of the listed long rows, a CTA per row: 256 lanes across the entries, four
+// entries per lane and step.
+template <bool SUMMARY>
+__global__ void __launch_bounds__(256) row_bounds_long_kernel(Csr A, Csr B, RowTables tab, ClassParams prm, DevCtl* ctl,
+                                                              const int4* __restrict__ brow) {
+    __shared__ i64 s_u[8];
+    __shared__ int s_lo[8], s_hi[8], s_bad[8];
+    const int n = min(ctl->n_long_a, A.nrows);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int r = blockIdx.x; r < n; r += gridDim.x) {
+        const int row = tab.warp_rows[r];
+        const i64 ps = A.pos[row], pe = A.pos[row + 1];
+        i64 u = 0;
+        int lo = 0x7fffffff, hi = -1, bad = 0;
+        for (i64 p0 = ps + tid; p0 < pe; p0 += 4 * 256) {
+            int k[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const i64 p = p0 + (i64)x * 256;
+                k[x] = p < pe ? __ldg(A.crd + p) : -1;
+                if (p < pe && (unsigned)k[x] >= (unsigned)B.nrows) bad = 1;
+            }
+            if (SUMMARY) {
+                int4 s[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) s[x] = (unsigned)k[x] < (unsigned)B.nrows ? __ldg(brow + k[x]) : make_int4(0x7fffffff, -1, 0, 0);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) { u += s[x].z; lo = min(lo, s[x].x); hi = max(hi, s[x].y); }
+            } else {
+                i64 qs[4], qe[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    qs[x] = qe[x] = 0;
+                    if ((unsigned)k[x] < (unsigned)B.nrows) { qs[x] = __ldg(B.pos + k[x]); qe[x] = __ldg(B.pos + k[x] + 1); }
+                }
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+                    if (qe[x] > qs[x]) {
+                        u += qe[x] - qs[x];
+                        lo = min(lo, __ldg(B.crd + qs[x]));
+                        hi = max(hi, __ldg(B.crd + qe[x] - 1));
+                    }
+            }
+        }
+        for (int d = 16; d > 0; d >>= 1) {
+            u += __shfl_xor_sync(0xffffffffu, u, d);
+            lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+            hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+            bad |= __shfl_xor_sync(0xffffffffu, bad, d);
+        }
+        __syncthreads();                                   // the previous row's totals have been read
+        if (lane == 0) { s_u[warp] = u; s_lo[warp] = lo; s_hi[warp] = hi; s_bad[warp] = bad; }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < 8; ++w) { u += s_u[w]; lo = min(lo, s_lo[w]); hi = max(hi, s_hi[w]); bad |= s_bad[w]; }
+            if (bad) raise_status(ctl, DEV_NONCANONICAL);
+            if (lo < 0 || hi >= B.ncols) { raise_status(ctl, DEV_NONCANONICAL); u = 0; }
+            if (u > 0) lo &= ~31;
+            const int cls = classify_row(u, pe - ps, lo, hi, prm, ctl);
+            tab.ub[row] = u;
+            tab.jmin[row] = lo;
+            tab.jmax[row] = hi;
+            tab.cnt[row] = cls == CLS_COPY8 ? (int)u : 0;
+            tab.cls[row] = (unsigned char)cls;
+            atomicAdd(&ctl->class_count[cls], 1);
+            if (u) {
+                atomicAdd((u64*)&ctl->class_products[cls], (u64)u);
+                atomicAdd((u64*)&ctl->products, (u64)u);
+                atomicMax(&ctl->max_ub, u);
+                if (cls == CLS_ISM_GLOBAL) atomicMax(&ctl->max_ub_global, u);
+                if (cls == CLS_ISM_SMEM) atomicMax(&ctl->max_ub_smem, u);
+                if (cls == CLS_DENSE_HUB || cls == CLS_DENSE_CTA || cls == CLS_DENSE_WARP)
+                    atomicMax(&ctl->max_span_words, (hi - lo) / 32 + 1);
+            }
+        }
+    }
+}
+
 cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i64 nnzA) {
     if (A.nrows == 0) return cudaSuccess;
     const double avg = (double)nnzA / (double)A.nrows;
@@ -269,12 +356,23 @@ cudaError_t launch_row_bounds(const LaunchCtx& c, const Csr& A, const Csr& B, i6
         brow_summary_kernel<<<(int)(want < cap ? want : cap), threads, 0, c.stream>>>(B, c.brow);
         ++c.launches;
     }
-    if (avg <= 1.5) row_bounds_kernel<1><<<grid_for(1), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
-    else if (avg <= 3.0) row_bounds_kernel<2><<<grid_for(2), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
-    else if (avg <= 6.0) row_bounds_kernel<4><<<grid_for(4), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
-    else if (avg <= 12.0) row_bounds_kernel<8><<<grid_for(8), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
-    else row_bounds_kernel<32><<<grid_for(32), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+    auto launch = [&](auto kernel, int G) { kernel<<<grid_for(G), threads, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow); };
+    const bool sm = c.brow != nullptr;
+    if (avg <= 1.5) sm ? launch(row_bounds_kernel<1, true>, 1) : launch(row_bounds_kernel<1, false>, 1);
+    else if (avg <= 3.0) sm ? launch(row_bounds_kernel<2, true>, 2) : launch(row_bounds_kernel<2, false>, 2);
+    else if (avg <= 6.0) sm ? launch(row_bounds_kernel<4, true>, 4) : launch(row_bounds_kernel<4, false>, 4);
+    else if (avg <= 12.0) sm ? launch(row_bounds_kernel<8, true>, 8) : launch(row_bounds_kernel<8, false>, 8);
+    else sm ? launch(row_bounds_kernel<32, true>, 32) : launch(row_bounds_kernel<32, false>, 32);
     ++c.launches;
+    // rows the kernel above listed as too long for a lane group (none, unless A has more than
+    // LONG_A_ROW entries in all)
+    if (nnzA > LONG_A_ROW) {
+        const i64 most = nnzA / LONG_A_ROW;
+        const int grid = (int)(most < (i64)c.sm_count * 4 ? most : (i64)c.sm_count * 4);
+        if (sm) row_bounds_long_kernel<true><<<grid, 256, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+        else row_bounds_long_kernel<false><<<grid, 256, 0, c.stream>>>(A, B, c.tab, c.prm, c.ctl, c.brow);
+        ++c.launches;
+    }
     return cudaGetLastError();
 }
 

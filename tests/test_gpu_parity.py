@@ -242,6 +242,31 @@ def test_bounds_kernel_widths_with_and_without_b_row_summaries(ctx, oracle_mod, 
         check_spgemm(ctx, oracle_mod, A, B, policy)
 
 
+@pytest.mark.parametrize("summaries", [True, False])
+def test_bounds_of_rows_with_thousands_of_entries(ctx, oracle_mod, summaries):
+    """Rows of A with more than 1024 entries get a CTA each in the bounds pass (listed by the lane-group
+    kernel, which skips them): a few such rows of different lengths among short and empty ones, at the
+    1024 / 1025 edge too, B with empty rows, with the per-B-row summaries and without."""
+    k = 7000
+    rng = np.random.default_rng(5)
+    lengths = [0, 3, 1024, 1025, 0, 6999, 17, 2500, 1, 4097] + [int(x) for x in rng.integers(0, 40, 300)]
+    rows, cols = [], []
+    for i, n in enumerate(lengths):
+        rows.append(np.full(n, i))
+        cols.append(np.sort(rng.choice(k, n, replace=False)))
+    rows, cols = np.concatenate(rows), np.concatenate(cols)
+    A = CSR.from_coo(len(lengths), k, rows, cols, rng.uniform(-1, 1, rows.size))
+    if summaries:                                   # at least four A entries per B row: stack A on itself
+        reps = 4 * k // A.nnz + 1
+        A = CSR.from_coo(reps * len(lengths), k, np.concatenate([rows + r * len(lengths) for r in range(reps)]),
+                         np.tile(cols, reps), rng.uniform(-1, 1, reps * rows.size))
+    assert (A.nnz >= 4 * k) == summaries
+    B = random_csr(k, 3000, 0.003, 6, empty_row_frac=0.3)
+    for policy in ("auto", "dense"):
+        stats = check_spgemm(ctx, oracle_mod, A, B, policy)
+        assert stats["rows"] == A.nrows
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_randomized_shapes_policies_and_thresholds(ctx, oracle_mod, seed):
     """Seeded random sweep: shapes from 1 x 1 to a few thousand rows and up to 2^20 columns, uniform /
